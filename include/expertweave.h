@@ -1,0 +1,190 @@
+/*
+ * expertweave.h - C ABI of the B200 (sm_100a) adapter-aware MoE layer forward of ExpertWeave.
+ *
+ * The library serves many ESFT adapters over one shared MoE base model.  All expert weights of a
+ * layer live in ONE slot-indexed pool per stacked linear (the "virtual weight tensor" of Section 4.1:
+ * first dimension M + N*E_max, base experts first, then E_max reserved slots per adapter), whose
+ * virtual address range is contiguous while physical pages are mapped only under live experts
+ * (Section 4.2).  A forward call takes a mixed batch of tokens, each tagged with an adapter id
+ * (-1 = base model, Section 4.3), routes them with the base router, rewrites the routed expert ids
+ * through the per-layer ESFT expert map Pi (batched rerouting, Section 4.1/4.3), and runs the usual
+ * dispatch -> grouped expert FFN -> weighted combine (Section 2.1) over the pool.
+ *
+ * Conventions
+ *   - Every function returns ew_status_t.  Nothing throws, aborts or traps the device.
+ *   - "host" / "device" in a parameter comment says where the pointer must live.
+ *   - bf16 tensors are passed as void* to raw 16-bit patterns, row-major, innermost dimension
+ *     contiguous.  int32 and float are the C types.
+ *   - One pool may be used by one host thread at a time.  Forward calls on one pool share one
+ *     workspace: issue them on one stream (or order them yourself).
+ *   - H and I must be multiples of 8 (16-byte rows); M <= 256; top_k <= 32 and <= M.
+ */
+#ifndef EXPERTWEAVE_H_
+#define EXPERTWEAVE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ew_pool ew_pool_t; /* opaque; created and destroyed by the library */
+
+typedef enum {
+    EW_OK = 0,
+    EW_ERR_INVALID_ARG = 1,      /* null pointer, size out of range, bad configuration             */
+    EW_ERR_OOM = 2,              /* device memory or the page budget is exhausted                  */
+    EW_ERR_SLOT_IN_USE = 3,      /* ew_load_adapter on an adapter id that is already loaded        */
+    EW_ERR_NOT_LOADED = 4,       /* ew_unload_adapter on an id that is not loaded; forward before ew_load_base */
+    EW_ERR_TOO_MANY_EXPERTS = 5, /* an adapter tunes more than E_max experts in some layer         */
+    EW_ERR_CUDA = 6,             /* a CUDA call failed; ew_last_error_string() has the detail      */
+    EW_ERR_TIMEOUT = 7,          /* a bounded device-side wait expired (reported by ew_last_device_error) */
+    EW_ERR_BAD_ADAPTER_ID_IN_BATCH = 8, /* some token carried an id outside [-1,N) or of an unloaded adapter */
+    EW_ERR_NO_DEVICE = 9         /* the call needs a GPU and the pool is an accounting-only pool   */
+} ew_status_t;
+
+/* Pool configuration (Section 3.1: N = adapters servable in one batch, E_max = slots per adapter). */
+typedef struct {
+    int32_t device;        /* CUDA device ordinal; -1 = accounting-only pool: the page bookkeeping of
+                              Section 4.2 runs, no device memory is touched, forward calls fail with
+                              EW_ERR_NO_DEVICE (for capacity planning and host-side tests)          */
+    int32_t num_layers;    /* L  MoE layers held by this pool                                      */
+    int32_t hidden;        /* H                                                                    */
+    int32_t inter;         /* I  expert intermediate size (SwiGLU: gate and up are [I,H], down [H,I]) */
+    int32_t num_experts;   /* M  routed experts of the base model                                  */
+    int32_t num_shared;    /* S  shared experts (always active, weight 1, never rerouted)          */
+    int32_t top_k;         /* k                                                                    */
+    int32_t max_adapters;  /* N                                                                    */
+    int32_t e_max;         /* E_max                                                                */
+    int32_t max_tokens;    /* largest n_tokens a forward call may pass (sizes the workspace)       */
+    int32_t renormalize;   /* 0: combine weights are the selected softmax probabilities; 1: divided by their sum */
+    float routed_scale;    /* multiplies the k combine weights (1.0 for the DeepSeek-V2-Lite shape) */
+    int32_t pool_mode;     /* 0: pages mapped on demand under live experts (Section 4.2)
+                              1: "padding" baseline of Section 3.1: the whole tensor is backed at creation */
+    int32_t reserved0;
+    uint64_t page_bytes;   /* physical page size; 0 = the driver's minimum granularity (2 MiB on B200);
+                              otherwise a multiple of it                                            */
+    uint64_t prealloc_pages; /* pages created up front and kept in the pool's free list            */
+    uint64_t max_pages;    /* 0 = unlimited; else creating more pages than this fails with EW_ERR_OOM */
+} ew_config_t;
+
+/* Memory accounting (Section 4.2; Section 3.1's F_mem is padding_bytes / live_expert_bytes). */
+typedef struct {
+    uint64_t page_bytes;
+    uint64_t va_reserved_bytes;   /* sum of the virtual ranges of all virtual weight tensors        */
+    uint64_t pages_mapped;        /* pages currently mapped under some live expert                  */
+    uint64_t pages_free;          /* created, unmapped, waiting in the pool's free list             */
+    uint64_t pages_created_total; /* pages ever created (reuse keeps this flat under churn)         */
+    uint64_t physical_bytes;      /* (pages_mapped + pages_free) * page_bytes                       */
+    uint64_t live_expert_bytes;   /* bytes of the experts that are loaded (base + adapters + shared) */
+    uint64_t padding_bytes;       /* what a fully backed [M + N*E_max (+S)] tensor would take       */
+    uint64_t live_experts;        /* routed base + adapter experts currently loaded, over all layers */
+    uint64_t adapters_loaded;
+    uint64_t workspace_bytes;
+} ew_stats_t;
+
+/* Create a pool: reserves, per layer and per stacked linear (gate|up fused as one tensor, down as
+ * another), a contiguous virtual range for M + N*E_max slots (+S trailing slots that hold the shared
+ * experts and are never addressed by the expert map) and maps nothing (Section 4.2, "reserves the
+ * contiguous virtual address space ... without mapping any physical memory page"); allocates the
+ * expert maps (identity rows), router storage and the forward workspace for cfg->max_tokens.
+ * Errors: EW_ERR_INVALID_ARG (bad sizes), EW_ERR_OOM, EW_ERR_CUDA.  *out is set only on EW_OK. */
+ew_status_t ew_pool_create(const ew_config_t *cfg, ew_pool_t **out);
+
+/* Unmaps and releases everything.  Blocks until forwards issued earlier have finished. */
+ew_status_t ew_pool_destroy(ew_pool_t *pool);
+
+/* Load the base model's weights of one layer: the range [0, M) of the pool plus the shared experts
+ * (Section 4.2: "loading of a range of consecutive experts, either from the base model at system
+ * initialization time or from an adapter at runtime").  All pointers are HOST bf16:
+ *   router_w [M,H]; w_gate, w_up [M,I,H]; w_down [M,H,I]; sh_gate, sh_up [S,I,H]; sh_down [S,H,I]
+ * (the sh_* pointers may be null when S = 0).  Data is copied before the call returns; the caller
+ * keeps ownership.  Calling it again for the same layer overwrites the weights in place. */
+ew_status_t ew_load_base(ew_pool_t *pool, int32_t layer, const void *router_w, const void *w_gate,
+                         const void *w_up, const void *w_down, const void *sh_gate, const void *sh_up,
+                         const void *sh_down);
+
+/* Load ESFT adapter `adapter_id` in [0,N) (Sections 4.1-4.2).
+ *   counts      host int32 [L]: e_i^(l), experts the adapter re-tunes in layer l (0 allowed)
+ *   expert_ids  host int32 [sum counts]: per layer, strictly ascending base expert ids in [0,M);
+ *               the r-th id of a layer gets delta = r, i.e. slot M + adapter_id*E_max + r
+ *   w_gate,w_up host bf16 [sum counts, I, H];  w_down host bf16 [sum counts, H, I], same order
+ * For each layer the byte range of slots [Delta_i, Delta_i + e) is backed by pages taken from the
+ * pool's free list (or created); a page shared with a neighbouring adapter is mapped once and
+ * reference-counted (sub-page allocation).  Weights are copied, then row adapter_id of every layer's
+ * expert map is published.  All-or-nothing: on any error every page mapped by this call is unmapped
+ * again and the maps are untouched.
+ * Errors: EW_ERR_INVALID_ARG, EW_ERR_SLOT_IN_USE, EW_ERR_TOO_MANY_EXPERTS, EW_ERR_OOM, EW_ERR_CUDA. */
+ew_status_t ew_load_adapter(ew_pool_t *pool, int32_t adapter_id, const int32_t *counts,
+                            const int32_t *expert_ids, const void *w_gate, const void *w_up,
+                            const void *w_down);
+
+/* Evict an adapter: its expert-map rows return to identity, the call then waits for every forward
+ * issued before it, and pages whose reference count drops to zero are unmapped and returned to the
+ * pool's free list for reuse (Section 4.2).  Errors: EW_ERR_INVALID_ARG, EW_ERR_NOT_LOADED. */
+ew_status_t ew_unload_adapter(ew_pool_t *pool, int32_t adapter_id);
+
+/* Release the free list's pages back to the driver ("eventually reclaimed", Section 4.2). */
+ew_status_t ew_pool_trim(ew_pool_t *pool);
+
+/* The adapter-aware MoE layer forward (Sections 2.1, 4.1, 4.3), asynchronous on `cuda_stream`:
+ *   softmax router + top-k over the M base experts (ties to the lower index)
+ *   -> batched rerouting  slot = adapter_ids[t] < 0 ? id : Pi[layer][adapter_ids[t]][id]
+ *   -> per-slot token counts, permutation into slot-contiguous rows
+ *   -> grouped SwiGLU FFN over the live slots and the shared experts (fp32 accumulation)
+ *   -> out[t] = sum_j w[t,j] * FFN_slot(t,j)(x[t]) + sum_shared FFN(x[t]), rounded once to bf16.
+ *   x            device bf16 [n_tokens, H], 16-byte aligned
+ *   adapter_ids  device int32 [n_tokens]; values outside [-1,N) or naming an adapter that is not
+ *                loaded are treated as -1 and raise EW_ERR_BAD_ADAPTER_ID_IN_BATCH in the device
+ *                error word (ew_last_device_error)
+ *   out          device bf16 [n_tokens, H]
+ *   cuda_stream  a cudaStream_t (null = the legacy default stream)
+ * No host synchronisation; token counts never leave the device.  n_tokens = 0 is a no-op.
+ * Errors: EW_ERR_INVALID_ARG (null, layer out of range, n_tokens > max_tokens), EW_ERR_NOT_LOADED,
+ * EW_ERR_NO_DEVICE, EW_ERR_CUDA (launch failure). */
+ew_status_t ew_moe_forward(ew_pool_t *pool, int32_t layer, const void *x, const int32_t *adapter_ids,
+                           int32_t n_tokens, void *out, void *cuda_stream);
+
+/* Same forward, also copying intermediate results to optional DEVICE buffers (null = skip):
+ *   topk_ids [n_tokens,k] int32 base expert ids, in (probability descending, index ascending) order
+ *   topk_w   [n_tokens,k] float combine weights, same order
+ *   slot_ids [n_tokens,k] int32 after rerouting
+ *   counts   [M + N*E_max] int32 tokens per slot
+ *   inv      [n_tokens,k] int32 row of pair (t,j) in the slot-contiguous order
+ *   offsets  [M + N*E_max + 1] int32 exclusive scan of counts                                      */
+ew_status_t ew_moe_forward_debug(ew_pool_t *pool, int32_t layer, const void *x, const int32_t *adapter_ids,
+                                 int32_t n_tokens, void *out, void *cuda_stream, int32_t *topk_ids,
+                                 float *topk_w, int32_t *slot_ids, int32_t *counts, int32_t *inv,
+                                 int32_t *offsets);
+
+/* The batched rerouting operator on its own (Section 4.3): given the router's top-k ids, write
+ * slot_ids[t,j] = adapter_ids[t] < 0 ? topk_ids[t,j] : Pi[layer][adapter_ids[t]][topk_ids[t,j]] and,
+ * if counts is not null, the number of pairs per slot (counts is overwritten, not accumulated).
+ * All pointers DEVICE: topk_ids, slot_ids [n_tokens,k] int32 (may alias), adapter_ids [n_tokens],
+ * counts [M + N*E_max].  n_tokens is not limited by max_tokens.  Ids outside [0,M) are passed
+ * through unchanged and flagged in the device error word. */
+ew_status_t ew_reroute(ew_pool_t *pool, int32_t layer, const int32_t *topk_ids, const int32_t *adapter_ids,
+                       int32_t n_tokens, int32_t *slot_ids, int32_t *counts, void *cuda_stream);
+
+/* Copy one layer's expert map Pi^(l) [N,M] to HOST memory (the host-side master copy). */
+ew_status_t ew_get_expert_map(ew_pool_t *pool, int32_t layer, int32_t *host_out);
+
+ew_status_t ew_pool_stats(ew_pool_t *pool, ew_stats_t *out);
+
+/* Read and clear the device error word (synchronises with the pool's last forward).  *code receives
+ * an ew_status_t: EW_OK, EW_ERR_BAD_ADAPTER_ID_IN_BATCH, EW_ERR_TIMEOUT or EW_ERR_INVALID_ARG. */
+ew_status_t ew_last_device_error(ew_pool_t *pool, int32_t *code);
+
+/* Device address of slot `slot` of a layer's fused gate|up tensor (which = 0) or down tensor
+ * (which = 1); slots M + N*E_max .. +S-1 are the shared experts.  For tests and tools: reading an
+ * unmapped slot faults, so callers must only touch slots of loaded experts. */
+ew_status_t ew_slot_address(ew_pool_t *pool, int32_t layer, int32_t which, int32_t slot, void **device_ptr);
+
+const char *ew_status_str(ew_status_t s);
+const char *ew_last_error_string(void); /* detail of the last EW_ERR_CUDA on this thread */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EXPERTWEAVE_H_ */

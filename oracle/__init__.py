@@ -93,6 +93,8 @@ class OracleLayer:
             a, p = _u16(arr)
             self._keep.append(a)
             setattr(st, name, p)
+            if name == "router_w":
+                self.router_w = a
         N = cfg.N
         adapters = list(adapters) if adapters is not None else [None] * N
         assert len(adapters) == N

@@ -1,0 +1,225 @@
+"""ctypes binding over libexpertweave.so: argument marshalling only.
+
+Function names mirror the C ABI (`include/expertweave.h`).  Host weights are numpy uint16 arrays of
+bf16 bit patterns; device operands are torch CUDA tensors, passed by data pointer together with the
+current CUDA stream.  There is no CPU fallback: if the library is missing or a call fails, an
+exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libexpertweave.so")
+
+EW_OK = 0
+STATUS_NAMES = ["EW_OK", "EW_ERR_INVALID_ARG", "EW_ERR_OOM", "EW_ERR_SLOT_IN_USE", "EW_ERR_NOT_LOADED",
+                "EW_ERR_TOO_MANY_EXPERTS", "EW_ERR_CUDA", "EW_ERR_TIMEOUT", "EW_ERR_BAD_ADAPTER_ID_IN_BATCH",
+                "EW_ERR_NO_DEVICE"]
+EXPORTS = ["ew_pool_create", "ew_pool_destroy", "ew_load_base", "ew_load_adapter", "ew_unload_adapter",
+           "ew_pool_trim", "ew_moe_forward", "ew_moe_forward_debug", "ew_reroute", "ew_get_expert_map",
+           "ew_pool_stats", "ew_last_device_error", "ew_slot_address", "ew_status_str", "ew_last_error_string"]
+
+
+class EwConfig(C.Structure):
+    _fields_ = [("device", C.c_int32), ("num_layers", C.c_int32), ("hidden", C.c_int32), ("inter", C.c_int32),
+                ("num_experts", C.c_int32), ("num_shared", C.c_int32), ("top_k", C.c_int32),
+                ("max_adapters", C.c_int32), ("e_max", C.c_int32), ("max_tokens", C.c_int32),
+                ("renormalize", C.c_int32), ("routed_scale", C.c_float), ("pool_mode", C.c_int32),
+                ("reserved0", C.c_int32), ("page_bytes", C.c_uint64), ("prealloc_pages", C.c_uint64),
+                ("max_pages", C.c_uint64)]
+
+
+class EwStats(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in
+                ("page_bytes", "va_reserved_bytes", "pages_mapped", "pages_free", "pages_created_total",
+                 "physical_bytes", "live_expert_bytes", "padding_bytes", "live_experts", "adapters_loaded",
+                 "workspace_bytes")]
+
+    def as_dict(self):
+        return {n: int(getattr(self, n)) for n, _ in self._fields_}
+
+
+class EwError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{where}: {name}" + (f" ({detail})" if detail else ""))
+
+
+_lib = None
+
+
+def lib():
+    """Load the shared library (raises if it has not been built: there is no fallback path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2508_17624_b200.build` "
+                               "(the CUDA extension is required; there is no CPU fallback)")
+        _lib = C.CDLL(LIB_PATH)
+        _lib.ew_status_str.restype = C.c_char_p
+        _lib.ew_last_error_string.restype = C.c_char_p
+        for name in EXPORTS:
+            getattr(_lib, name)
+    return _lib
+
+
+def _check(rc: int, where: str):
+    if rc != EW_OK:
+        detail = lib().ew_last_error_string().decode() if rc == 6 or rc == 2 or rc == 1 else ""
+        raise EwError(rc, where, detail)
+
+
+def _host(a, dtype=np.uint16) -> Optional[np.ndarray]:
+    if a is None:
+        return None
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _hp(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _dp(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class Pool:
+    """Owner of one `ew_pool_t`.  Methods carry the names of the C entry points without the prefix."""
+
+    def __init__(self, *, device: int = 0, num_layers: int = 1, hidden: int, inter: int, num_experts: int,
+                 num_shared: int, top_k: int, max_adapters: int, e_max: int, max_tokens: int,
+                 renormalize: int = 0, routed_scale: float = 1.0, pool_mode: int = 0, page_bytes: int = 0,
+                 prealloc_pages: int = 0, max_pages: int = 0):
+        self.cfg = EwConfig(device, num_layers, hidden, inter, num_experts, num_shared, top_k, max_adapters,
+                            e_max, max_tokens, renormalize, routed_scale, pool_mode, 0, page_bytes,
+                            prealloc_pages, max_pages)
+        self._h = C.c_void_p()
+        _check(lib().ew_pool_create(C.byref(self.cfg), C.byref(self._h)), "ew_pool_create")
+
+    @classmethod
+    def from_config(cls, cfg, *, device: int = 0, max_tokens: Optional[int] = None, **kw) -> "Pool":
+        """`cfg` is a `workloads.MoEConfig`."""
+        return cls(device=device, num_layers=cfg.num_layers, hidden=cfg.hidden, inter=cfg.inter,
+                   num_experts=cfg.num_experts, num_shared=cfg.num_shared, top_k=cfg.top_k,
+                   max_adapters=cfg.max_adapters, e_max=cfg.e_max, max_tokens=max_tokens or cfg.n_tokens, **kw)
+
+    @property
+    def num_slots(self) -> int:
+        return self.cfg.num_experts + self.cfg.max_adapters * self.cfg.e_max
+
+    def destroy(self):
+        if self._h:
+            _check(lib().ew_pool_destroy(self._h), "ew_pool_destroy")
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def load_base(self, layer, router_w, w_gate, w_up, w_down, sh_gate=None, sh_up=None, sh_down=None):
+        arrs = [_host(a) for a in (router_w, w_gate, w_up, w_down, sh_gate, sh_up, sh_down)]
+        _check(lib().ew_load_base(self._h, layer, *[_hp(a) for a in arrs]), "ew_load_base")
+
+    def load_adapter(self, adapter_id, counts, expert_ids, w_gate, w_up, w_down):
+        counts = _host(counts, np.int32)
+        expert_ids = _host(expert_ids, np.int32)
+        g, u, d = _host(w_gate), _host(w_up), _host(w_down)
+        _check(lib().ew_load_adapter(self._h, adapter_id, _hp(counts), _hp(expert_ids), _hp(g), _hp(u), _hp(d)),
+               "ew_load_adapter")
+
+    def unload_adapter(self, adapter_id):
+        _check(lib().ew_unload_adapter(self._h, adapter_id), "ew_unload_adapter")
+
+    def trim(self):
+        _check(lib().ew_pool_trim(self._h), "ew_pool_trim")
+
+    def moe_forward(self, layer, x, adapter_ids, out=None):
+        import torch
+        if out is None:
+            out = torch.empty_like(x)
+        _check(lib().ew_moe_forward(self._h, layer, _dp(x), _dp(adapter_ids), x.shape[0], _dp(out), _stream()),
+               "ew_moe_forward")
+        return out
+
+    def moe_forward_debug(self, layer, x, adapter_ids):
+        import torch
+        B, k, P = x.shape[0], self.cfg.top_k, self.num_slots
+        dev = x.device
+        out = torch.empty_like(x)
+        r = dict(topk_ids=torch.empty((B, k), dtype=torch.int32, device=dev),
+                 topk_w=torch.empty((B, k), dtype=torch.float32, device=dev),
+                 slot_ids=torch.empty((B, k), dtype=torch.int32, device=dev),
+                 counts=torch.empty((P,), dtype=torch.int32, device=dev),
+                 inv=torch.empty((B, k), dtype=torch.int32, device=dev),
+                 offsets=torch.empty((P + 1,), dtype=torch.int32, device=dev))
+        _check(lib().ew_moe_forward_debug(self._h, layer, _dp(x), _dp(adapter_ids), B, _dp(out), _stream(),
+                                          _dp(r["topk_ids"]), _dp(r["topk_w"]), _dp(r["slot_ids"]), _dp(r["counts"]),
+                                          _dp(r["inv"]), _dp(r["offsets"])), "ew_moe_forward_debug")
+        r["out"] = out
+        return r
+
+    def reroute(self, layer, topk_ids, adapter_ids, slot_ids=None, counts=None, want_counts=True):
+        import torch
+        if slot_ids is None:
+            slot_ids = torch.empty_like(topk_ids)
+        if counts is None and want_counts:
+            counts = torch.empty((self.num_slots,), dtype=torch.int32, device=topk_ids.device)
+        _check(lib().ew_reroute(self._h, layer, _dp(topk_ids), _dp(adapter_ids), topk_ids.shape[0], _dp(slot_ids),
+                                _dp(counts), _stream()), "ew_reroute")
+        return slot_ids, counts
+
+    def get_expert_map(self, layer) -> np.ndarray:
+        out = np.empty((self.cfg.max_adapters, self.cfg.num_experts), np.int32)
+        _check(lib().ew_get_expert_map(self._h, layer, _hp(out)), "ew_get_expert_map")
+        return out
+
+    def stats(self) -> dict:
+        s = EwStats()
+        _check(lib().ew_pool_stats(self._h, C.byref(s)), "ew_pool_stats")
+        return s.as_dict()
+
+    def last_device_error(self) -> int:
+        code = C.c_int32(0)
+        _check(lib().ew_last_device_error(self._h, C.byref(code)), "ew_last_device_error")
+        return code.value
+
+    def slot_address(self, layer, which, slot) -> int:
+        p = C.c_void_p()
+        _check(lib().ew_slot_address(self._h, layer, which, slot, C.byref(p)), "ew_slot_address")
+        return p.value or 0
+
+
+def load_model(pool: Pool, cfg, bank=None, layers=None, adapters=None, tuned=None):
+    """Fill a pool with the seeded synthetic model of `cfg` (a workloads.MoEConfig): base weights of the
+    given layers, then the given adapters.  Returns (tuned sets, dict layer -> BaseLayer) for the tests."""
+    from . import workloads as wl
+    bank = bank or wl.NoiseBank(cfg.seed)
+    layers = list(range(cfg.num_layers)) if layers is None else layers
+    tuned = wl.tuned_sets(cfg) if tuned is None else tuned
+    bases = {}
+    for l in layers:
+        b = wl.gen_base_layer(cfg, l, bank)
+        pool.load_base(l, b.router_w, b.routed.w_gate, b.routed.w_up, b.routed.w_down,
+                       b.shared.w_gate, b.shared.w_up, b.shared.w_down)
+        bases[l] = b
+    adapters = list(range(cfg.max_adapters)) if adapters is None else adapters
+    for i in adapters:
+        per_layer = [wl.gen_adapter_layer(cfg, i, l, tuned[i][l], bank) for l in range(cfg.num_layers)]
+        counts = np.array([len(tuned[i][l]) for l in range(cfg.num_layers)], np.int32)
+        ids = np.concatenate([tuned[i][l] for l in range(cfg.num_layers)]).astype(np.int32)
+        pool.load_adapter(i, counts, ids, np.concatenate([e.w_gate for e in per_layer]),
+                          np.concatenate([e.w_up for e in per_layer]), np.concatenate([e.w_down for e in per_layer]))
+    return tuned, bases

@@ -1,0 +1,375 @@
+// Grouped expert GEMMs on the 5th-generation tensor cores (tcgen05 + TMEM, operands by TMA).
+//
+// The grouped matrix multiplication of Section 2.1 ("GMM on the permuted tokens and the stacked
+// expert weight tensor"), run unmodified over the virtual weight tensor of Section 4.1: the kernel
+// only ever sees a slot index.  Empty slots produce no work item, so unmapped (padding) slots of the
+// tensor are never touched.
+//
+// Orientation ("swap-AB"): the 128-row MMA dimension is a tile of the WEIGHT matrix, the MMA N
+// dimension (16..256) is the token rows of one slot.  At decode a slot has a handful of rows, so the
+// tensor-core tile is filled by weight rows and the kernel is a pure weight stream; at prefill N
+// grows to 256 and the same instruction shape runs at full rate.
+//
+//   GEMM-1 (GLU = true):  act[row, i] = silu(Wgate[slot][i,:] . x_row) * (Wup[slot][i,:] . x_row)   -> bf16
+//                         two accumulators (gate, up) share the token operand; SwiGLU in the epilogue
+//   GEMM-2 (GLU = false): y[row, o]   = Wdown[slot][o,:] . act_row                                  -> fp32
+//
+// One persistent CTA per SM walks the device-built item list.  Warp 0 lane 0 issues TMA loads into a
+// ring of shared-memory stages, warp 1 lane 0 issues tcgen05.mma, warps 2..5 drain TMEM.  Every
+// barrier wait is bounded in time: on expiry the CTA raises bit 1 of the device error word, stops
+// issuing work, lets its copies in flight land, frees its TMEM and returns.
+#include <cuda_bf16.h>
+
+#include "ew_internal.h"
+
+namespace ew {
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kTileRows = 128;      // weight rows per tile = MMA M
+constexpr int kBlockK = 64;         // bf16 elements per stage along K = one 128-byte swizzle row
+constexpr int kATileBytes = kTileRows * kBlockK * 2;   // 16 KiB
+constexpr int kChunkRows = 32;      // token rows per TMA box
+constexpr int kChunkBytes = kChunkRows * kBlockK * 2;  // 4 KiB
+constexpr int kSmemBudget = 227 * 1024 - 2048;
+constexpr long long kWaitLimitCycles = 2000000000ll;   // about one second
+
+template <int NT, bool GLU>
+struct Cfg {
+    static constexpr int kStageBytes = (GLU ? 2 : 1) * kATileBytes + NT * kBlockK * 2;
+    static constexpr int kStagesRaw = kSmemBudget / kStageBytes;
+    static constexpr int kStages = kStagesRaw > 8 ? 8 : kStagesRaw;
+    static constexpr int kAccCols = (GLU ? 2 : 1) * NT;                  // TMEM columns per accumulator set
+    static constexpr int kAccStages = (2 * kAccCols <= 512) ? 2 : 1;
+    static constexpr int kTmemColsRaw = kAccCols * kAccStages;
+    static constexpr int kTmemCols = kTmemColsRaw <= 32 ? 32 : kTmemColsRaw <= 64 ? 64 : kTmemColsRaw <= 128 ? 128
+                                     : kTmemColsRaw <= 256 ? 256 : 512;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+// ---------------------------------------------------------------------------------------------- PTX
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out of time).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err) {
+    if (mbar_try(bar, parity)) return true;
+    long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try(bar, parity)) return true;
+        if ((it & 63u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitLimitCycles) {
+                *abort_flag = 1;
+                atomicOr(err, 2);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+__device__ __forceinline__ void prefetch_map(const CUtensorMap *map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]^T, bf16 x bf16 -> fp32, M = 128, N from the descriptor
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread i gets lane (base + i)
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major operand tile in shared memory, 128-byte swizzle (what TMA wrote): rows of 128 bytes,
+// groups of 8 rows every 1024 bytes.  Start address and offsets are encoded in 16-byte units.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFF) >> 4);          // start address
+    d |= (uint64_t)1 << 16;                          // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset: next 8-row group
+    d |= (uint64_t)1 << 46;                          // descriptor version for sm_100
+    d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
+    return d;
+}
+// bf16 x bf16 -> fp32, A and B K-major, M = 128, N = n
+__device__ __forceinline__ uint32_t instr_desc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------------- kernel
+template <int NT, bool GLU>
+__global__ void __launch_bounds__(kThreads, 1)
+grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
+                    const __grid_constant__ CUtensorMap map_x, const GemmItem *__restrict__ items,
+                    const int32_t *__restrict__ n_items_ptr, int K, int out_rows_per_slot, void *__restrict__ out,
+                    int *err) {
+    using C = Cfg<NT, GLU>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_al + C::kStages * C::kStageBytes);
+    // barrier layout: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2], then tmem base and abort flag
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * C::kStages;
+    const uint32_t bar_tfull = bar_empty + 8 * C::kStages, bar_tempty = bar_tfull + 16;
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(bars + 2 * C::kStages + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_items = *n_items_ptr;
+    const int num_kb = (K + kBlockK - 1) / kBlockK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::kStages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_tfull + 8 * a, 1);
+            mbar_init(bar_tempty + 8 * a, 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_map(&map_w);
+        prefetch_map(&map_a);
+        if (GLU) prefetch_map(&map_x);
+    }
+    if (warp == 1) {   // TMEM allocation is a whole-warp operation
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)),
+                     "r"((uint32_t)C::kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
+                const GemmItem it = items[w];
+                const int nchunk = (it.rows + kChunkRows - 1) / kChunkRows;
+                const CUtensorMap *amap = (GLU && it.from_x) ? &map_x : &map_a;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1, abort_flag, err))) break;
+                    const uint32_t sa = smem_base + stage * C::kStageBytes;
+                    const uint32_t full = bar_full + 8 * stage;
+                    mbar_expect_tx(full, (GLU ? 2 : 1) * kATileBytes + nchunk * kChunkBytes);
+                    if (GLU) {
+                        tma_load_3d(sa, &map_w, kb * kBlockK, it.tile * kTileRows, it.slot * 2, full);
+                        tma_load_3d(sa + kATileBytes, &map_w, kb * kBlockK, it.tile * kTileRows, it.slot * 2 + 1, full);
+                    } else {
+                        tma_load_3d(sa, &map_w, kb * kBlockK, it.tile * kTileRows, it.slot, full);
+                    }
+                    const uint32_t sb = sa + (GLU ? 2 : 1) * kATileBytes;
+                    for (int c = 0; c < nchunk; ++c)
+                        tma_load_2d(sb + c * kChunkBytes, amap, kb * kBlockK, it.in_row + c * kChunkRows, full);
+                    if (++stage == C::kStages) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            bool ok = true;
+            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
+                const GemmItem it = items[w];
+                const int n = ((it.rows + 15) >> 4) << 4;
+                const uint32_t idesc = instr_desc(n);
+                if (!(ok = mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, abort_flag, err))) break;
+                tc_fence_after();
+                const uint32_t d0 = tmem_base + acc * C::kAccCols;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!(ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, err))) break;
+                    tc_fence_after();
+                    const uint32_t sa = smem_base + stage * C::kStageBytes;
+                    const uint64_t a0 = smem_desc_sw128(sa);
+                    const uint64_t a1 = smem_desc_sw128(sa + kATileBytes);
+                    const uint64_t b = smem_desc_sw128(sa + (GLU ? 2 : 1) * kATileBytes);
+#pragma unroll
+                    for (int ki = 0; ki < kBlockK / 16; ++ki) {     // 16 bf16 = 32 bytes = 2 descriptor units per step
+                        const uint32_t accum = (kb | ki) ? 1u : 0u;
+                        tc_mma(d0, a0 + 2 * ki, b + 2 * ki, idesc, accum);
+                        if (GLU) tc_mma(d0 + NT, a1 + 2 * ki, b + 2 * ki, idesc, accum);
+                    }
+                    tc_commit(bar_empty + 8 * stage);   // frees the stage once these MMAs have read it
+                    if (++stage == C::kStages) { stage = 0; phase ^= 1; }
+                }
+                if (!ok) break;
+                tc_commit(bar_tfull + 8 * acc);         // accumulator complete
+                if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int lg = warp & 3;                        // TMEM lane group this warp may read
+        const int row = lg * 32 + lane;                 // row inside the 128-row weight tile
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
+            const GemmItem it = items[w];
+            if (!(ok = mbar_wait(bar_tfull + 8 * acc, acc_phase, abort_flag, err))) break;
+            tc_fence_after();
+            const uint32_t t0 = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * C::kAccCols;
+            const int orow = it.tile * kTileRows + row;            // output feature index
+            const bool row_ok = orow < out_rows_per_slot;
+            const int n = ((it.rows + 15) >> 4) << 4;
+            for (int c0 = 0; c0 < n; c0 += 32) {
+                uint32_t g[32], u[32];
+                if (n - c0 >= 32) {
+                    tc_ld32(t0 + c0, g);
+                    if (GLU) tc_ld32(t0 + NT + c0, u);
+                } else {
+                    tc_ld16(t0 + c0, g);
+                    if (GLU) tc_ld16(t0 + NT + c0, u);
+                }
+                tc_wait_ld();
+                const int lim = min(32, it.rows - c0);
+                if (row_ok) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if (j < lim) {
+                            const size_t o = (size_t)(it.out_row + c0 + j) * out_rows_per_slot + orow;
+                            if (GLU) {
+                                const float gv = __uint_as_float(g[j]), uv = __uint_as_float(u[j]);
+                                const float a = (gv / (1.f + __expf(-gv))) * uv;
+                                reinterpret_cast<__nv_bfloat16 *>(out)[o] = __float2bfloat16_rn(a);
+                            } else {
+                                reinterpret_cast<float *>(out)[o] = __uint_as_float(g[j]);
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+            if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1; }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    if (*abort_flag) {                                  // let copies in flight land before the CTA's memory is reused
+        long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) {}
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols)
+                     : "memory");
+    }
+}
+
+template <int NT, bool GLU>
+int launch_one(ew_pool *p, const CUtensorMap &mw, const CUtensorMap &ma, const CUtensorMap &mx, const GemmItem *items,
+               const int32_t *n_items, int K, int out_rows, void *out, cudaStream_t st) {
+    using C = Cfg<NT, GLU>;
+    grouped_gemm_kernel<NT, GLU><<<p->sm_count, kThreads, C::kSmemBytes, st>>>(mw, ma, mx, items, n_items, K, out_rows,
+                                                                              out, p->ws.err);
+    return (int)cudaGetLastError();
+}
+
+template <int NT, bool GLU>
+int setup_one() {
+    return (int)cudaFuncSetAttribute(grouped_gemm_kernel<NT, GLU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     Cfg<NT, GLU>::kSmemBytes);
+}
+
+}  // namespace
+
+int gemm_setup(ew_pool *) {
+    int rc = 0;
+    rc |= setup_one<32, true>() | setup_one<64, true>() | setup_one<128, true>() | setup_one<256, true>();
+    rc |= setup_one<32, false>() | setup_one<64, false>() | setup_one<128, false>() | setup_one<256, false>();
+    if (rc) set_last_error("cudaFuncSetAttribute(max dynamic shared memory) failed for a grouped GEMM kernel");
+    return rc;
+}
+
+int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, int, cudaStream_t st) {
+    const LayerState &L = p->layers[layer];
+    const int K = p->cfg.hidden, I = p->cfg.inter;
+    switch (p->token_tile) {
+        case 32: return launch_one<32, true>(p, L.map_w13, p->map_xp, map_x, p->ws.items1, p->ws.n_items, K, I, p->ws.act, st);
+        case 64: return launch_one<64, true>(p, L.map_w13, p->map_xp, map_x, p->ws.items1, p->ws.n_items, K, I, p->ws.act, st);
+        case 128: return launch_one<128, true>(p, L.map_w13, p->map_xp, map_x, p->ws.items1, p->ws.n_items, K, I, p->ws.act, st);
+        default: return launch_one<256, true>(p, L.map_w13, p->map_xp, map_x, p->ws.items1, p->ws.n_items, K, I, p->ws.act, st);
+    }
+}
+
+int launch_gemm2(ew_pool *p, int layer, int, cudaStream_t st) {
+    const LayerState &L = p->layers[layer];
+    const int K = p->cfg.inter, H = p->cfg.hidden;
+    switch (p->token_tile) {
+        case 32: return launch_one<32, false>(p, L.map_w2, p->map_act, p->map_act, p->ws.items2, p->ws.n_items + 1, K, H, p->ws.y, st);
+        case 64: return launch_one<64, false>(p, L.map_w2, p->map_act, p->map_act, p->ws.items2, p->ws.n_items + 1, K, H, p->ws.y, st);
+        case 128: return launch_one<128, false>(p, L.map_w2, p->map_act, p->map_act, p->ws.items2, p->ws.n_items + 1, K, H, p->ws.y, st);
+        default: return launch_one<256, false>(p, L.map_w2, p->map_act, p->map_act, p->ws.items2, p->ws.n_items + 1, K, H, p->ws.y, st);
+    }
+}
+
+}  // namespace ew

@@ -1,0 +1,96 @@
+// Internal state of a pool and the launch interface between the host API and the kernels.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime_api.h>
+
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "../../include/expertweave.h"
+#include "ew_vmm.h"
+
+namespace ew {
+
+// One work item of the grouped GEMMs: a 128-row tile of one slot's weight matrix times up to NT
+// token rows of that slot.  Built on the device from the per-slot counts.
+struct alignas(16) GemmItem {
+    int32_t slot;       // first-dimension index into the virtual weight tensor (>= P: shared expert)
+    int32_t tile;       // 128-row tile of the weight matrix
+    int32_t in_row;     // first activation row (x rows for shared experts, permuted rows otherwise)
+    int32_t out_row;    // first output row
+    int32_t rows;       // token rows in this item (1..NT)
+    int32_t from_x;     // 1: activation rows come straight from the caller's x (shared experts)
+    int32_t pad0, pad1;
+};
+
+struct Workspace {
+    int32_t *topk_ids = nullptr;   // [Bmax, k]
+    float *topk_w = nullptr;       // [Bmax, k]
+    int32_t *slot_ids = nullptr;   // [Bmax, k]
+    int32_t *rank = nullptr;       // [Bmax, k] position of the pair inside its slot's chunk
+    int32_t *inv = nullptr;        // [Bmax, k] row of the pair in slot-contiguous order
+    int32_t *counts = nullptr;     // [P]
+    int32_t *offsets = nullptr;    // [P + 1]
+    int32_t *n_items = nullptr;    // [2]  items of GEMM-1, GEMM-2
+    GemmItem *items1 = nullptr;
+    GemmItem *items2 = nullptr;
+    int32_t max_items1 = 0, max_items2 = 0;
+    void *xp = nullptr;            // [Bmax*k, H] bf16 permuted activations
+    void *act = nullptr;           // [S*Bmax + Bmax*k, I] bf16 SwiGLU output
+    float *y = nullptr;            // [S*Bmax + Bmax*k, H] fp32 expert outputs
+    int32_t *err = nullptr;        // device error word
+    int32_t *loaded = nullptr;     // [N] 1 = adapter loaded
+    size_t bytes = 0;
+};
+
+struct LayerState {
+    VirtualTensor w13;             // [P + S, 2, I, H] bf16: per slot the gate block then the up block
+    VirtualTensor w2;              // [P + S, H, I] bf16
+    void *router_w = nullptr;      // device [M, H] bf16
+    int32_t *pi_dev = nullptr;     // device [N, M]
+    std::vector<int32_t> pi_host;  // master copy
+    bool base_loaded = false;
+    CUtensorMap map_w13, map_w2;   // TMA descriptors over the two virtual tensors
+};
+
+}  // namespace ew
+
+struct ew_pool {
+    ew_config_t cfg;
+    int P = 0;                      // M + N * E_max
+    int token_tile = 32;            // NT: token rows per GEMM work item
+    ew::PageBackend *be = nullptr;
+    ew::PagePool pages;
+    std::vector<ew::LayerState> layers;
+    std::vector<std::vector<int32_t>> adapter_counts;   // [N][L]; empty = not loaded
+    ew::Workspace ws;
+    CUtensorMap map_xp, map_act;   // TMA descriptors over the workspace activations
+    cudaStream_t copy_stream = nullptr;
+    std::vector<std::pair<cudaStream_t, cudaEvent_t>> fwd_events;   // last forward per caller stream
+    int sm_count = 148;
+    uint64_t live_expert_bytes = 0, live_experts = 0;
+    CUresult (*encode_tiled)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                             const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill) = nullptr;
+};
+
+namespace ew {
+
+void set_last_error(const std::string &s);
+
+// bf16 2-D/3-D tiled descriptor with 128-byte swizzle; dims/box innermost first.
+int make_tensor_map(ew_pool *p, CUtensorMap *out, const void *base, int rank, const uint64_t *dims,
+                    const uint32_t *box);
+
+// Kernel launchers (all asynchronous on `st`; return cudaError_t as int).
+int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B, cudaStream_t st);
+int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st);
+int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, int B, cudaStream_t st);
+int launch_gemm2(ew_pool *p, int layer, int B, cudaStream_t st);
+int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st);
+int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid, int B, int32_t *slots,
+                   int32_t *counts, cudaStream_t st);
+int gemm_setup(ew_pool *p);   // once per pool: opt in to the shared memory the GEMM kernels need
+
+}  // namespace ew

@@ -1,0 +1,531 @@
+// Host side of the C ABI: pool creation, base / adapter loading and eviction, the forward call.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "ew_internal.h"
+
+namespace ew {
+static thread_local std::string g_last_error;
+void set_last_error(const std::string &s) { g_last_error = s; }
+}  // namespace ew
+
+using namespace ew;
+
+#define CU_TRY(expr)                                                                         \
+    do {                                                                                     \
+        cudaError_t e__ = (expr);                                                            \
+        if (e__ != cudaSuccess) {                                                            \
+            set_last_error(std::string(#expr) + ": " + cudaGetErrorString(e__));             \
+            return e__ == cudaErrorMemoryAllocation ? EW_ERR_OOM : EW_ERR_CUDA;              \
+        }                                                                                    \
+    } while (0)
+
+static ew_status_t be_status(ew_pool *p, int rc) {
+    if (rc == 0) return EW_OK;
+    set_last_error(p->be->last_error);
+    return rc == 2 ? EW_ERR_OOM : EW_ERR_CUDA;
+}
+
+extern "C" const char *ew_status_str(ew_status_t s) {
+    switch (s) {
+        case EW_OK: return "EW_OK";
+        case EW_ERR_INVALID_ARG: return "EW_ERR_INVALID_ARG";
+        case EW_ERR_OOM: return "EW_ERR_OOM";
+        case EW_ERR_SLOT_IN_USE: return "EW_ERR_SLOT_IN_USE";
+        case EW_ERR_NOT_LOADED: return "EW_ERR_NOT_LOADED";
+        case EW_ERR_TOO_MANY_EXPERTS: return "EW_ERR_TOO_MANY_EXPERTS";
+        case EW_ERR_CUDA: return "EW_ERR_CUDA";
+        case EW_ERR_TIMEOUT: return "EW_ERR_TIMEOUT";
+        case EW_ERR_BAD_ADAPTER_ID_IN_BATCH: return "EW_ERR_BAD_ADAPTER_ID_IN_BATCH";
+        case EW_ERR_NO_DEVICE: return "EW_ERR_NO_DEVICE";
+    }
+    return "EW_ERR_?";
+}
+
+extern "C" const char *ew_last_error_string(void) { return g_last_error.c_str(); }
+
+int ew::make_tensor_map(ew_pool *p, CUtensorMap *out, const void *base, int rank, const uint64_t *dims,
+                        const uint32_t *box) {
+    cuuint64_t gdim[5], gstride[5];
+    cuuint32_t bx[5], estr[5];
+    uint64_t stride = 2;
+    for (int i = 0; i < rank; ++i) {
+        gdim[i] = dims[i];
+        bx[i] = box[i];
+        estr[i] = 1;
+        stride *= dims[i];
+        if (i + 1 < rank) gstride[i] = stride;   // byte stride of dimension i+1
+    }
+    CUresult r = p->encode_tiled(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), gdim,
+                                 gstride, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_last_error("cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
+        return 1;
+    }
+    return 0;
+}
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static ew_status_t alloc_workspace(ew_pool *p) {
+    const ew_config_t &c = p->cfg;
+    size_t Bm = (size_t)c.max_tokens, k = c.top_k, P = p->P, S = c.num_shared, H = c.hidden, I = c.inter;
+    size_t rb = P + S * ((Bm + 31) / 32) + (Bm * k + 31) / 32 + 1;
+    size_t r1 = (I + 127) / 128, r2 = (H + 127) / 128;
+    p->ws.max_items1 = (int32_t)(rb * r1);
+    p->ws.max_items2 = (int32_t)(rb * r2);
+    size_t rows = S * Bm + Bm * k + 32;     // +32: a token tile may start at the last row
+    struct Seg { void **ptr; size_t bytes; };
+    Workspace &w = p->ws;
+    Seg segs[] = {
+        {(void **)&w.topk_ids, Bm * k * 4}, {(void **)&w.topk_w, Bm * k * 4}, {(void **)&w.slot_ids, Bm * k * 4},
+        {(void **)&w.rank, Bm * k * 4}, {(void **)&w.inv, Bm * k * 4}, {(void **)&w.counts, P * 4},
+        {(void **)&w.offsets, (P + 1) * 4}, {(void **)&w.n_items, 16}, {(void **)&w.items1, rb * r1 * sizeof(GemmItem)},
+        {(void **)&w.items2, rb * r2 * sizeof(GemmItem)}, {(void **)&w.xp, (Bm * k + 32) * H * 2},
+        {(void **)&w.act, rows * I * 2}, {(void **)&w.y, rows * H * 4}, {(void **)&w.err, 16},
+        {(void **)&w.loaded, (size_t)c.max_adapters * 4 + 16},
+    };
+    size_t total = 0;
+    for (auto &s : segs) total += align_up(s.bytes, 1024);
+    char *base = nullptr;
+    CU_TRY(cudaMalloc(&base, total));
+    CU_TRY(cudaMemset(base, 0, total));
+    size_t off = 0;
+    for (auto &s : segs) {
+        *s.ptr = base + off;
+        off += align_up(s.bytes, 1024);
+    }
+    w.bytes = total;
+    // TMA descriptors over the permuted activations and the SwiGLU output (box = 64 k-elements x 32 rows)
+    uint64_t d_xp[2] = {H, Bm * k + 32}, d_act[2] = {I, rows};
+    uint32_t box[2] = {64, 32};
+    if (make_tensor_map(p, &p->map_xp, w.xp, 2, d_xp, box) || make_tensor_map(p, &p->map_act, w.act, 2, d_act, box))
+        return EW_ERR_CUDA;
+    return EW_OK;
+}
+
+static void destroy_pool(ew_pool *p) {
+    if (!p) return;
+    bool gpu = p->cfg.device >= 0;
+    if (gpu) {
+        cudaSetDevice(p->cfg.device);
+        cudaDeviceSynchronize();
+    }
+    for (auto &L : p->layers) {
+        L.w13.destroy();
+        L.w2.destroy();
+        if (gpu && L.router_w) cudaFree(L.router_w);
+        if (gpu && L.pi_dev) cudaFree(L.pi_dev);
+    }
+    p->pages.trim();
+    if (gpu) {
+        if (p->ws.topk_ids) cudaFree(p->ws.topk_ids);   // the workspace is one allocation; topk_ids is its base
+        for (auto &e : p->fwd_events) cudaEventDestroy(e.second);
+        if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
+    }
+    delete p->be;
+    delete p;
+}
+
+extern "C" ew_status_t ew_pool_create(const ew_config_t *cfg, ew_pool_t **out) {
+    if (!cfg || !out) return EW_ERR_INVALID_ARG;
+    const ew_config_t &c = *cfg;
+    if (c.num_layers < 1 || c.hidden < 8 || c.inter < 8 || c.hidden % 8 || c.inter % 8 || c.num_experts < 1 ||
+        c.num_experts > 256 || c.num_shared < 0 || c.top_k < 1 || c.top_k > 32 || c.top_k > c.num_experts ||
+        c.max_adapters < 0 || c.e_max < 0 || c.max_tokens < 1 || (c.pool_mode != 0 && c.pool_mode != 1) ||
+        (c.max_adapters > 0 && c.e_max < 1)) {
+        set_last_error("ew_pool_create: configuration out of range");
+        return EW_ERR_INVALID_ARG;
+    }
+    ew_pool *p = new (std::nothrow) ew_pool();
+    if (!p) return EW_ERR_OOM;
+    p->cfg = c;
+    p->P = c.num_experts + c.max_adapters * c.e_max;
+    bool gpu = c.device >= 0;
+    ew_status_t st = EW_OK;
+    std::string err;
+    if (gpu) {
+        cudaError_t e = cudaSetDevice(c.device);
+        if (e != cudaSuccess) {
+            set_last_error(std::string("cudaSetDevice: ") + cudaGetErrorString(e));
+            delete p;
+            return EW_ERR_CUDA;
+        }
+        cudaFree(0);
+        p->be = make_cuda_backend(c.device, &err);
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (p->be && cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess && fn)
+            p->encode_tiled = reinterpret_cast<decltype(p->encode_tiled)>(fn);
+        if (!p->be || !p->encode_tiled) {
+            set_last_error(err.empty() ? "cuTensorMapEncodeTiled not available" : err);
+            delete p->be;
+            delete p;
+            return EW_ERR_CUDA;
+        }
+        cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, c.device);
+    } else {
+        p->be = make_mock_backend();
+    }
+    size_t gran = 0;
+    if ((st = be_status(p, p->be->granularity(&gran))) != EW_OK) { destroy_pool(p); return st; }
+    size_t page = c.page_bytes ? (size_t)c.page_bytes : gran;
+    if (page % gran) {
+        set_last_error("page_bytes must be a multiple of the allocation granularity");
+        destroy_pool(p);
+        return EW_ERR_INVALID_ARG;
+    }
+    p->pages.be = p->be;
+    p->pages.page_bytes = page;
+    p->pages.max_pages = c.max_pages;
+    p->adapter_counts.assign(c.max_adapters, {});
+    size_t H = c.hidden, I = c.inter, slots = (size_t)p->P + c.num_shared;
+    p->layers.resize(c.num_layers);
+    for (auto &L : p->layers) {
+        if ((st = be_status(p, L.w13.init(p->be, &p->pages, 2 * I * H * 2, slots))) != EW_OK) break;
+        if ((st = be_status(p, L.w2.init(p->be, &p->pages, H * I * 2, slots))) != EW_OK) break;
+        L.pi_host.resize((size_t)c.max_adapters * c.num_experts);
+        for (int i = 0; i < c.max_adapters; ++i)
+            for (int j = 0; j < c.num_experts; ++j) L.pi_host[(size_t)i * c.num_experts + j] = j;
+    }
+    if (st == EW_OK) st = be_status(p, p->pages.prealloc(c.prealloc_pages));
+    if (st == EW_OK && c.pool_mode == 1)   // padding baseline: back the whole tensor now
+        for (auto &L : p->layers) {
+            if ((st = be_status(p, L.w13.map_slots(0, slots))) != EW_OK) break;
+            if ((st = be_status(p, L.w2.map_slots(0, slots))) != EW_OK) break;
+        }
+    if (st == EW_OK && gpu) {
+        auto body = [&]() -> ew_status_t {
+            CU_TRY(cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking));
+            for (auto &L : p->layers) {
+                CU_TRY(cudaMalloc(&L.router_w, (size_t)c.num_experts * H * 2));
+                size_t pib = std::max<size_t>(L.pi_host.size() * 4, 16);
+                CU_TRY(cudaMalloc(&L.pi_dev, pib));
+                if (!L.pi_host.empty())
+                    CU_TRY(cudaMemcpy(L.pi_dev, L.pi_host.data(), L.pi_host.size() * 4, cudaMemcpyHostToDevice));
+                // gate|up tensor seen as [2*(P+S), I, H]; down tensor as [P+S, H, I]; box = 64 x 128 x 1
+                uint64_t d13[3] = {H, I, 2 * slots}, d2[3] = {I, H, slots};
+                uint32_t box[3] = {64, 128, 1};
+                if (make_tensor_map(p, &L.map_w13, (void *)L.w13.base, 3, d13, box) ||
+                    make_tensor_map(p, &L.map_w2, (void *)L.w2.base, 3, d2, box))
+                    return EW_ERR_CUDA;
+            }
+            ew_status_t s = alloc_workspace(p);
+            if (s != EW_OK) return s;
+            if (gemm_setup(p)) return EW_ERR_CUDA;
+            return EW_OK;
+        };
+        st = body();
+    }
+    if (st != EW_OK) {
+        std::string keep = g_last_error;
+        destroy_pool(p);
+        set_last_error(keep);
+        return st;
+    }
+    *out = p;
+    return EW_OK;
+}
+
+extern "C" ew_status_t ew_pool_destroy(ew_pool_t *pool) {
+    if (!pool) return EW_ERR_INVALID_ARG;
+    destroy_pool(pool);
+    return EW_OK;
+}
+
+extern "C" ew_status_t ew_pool_trim(ew_pool_t *p) {
+    if (!p) return EW_ERR_INVALID_ARG;
+    return be_status(p, p->pages.trim());
+}
+
+// Copy e experts' gate and up blocks into slots [first, first+e) of the fused tensor, and the down
+// blocks into the down tensor.  Source layout: [e, I, H], [e, I, H], [e, H, I].
+static ew_status_t copy_experts(ew_pool *p, LayerState &L, size_t first, size_t e, const void *g, const void *u,
+                                const void *d) {
+    if (e == 0 || p->cfg.device < 0) return EW_OK;
+    size_t blk = (size_t)p->cfg.inter * p->cfg.hidden * 2;
+    char *dst13 = (char *)L.w13.slot_addr(first);
+    CU_TRY(cudaMemcpy2DAsync(dst13, 2 * blk, g, blk, blk, e, cudaMemcpyHostToDevice, p->copy_stream));
+    CU_TRY(cudaMemcpy2DAsync(dst13 + blk, 2 * blk, u, blk, blk, e, cudaMemcpyHostToDevice, p->copy_stream));
+    CU_TRY(cudaMemcpyAsync((void *)L.w2.slot_addr(first), d, blk * e, cudaMemcpyHostToDevice, p->copy_stream));
+    return EW_OK;
+}
+
+extern "C" ew_status_t ew_load_base(ew_pool_t *p, int32_t layer, const void *router_w, const void *w_gate,
+                                    const void *w_up, const void *w_down, const void *sh_gate, const void *sh_up,
+                                    const void *sh_down) {
+    if (!p || layer < 0 || layer >= p->cfg.num_layers) return EW_ERR_INVALID_ARG;
+    const ew_config_t &c = p->cfg;
+    bool gpu = c.device >= 0;
+    if (gpu && (!router_w || !w_gate || !w_up || !w_down || (c.num_shared > 0 && (!sh_gate || !sh_up || !sh_down))))
+        return EW_ERR_INVALID_ARG;
+    if (gpu) CU_TRY(cudaSetDevice(c.device));
+    LayerState &L = p->layers[layer];
+    size_t M = c.num_experts, S = c.num_shared, P = p->P;
+    if (!L.base_loaded && c.pool_mode == 0) {
+        ew_status_t st;
+        if ((st = be_status(p, L.w13.map_slots(0, M))) != EW_OK) return st;
+        if ((st = be_status(p, L.w2.map_slots(0, M))) != EW_OK) { L.w13.unmap_slots(0, M); return st; }
+        if ((st = be_status(p, L.w13.map_slots(P, S))) != EW_OK) { L.w13.unmap_slots(0, M); L.w2.unmap_slots(0, M); return st; }
+        if ((st = be_status(p, L.w2.map_slots(P, S))) != EW_OK) {
+            L.w13.unmap_slots(0, M); L.w2.unmap_slots(0, M); L.w13.unmap_slots(P, S);
+            return st;
+        }
+    }
+    if (!L.base_loaded) {
+        p->live_experts += M;
+        p->live_expert_bytes += (M + S) * 3 * (size_t)c.inter * c.hidden * 2;
+    }
+    if (gpu) {
+        // forwards in flight may still read the old weights of this layer
+        for (auto &e : p->fwd_events) CU_TRY(cudaEventSynchronize(e.second));
+        CU_TRY(cudaMemcpyAsync(L.router_w, router_w, M * c.hidden * 2, cudaMemcpyHostToDevice, p->copy_stream));
+        ew_status_t st = copy_experts(p, L, 0, M, w_gate, w_up, w_down);
+        if (st == EW_OK && S) st = copy_experts(p, L, P, S, sh_gate, sh_up, sh_down);
+        if (st != EW_OK) return st;
+        CU_TRY(cudaStreamSynchronize(p->copy_stream));
+    }
+    L.base_loaded = true;
+    return EW_OK;
+}
+
+extern "C" ew_status_t ew_load_adapter(ew_pool_t *p, int32_t a, const int32_t *counts, const int32_t *expert_ids,
+                                       const void *w_gate, const void *w_up, const void *w_down) {
+    if (!p || !counts || a < 0 || a >= p->cfg.max_adapters) return EW_ERR_INVALID_ARG;
+    const ew_config_t &c = p->cfg;
+    bool gpu = c.device >= 0;
+    int L = c.num_layers, M = c.num_experts;
+    if (!p->adapter_counts[a].empty()) return EW_ERR_SLOT_IN_USE;
+    size_t total = 0;
+    for (int l = 0; l < L; ++l) {
+        if (counts[l] < 0) return EW_ERR_INVALID_ARG;
+        if (counts[l] > c.e_max) return EW_ERR_TOO_MANY_EXPERTS;
+        total += counts[l];
+    }
+    if (total && (!expert_ids || (gpu && (!w_gate || !w_up || !w_down)))) return EW_ERR_INVALID_ARG;
+    for (size_t l = 0, q = 0; l < (size_t)L; ++l)
+        for (int r = 0; r < counts[l]; ++r, ++q) {
+            int j = expert_ids[q];
+            if (j < 0 || j >= M || (r > 0 && expert_ids[q - 1] >= j)) {
+                set_last_error("ew_load_adapter: expert ids must be strictly ascending in [0,M) per layer");
+                return EW_ERR_INVALID_ARG;
+            }
+        }
+    if (gpu) CU_TRY(cudaSetDevice(c.device));
+    size_t delta = (size_t)M + (size_t)a * c.e_max;     // Delta_i = M + i * E_max
+    ew_status_t st = EW_OK;
+    int done = 0;                                       // layers fully mapped so far (for rollback)
+    if (c.pool_mode == 0)
+        for (; done < L; ++done) {
+            LayerState &Ls = p->layers[done];
+            if ((st = be_status(p, Ls.w13.map_slots(delta, counts[done]))) != EW_OK) break;
+            if ((st = be_status(p, Ls.w2.map_slots(delta, counts[done]))) != EW_OK) {
+                Ls.w13.unmap_slots(delta, counts[done]);
+                break;
+            }
+        }
+    size_t blk = (size_t)c.inter * c.hidden * 2;
+    if (st == EW_OK && gpu) {
+        size_t q = 0;
+        for (int l = 0; l < L && st == EW_OK; ++l) {
+            st = copy_experts(p, p->layers[l], delta, counts[l], (const char *)w_gate + q * blk,
+                              (const char *)w_up + q * blk, (const char *)w_down + q * blk);
+            q += counts[l];
+        }
+        if (st == EW_OK && cudaStreamSynchronize(p->copy_stream) != cudaSuccess) {
+            set_last_error("ew_load_adapter: weight copy failed");
+            st = EW_ERR_CUDA;
+        }
+    }
+    if (st != EW_OK) {
+        if (c.pool_mode == 0)
+            for (int l = 0; l < done; ++l) {
+                p->layers[l].w13.unmap_slots(delta, counts[l]);
+                p->layers[l].w2.unmap_slots(delta, counts[l]);
+            }
+        return st;
+    }
+    // publish: Pi[l][a][j] = Delta + rank of j, only after the weights are in place
+    for (size_t l = 0, q = 0; l < (size_t)L; ++l) {
+        LayerState &Ls = p->layers[l];
+        int32_t *row = Ls.pi_host.data() + (size_t)a * M;
+        for (int r = 0; r < counts[l]; ++r, ++q) row[expert_ids[q]] = (int32_t)(delta + r);
+        if (gpu) CU_TRY(cudaMemcpyAsync(Ls.pi_dev + (size_t)a * M, row, (size_t)M * 4, cudaMemcpyHostToDevice, p->copy_stream));
+    }
+    if (gpu) {
+        int32_t one = 1;
+        CU_TRY(cudaMemcpyAsync(p->ws.loaded + a, &one, 4, cudaMemcpyHostToDevice, p->copy_stream));
+        CU_TRY(cudaStreamSynchronize(p->copy_stream));
+    }
+    p->adapter_counts[a].assign(counts, counts + L);
+    p->live_experts += total;
+    p->live_expert_bytes += total * 3 * blk;
+    return EW_OK;
+}
+
+extern "C" ew_status_t ew_unload_adapter(ew_pool_t *p, int32_t a) {
+    if (!p || a < 0 || a >= p->cfg.max_adapters) return EW_ERR_INVALID_ARG;
+    if (p->adapter_counts[a].empty()) return EW_ERR_NOT_LOADED;
+    const ew_config_t &c = p->cfg;
+    bool gpu = c.device >= 0;
+    int L = c.num_layers, M = c.num_experts;
+    if (gpu) CU_TRY(cudaSetDevice(c.device));
+    // 1. rows back to identity, so that later forwards no longer reach the adapter's slots
+    for (int l = 0; l < L; ++l) {
+        LayerState &Ls = p->layers[l];
+        int32_t *row = Ls.pi_host.data() + (size_t)a * M;
+        for (int j = 0; j < M; ++j) row[j] = j;
+        if (gpu) CU_TRY(cudaMemcpyAsync(Ls.pi_dev + (size_t)a * M, row, (size_t)M * 4, cudaMemcpyHostToDevice, p->copy_stream));
+    }
+    if (gpu) {
+        int32_t zero = 0;
+        CU_TRY(cudaMemcpyAsync(p->ws.loaded + a, &zero, 4, cudaMemcpyHostToDevice, p->copy_stream));
+        CU_TRY(cudaStreamSynchronize(p->copy_stream));
+        // 2. forwards issued earlier may still read those slots: wait for them
+        for (auto &e : p->fwd_events) CU_TRY(cudaEventSynchronize(e.second));
+    }
+    // 3. drop the reference counts; pages reaching zero go back to the pool
+    size_t delta = (size_t)M + (size_t)a * c.e_max, total = 0;
+    for (int l = 0; l < L; ++l) {
+        int e = p->adapter_counts[a][l];
+        total += e;
+        if (c.pool_mode == 0) {
+            p->layers[l].w13.unmap_slots(delta, e);
+            p->layers[l].w2.unmap_slots(delta, e);
+        }
+    }
+    p->adapter_counts[a].clear();
+    p->live_experts -= total;
+    p->live_expert_bytes -= total * 3 * (size_t)c.inter * c.hidden * 2;
+    return EW_OK;
+}
+
+extern "C" ew_status_t ew_get_expert_map(ew_pool_t *p, int32_t layer, int32_t *host_out) {
+    if (!p || !host_out || layer < 0 || layer >= p->cfg.num_layers) return EW_ERR_INVALID_ARG;
+    const auto &pi = p->layers[layer].pi_host;
+    if (!pi.empty()) memcpy(host_out, pi.data(), pi.size() * 4);
+    return EW_OK;
+}
+
+extern "C" ew_status_t ew_pool_stats(ew_pool_t *p, ew_stats_t *out) {
+    if (!p || !out) return EW_ERR_INVALID_ARG;
+    memset(out, 0, sizeof(*out));
+    const ew_config_t &c = p->cfg;
+    out->page_bytes = p->pages.page_bytes;
+    for (auto &L : p->layers) {
+        out->va_reserved_bytes += L.w13.va_bytes + L.w2.va_bytes;
+        out->pages_mapped += L.w13.pages_mapped + L.w2.pages_mapped;
+    }
+    out->pages_free = p->pages.free_list.size();
+    out->pages_created_total = p->pages.created_total;
+    out->physical_bytes = (out->pages_mapped + out->pages_free) * out->page_bytes;
+    out->live_expert_bytes = p->live_expert_bytes;
+    out->padding_bytes = (uint64_t)c.num_layers * ((uint64_t)p->P + c.num_shared) * 3 * c.inter * c.hidden * 2;
+    out->live_experts = p->live_experts;
+    for (auto &a : p->adapter_counts) out->adapters_loaded += !a.empty();
+    out->workspace_bytes = p->ws.bytes;
+    return EW_OK;
+}
+
+extern "C" ew_status_t ew_slot_address(ew_pool_t *p, int32_t layer, int32_t which, int32_t slot, void **ptr) {
+    if (!p || !ptr || layer < 0 || layer >= p->cfg.num_layers || slot < 0 || slot >= p->P + p->cfg.num_shared ||
+        (which != 0 && which != 1))
+        return EW_ERR_INVALID_ARG;
+    LayerState &L = p->layers[layer];
+    *ptr = (void *)(which == 0 ? L.w13.slot_addr(slot) : L.w2.slot_addr(slot));
+    return EW_OK;
+}
+
+extern "C" ew_status_t ew_last_device_error(ew_pool_t *p, int32_t *code) {
+    if (!p || !code) return EW_ERR_INVALID_ARG;
+    if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
+    CU_TRY(cudaSetDevice(p->cfg.device));
+    for (auto &e : p->fwd_events) CU_TRY(cudaEventSynchronize(e.second));
+    int32_t v = 0;
+    CU_TRY(cudaMemcpy(&v, p->ws.err, 4, cudaMemcpyDeviceToHost));
+    CU_TRY(cudaMemset(p->ws.err, 0, 4));
+    // the word is a bit set: 1 = bad adapter id, 2 = a bounded wait expired, 4 = expert id out of range
+    *code = (v & 2) ? EW_ERR_TIMEOUT : (v & 1) ? EW_ERR_BAD_ADAPTER_ID_IN_BATCH : (v & 4) ? EW_ERR_INVALID_ARG : EW_OK;
+    return EW_OK;
+}
+
+static ew_status_t note_forward(ew_pool *p, cudaStream_t st) {
+    for (auto &e : p->fwd_events)
+        if (e.first == st) {
+            CU_TRY(cudaEventRecord(e.second, st));
+            return EW_OK;
+        }
+    cudaEvent_t ev;
+    CU_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+    CU_TRY(cudaEventRecord(ev, st));
+    p->fwd_events.push_back({st, ev});
+    return EW_OK;
+}
+
+#define LAUNCH_TRY(call)                                                                       \
+    do {                                                                                       \
+        int e__ = (call);                                                                      \
+        if (e__ != 0) {                                                                        \
+            set_last_error(std::string(#call) + ": " + cudaGetErrorString((cudaError_t)e__));  \
+            return EW_ERR_CUDA;                                                                \
+        }                                                                                      \
+    } while (0)
+
+extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const void *x, const int32_t *aid,
+                                            int32_t B, void *out, void *cuda_stream, int32_t *topk_ids,
+                                            float *topk_w, int32_t *slot_ids, int32_t *counts, int32_t *inv,
+                                            int32_t *offsets) {
+    if (!p || layer < 0 || layer >= p->cfg.num_layers || B < 0 || B > p->cfg.max_tokens) return EW_ERR_INVALID_ARG;
+    if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
+    if (B == 0) return EW_OK;
+    if (!x || !aid || !out || ((uintptr_t)x & 15) || ((uintptr_t)out & 15)) return EW_ERR_INVALID_ARG;
+    if (!p->layers[layer].base_loaded) return EW_ERR_NOT_LOADED;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const ew_config_t &c = p->cfg;
+    int dev = -1;
+    CU_TRY(cudaGetDevice(&dev));
+    if (dev != c.device) CU_TRY(cudaSetDevice(c.device));
+    // the caller's x becomes the activation operand of the shared experts: describe it for TMA
+    CUtensorMap map_x;
+    uint64_t dx[2] = {(uint64_t)c.hidden, (uint64_t)B};
+    uint32_t box[2] = {64, 32};
+    if (make_tensor_map(p, &map_x, x, 2, dx, box)) return EW_ERR_CUDA;
+    size_t nk = (size_t)B * c.top_k;
+    CU_TRY(cudaMemsetAsync(p->ws.counts, 0, (size_t)p->P * 4, st));
+    LAUNCH_TRY(launch_route(p, layer, x, aid, B, st));
+    LAUNCH_TRY(launch_permute(p, x, B, st));
+    if (topk_ids) CU_TRY(cudaMemcpyAsync(topk_ids, p->ws.topk_ids, nk * 4, cudaMemcpyDeviceToDevice, st));
+    if (topk_w) CU_TRY(cudaMemcpyAsync(topk_w, p->ws.topk_w, nk * 4, cudaMemcpyDeviceToDevice, st));
+    if (slot_ids) CU_TRY(cudaMemcpyAsync(slot_ids, p->ws.slot_ids, nk * 4, cudaMemcpyDeviceToDevice, st));
+    if (counts) CU_TRY(cudaMemcpyAsync(counts, p->ws.counts, (size_t)p->P * 4, cudaMemcpyDeviceToDevice, st));
+    if (inv) CU_TRY(cudaMemcpyAsync(inv, p->ws.inv, nk * 4, cudaMemcpyDeviceToDevice, st));
+    if (offsets) CU_TRY(cudaMemcpyAsync(offsets, p->ws.offsets, ((size_t)p->P + 1) * 4, cudaMemcpyDeviceToDevice, st));
+    LAUNCH_TRY(launch_gemm1(p, layer, map_x, B, st));
+    LAUNCH_TRY(launch_gemm2(p, layer, B, st));
+    LAUNCH_TRY(launch_combine(p, B, out, st));
+    return note_forward(p, st);
+}
+
+extern "C" ew_status_t ew_moe_forward(ew_pool_t *p, int32_t layer, const void *x, const int32_t *aid, int32_t B,
+                                      void *out, void *cuda_stream) {
+    return ew_moe_forward_debug(p, layer, x, aid, B, out, cuda_stream, nullptr, nullptr, nullptr, nullptr, nullptr,
+                                nullptr);
+}
+
+extern "C" ew_status_t ew_reroute(ew_pool_t *p, int32_t layer, const int32_t *topk_ids, const int32_t *aid,
+                                  int32_t B, int32_t *slot_ids, int32_t *counts, void *cuda_stream) {
+    if (!p || layer < 0 || layer >= p->cfg.num_layers || B < 0) return EW_ERR_INVALID_ARG;
+    if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int dev = -1;
+    CU_TRY(cudaGetDevice(&dev));
+    if (dev != p->cfg.device) CU_TRY(cudaSetDevice(p->cfg.device));
+    if (counts) CU_TRY(cudaMemsetAsync(counts, 0, (size_t)p->P * 4, st));
+    if (B == 0) return EW_OK;
+    if (!topk_ids || !aid || !slot_ids) return EW_ERR_INVALID_ARG;
+    LAUNCH_TRY(launch_reroute(p, layer, topk_ids, aid, B, slot_ids, counts, st));
+    return note_forward(p, st);
+}

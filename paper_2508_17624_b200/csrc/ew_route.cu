@@ -1,0 +1,367 @@
+// Routing-side kernels of the adapter-aware MoE layer:
+//   route_kernel     router logits + softmax + top-k + batched rerouting + per-slot histogram (fused)
+//   reroute_kernel   the batched rerouting operator alone (Section 4.3) + histogram
+//   permute_kernel   exclusive scan of the counts, scatter of token rows into slot-contiguous order,
+//                    and (one extra CTA) the work-item lists of the grouped GEMMs
+//   combine_kernel   weighted un-permute and sum, one rounding to bf16 (Section 2.1)
+#include <cuda_bf16.h>
+
+#include "ew_internal.h"
+
+namespace ew {
+namespace {
+
+constexpr int kMaxPerLane = 8;   // experts per lane: M <= 256
+
+__device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+
+__device__ __forceinline__ float dot8(const uint4 &a, const uint4 &b, float acc) {
+    acc = fmaf(bf_lo(a.x), bf_lo(b.x), acc); acc = fmaf(bf_hi(a.x), bf_hi(b.x), acc);
+    acc = fmaf(bf_lo(a.y), bf_lo(b.y), acc); acc = fmaf(bf_hi(a.y), bf_hi(b.y), acc);
+    acc = fmaf(bf_lo(a.z), bf_lo(b.z), acc); acc = fmaf(bf_hi(a.z), bf_hi(b.z), acc);
+    acc = fmaf(bf_lo(a.w), bf_lo(b.w), acc); acc = fmaf(bf_hi(a.w), bf_hi(b.w), acc);
+    return acc;
+}
+
+// slot = aid < 0 ? id : Pi[aid][id]; bad adapter ids behave as -1 and raise bit 0 of the error word
+__device__ __forceinline__ int checked_aid(int a, int N, const int32_t *loaded, int *err) {
+    if (a < -1 || a >= N || (a >= 0 && !loaded[a])) {
+        atomicOr(err, 1);
+        return -1;
+    }
+    return a;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Fused router: one warp per token.  The token row sits in shared memory, router rows stream through
+// L1/L2 with 16-byte loads, fp32 accumulation, warp-shuffle reductions for the dot products, the
+// softmax statistics and the k arg-max rounds (value descending, index ascending).  The expert map
+// of the layer is staged in shared memory; the per-slot histogram is built with one atomic per pair,
+// whose return value is the pair's position inside its slot's chunk.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) route_kernel(const uint4 *__restrict__ x, const uint4 *__restrict__ wg,
+                                                    const int32_t *__restrict__ aid, const int32_t *__restrict__ pi,
+                                                    const int32_t *__restrict__ loaded, int B, int H, int M, int k, int N,
+                                                    int renormalize, float scale, int32_t *__restrict__ topk_ids,
+                                                    float *__restrict__ topk_w, int32_t *__restrict__ slot_ids,
+                                                    int32_t *__restrict__ rank, int32_t *__restrict__ counts, int *err) {
+    extern __shared__ uint4 smem4[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int hv = H >> 3;                                   // 16-byte vectors per row
+    uint4 *xs = smem4 + (size_t)warp * hv;                   // this warp's token row
+    int32_t *pi_s = reinterpret_cast<int32_t *>(smem4 + (size_t)8 * hv);
+    for (int i = threadIdx.x; i < N * M; i += blockDim.x) pi_s[i] = pi[i];
+    const int t = blockIdx.x * 8 + warp;
+    if (t < B)
+        for (int v = lane; v < hv; v += 32) xs[v] = x[(size_t)t * hv + v];
+    __syncthreads();
+    if (t >= B) return;
+
+    float z[kMaxPerLane];                                    // lane holds experts j = q*32 + lane
+#pragma unroll
+    for (int q = 0; q < kMaxPerLane; ++q) z[q] = -INFINITY;
+#pragma unroll
+    for (int q = 0; q < kMaxPerLane; ++q) {
+        if (q * 32 < M) {
+            for (int jl = 0; jl < 32 && q * 32 + jl < M; ++jl) {
+                const uint4 *wr = wg + (size_t)(q * 32 + jl) * hv;
+                float acc = 0.f;
+                for (int v = lane; v < hv; v += 32) acc = dot8(xs[v], __ldg(wr + v), acc);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+                if (lane == jl) z[q] = acc;
+            }
+        }
+    }
+    // softmax over the M logits
+    float mx = z[0];
+#pragma unroll
+    for (int q = 1; q < kMaxPerLane; ++q) mx = fmaxf(mx, z[q]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float sum = 0.f;
+#pragma unroll
+    for (int q = 0; q < kMaxPerLane; ++q) {
+        z[q] = (q * 32 + lane < M) ? expf(z[q] - mx) : -1.f;     // -1 marks "no expert here" (probabilities are >= 0)
+        sum += fmaxf(z[q], 0.f);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+#pragma unroll
+    for (int q = 0; q < kMaxPerLane; ++q)
+        if (z[q] >= 0.f) z[q] = z[q] / sum;
+    // k rounds of arg-max; lane r keeps the r-th selection
+    int my_id = 0;
+    float my_w = 0.f, wsum = 0.f;
+    for (int r = 0; r < k; ++r) {
+        float bv = -1.f;
+        int bi = 0x7fffffff;
+#pragma unroll
+        for (int q = 0; q < kMaxPerLane; ++q)
+            if (z[q] > bv) { bv = z[q]; bi = q * 32 + lane; }      // ascending q: the lower index keeps a tie
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        if (lane == r) { my_id = bi; my_w = bv; }
+        wsum += bv;
+        if ((bi & 31) == lane) {
+#pragma unroll
+            for (int q = 0; q < kMaxPerLane; ++q)
+                if (q == (bi >> 5)) z[q] = -1.f;                     // taken
+        }
+    }
+    if (lane < k) {
+        if (renormalize) my_w = my_w / wsum;
+        my_w *= scale;
+        const int a = checked_aid(aid[t], N, loaded, err);
+        const int slot = a < 0 ? my_id : pi_s[a * M + my_id];
+        const size_t o = (size_t)t * k + lane;
+        topk_ids[o] = my_id;
+        topk_w[o] = my_w;
+        slot_ids[o] = slot;
+        rank[o] = atomicAdd(counts + slot, 1);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Batched rerouting alone: four pairs per thread (16-byte loads and stores), expert map in shared
+// memory, per-CTA shared-memory histogram flushed with one atomic per non-empty slot.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) reroute_kernel(const int32_t *__restrict__ ids, const int32_t *__restrict__ aid,
+                                                      const int32_t *__restrict__ pi, const int32_t *__restrict__ loaded,
+                                                      long long n_pairs, int k, int M, int N, int P,
+                                                      int32_t *__restrict__ slots, int32_t *__restrict__ counts, int *err) {
+    extern __shared__ int32_t smem_i[];
+    int32_t *pi_s = smem_i, *hist = smem_i + N * M;
+    for (int i = threadIdx.x; i < N * M; i += blockDim.x) pi_s[i] = pi[i];
+    if (counts)
+        for (int i = threadIdx.x; i < P; i += blockDim.x) hist[i] = 0;
+    __syncthreads();
+    const long long n_vec = (n_pairs + 3) >> 2;
+    for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < n_vec; v += (long long)gridDim.x * blockDim.x) {
+        const long long q0 = v << 2;
+        int id[4];
+        const bool full = q0 + 3 < n_pairs;
+        if (full) {
+            const int4 r = *reinterpret_cast<const int4 *>(ids + q0);
+            id[0] = r.x; id[1] = r.y; id[2] = r.z; id[3] = r.w;
+        } else {
+            for (int j = 0; j < 4; ++j) id[j] = q0 + j < n_pairs ? ids[q0 + j] : 0;
+        }
+        int s[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const long long q = q0 + j;
+            if (q < n_pairs) {
+                const int a = checked_aid(__ldg(aid + q / k), N, loaded, err);
+                int e = id[j];
+                if (e < 0 || e >= M) { atomicOr(err, 4); s[j] = e; }
+                else {
+                    s[j] = a < 0 ? e : pi_s[a * M + e];
+                    if (counts) atomicAdd(hist + s[j], 1);
+                }
+            } else s[j] = 0;
+        }
+        if (full) *reinterpret_cast<int4 *>(slots + q0) = make_int4(s[0], s[1], s[2], s[3]);
+        else
+            for (int j = 0; j < 4; ++j)
+                if (q0 + j < n_pairs) slots[q0 + j] = s[j];
+    }
+    if (counts) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < P; i += blockDim.x)
+            if (hist[i]) atomicAdd(counts + i, hist[i]);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Scan + permute + plan.  Every CTA recomputes the exclusive scan of the (small) count array in
+// shared memory; CTAs 0..n-2 copy one token row per warp to its slot-contiguous position, the last
+// CTA publishes the offsets and writes the GEMM work items:
+//   shared experts first (all B rows each), then every non-empty slot; per group the items are ordered
+//   (weight tile, token block) so that CTAs working at the same time share a weight tile through L2.
+// ------------------------------------------------------------------------------------------------
+__device__ void block_exclusive_scan(const int32_t *__restrict__ in, int32_t *out, int n, int32_t *warp_sums) {
+    // out[0..n] = exclusive scan of in[0..n-1] (out[n] = total); blockDim.x = 256
+    const int per = (n + 255) / 256;
+    const int lo = min(threadIdx.x * per, n), hi = min(lo + per, n);
+    int32_t s = 0;
+    for (int i = lo; i < hi; ++i) s += in[i];
+    int32_t incl = s;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    int32_t base = 0;
+    for (int w = 0; w < warp; ++w) base += warp_sums[w];
+    int32_t run = base + incl - s;
+    for (int i = lo; i < hi; ++i) { out[i] = run; run += in[i]; }
+    if (threadIdx.x == 255) out[n] = run;     // thread 255's range ends at n
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(256) permute_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ slot_ids,
+                                                      const int32_t *__restrict__ rank, const int32_t *__restrict__ counts,
+                                                      int B, int k, int H, int P, int S, int NT, int R1, int R2,
+                                                      int32_t *__restrict__ offsets, int32_t *__restrict__ inv,
+                                                      uint4 *__restrict__ xp, GemmItem *__restrict__ items1,
+                                                      GemmItem *__restrict__ items2, int32_t *__restrict__ n_items) {
+    extern __shared__ int32_t sm[];
+    int32_t *off = sm;                 // [P + 1]
+    int32_t *blk = sm + P + 1;         // [P + S + 1] token blocks per group, scanned
+    __shared__ int32_t warp_sums[8];
+    block_exclusive_scan(counts, off, P, warp_sums);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (blockIdx.x + 1 < gridDim.x) {
+        const long long q = (long long)blockIdx.x * 8 + warp;
+        if (q < (long long)B * k) {
+            const int dest = off[slot_ids[q]] + rank[q];
+            if (lane == 0) inv[q] = dest;
+            const int hv = H >> 3;
+            const uint4 *src = x + (size_t)(q / k) * hv;
+            uint4 *dst = xp + (size_t)dest * hv;
+            for (int v = lane; v < hv; v += 32) dst[v] = src[v];
+        }
+        return;
+    }
+    // ---- planner CTA
+    for (int i = threadIdx.x; i <= P; i += 256) offsets[i] = off[i];
+    // groups: g < S shared expert g (rows = B); g >= S slot g - S (rows = counts)
+    const int G = P + S;
+    int32_t *nblk = blk + G + 1;       // [G] scratch
+    for (int g = threadIdx.x; g < G; g += 256) {
+        const int rows = g < S ? B : counts[g - S];
+        nblk[g] = (rows + NT - 1) / NT;
+    }
+    __syncthreads();
+    block_exclusive_scan(nblk, blk, G, warp_sums);
+    const int total_blocks = blk[G];
+    if (threadIdx.x == 0) { n_items[0] = total_blocks * R1; n_items[1] = total_blocks * R2; }
+    for (int g = warp; g < G; g += 8) {
+        const int nb = nblk[g];
+        if (nb == 0) continue;
+        const bool shared = g < S;
+        const int rows = shared ? B : counts[g - S];
+        const int slot = shared ? P + g : g - S;
+        const int in0 = shared ? 0 : off[g - S];
+        const int out0 = shared ? g * B : S * B + off[g - S];
+        for (int pass = 0; pass < 2; ++pass) {
+            const int R = pass ? R2 : R1;
+            GemmItem *dst = (pass ? items2 : items1) + (size_t)blk[g] * R;
+            for (int i = lane; i < nb * R; i += 32) {
+                const int tile = i / nb, c = i % nb;
+                GemmItem it;
+                it.slot = slot; it.tile = tile;
+                it.in_row = (pass ? out0 : in0) + c * NT;     // GEMM-2 reads what GEMM-1 wrote
+                it.out_row = out0 + c * NT;
+                it.rows = min(NT, rows - c * NT);
+                it.from_x = (!pass && shared) ? 1 : 0;
+                it.pad0 = it.pad1 = 0;
+                dst[i] = it;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// out[t] = sum_j w[t,j] * Y[S*B + inv[t,j]] + sum_q Y[q*B + t], fp32, j in router order, one rounding
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) combine_kernel(const float4 *__restrict__ y, const int32_t *__restrict__ inv,
+                                                      const float *__restrict__ w, int B, int k, int H, int S,
+                                                      uint2 *__restrict__ out) {
+    __shared__ int32_t rows[32];
+    __shared__ float wts[32];
+    const int t = blockIdx.x;
+    if (threadIdx.x < k) {
+        rows[threadIdx.x] = S * B + inv[(size_t)t * k + threadIdx.x];
+        wts[threadIdx.x] = w[(size_t)t * k + threadIdx.x];
+    }
+    __syncthreads();
+    const int hv = H >> 2;
+    for (int v = threadIdx.x; v < hv; v += blockDim.x) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int j = 0; j < k; ++j) {
+            const float4 a = __ldg(y + (size_t)rows[j] * hv + v);
+            const float wj = wts[j];
+            acc.x = fmaf(wj, a.x, acc.x); acc.y = fmaf(wj, a.y, acc.y);
+            acc.z = fmaf(wj, a.z, acc.z); acc.w = fmaf(wj, a.w, acc.w);
+        }
+        for (int q = 0; q < S; ++q) {
+            const float4 a = __ldg(y + ((size_t)q * B + t) * hv + v);
+            acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
+        }
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+        uint2 o;
+        o.x = *reinterpret_cast<const uint32_t *>(&lo);
+        o.y = *reinterpret_cast<const uint32_t *>(&hi);
+        out[(size_t)t * hv + v] = o;
+    }
+}
+
+}  // namespace
+
+// Token rows per GEMM work item: the smallest tile that holds ~1.5x the mean rows per routed expert.
+static int pick_token_tile(const ew_pool *p, int B) {
+    const double mean = (double)B * p->cfg.top_k / p->cfg.num_experts;
+    const double want = mean * 1.5;
+    return want <= 32 ? 32 : want <= 64 ? 64 : want <= 128 ? 128 : 256;
+}
+
+int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B, cudaStream_t st) {
+    const ew_config_t &c = p->cfg;
+    const LayerState &L = p->layers[layer];
+    const size_t smem = (size_t)8 * c.hidden * 2 + (size_t)c.max_adapters * c.num_experts * 4 + 16;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+    }
+    route_kernel<<<(B + 7) / 8, 256, smem, st>>>((const uint4 *)x, (const uint4 *)L.router_w, aid, L.pi_dev, p->ws.loaded,
+                                                 B, c.hidden, c.num_experts, c.top_k, c.max_adapters, c.renormalize,
+                                                 c.routed_scale, p->ws.topk_ids, p->ws.topk_w, p->ws.slot_ids,
+                                                 p->ws.rank, p->ws.counts, p->ws.err);
+    return (int)cudaGetLastError();
+}
+
+int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st) {
+    const ew_config_t &c = p->cfg;
+    p->token_tile = pick_token_tile(p, B);
+    const int R1 = (c.inter + 127) / 128, R2 = (c.hidden + 127) / 128;
+    const long long pairs = (long long)B * c.top_k;
+    const int grid = (int)((pairs + 7) / 8) + 1;
+    const size_t smem = ((size_t)(p->P + 1) + 2 * (size_t)(p->P + c.num_shared) + 2) * 4;
+    permute_kernel<<<grid, 256, smem, st>>>((const uint4 *)x, p->ws.slot_ids, p->ws.rank, p->ws.counts, B, c.top_k,
+                                            c.hidden, p->P, c.num_shared, p->token_tile, R1, R2, p->ws.offsets,
+                                            p->ws.inv, (uint4 *)p->ws.xp, p->ws.items1, p->ws.items2, p->ws.n_items);
+    return (int)cudaGetLastError();
+}
+
+int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st) {
+    const ew_config_t &c = p->cfg;
+    combine_kernel<<<B, 256, 0, st>>>((const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B, c.top_k, c.hidden,
+                                      c.num_shared, (uint2 *)out);
+    return (int)cudaGetLastError();
+}
+
+int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid, int B, int32_t *slots,
+                   int32_t *counts, cudaStream_t st) {
+    const ew_config_t &c = p->cfg;
+    const long long pairs = (long long)B * c.top_k;
+    const long long vecs = (pairs + 3) / 4;
+    long long blocks = (vecs + 255) / 256;
+    const long long cap = (long long)p->sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    const size_t smem = ((size_t)c.max_adapters * c.num_experts + p->P) * 4 + 16;
+    reroute_kernel<<<(int)blocks, 256, smem, st>>>(ids, aid, p->layers[layer].pi_dev, p->ws.loaded, pairs, c.top_k,
+                                                   c.num_experts, c.max_adapters, p->P, slots, counts, p->ws.err);
+    return (int)cudaGetLastError();
+}
+
+}  // namespace ew

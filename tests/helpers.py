@@ -1,0 +1,99 @@
+"""Shared test plumbing: build the oracle's layer and the GPU pool from the same seeded bits, and the
+staged comparison of a GPU forward against the oracle."""
+from __future__ import annotations
+
+import numpy as np
+
+import oracle
+from paper_2508_17624_b200 import workloads as wl
+
+NEAR_TIE = 1e-5          # a token whose k-th and (k+1)-th probabilities differ by less is a near-tie
+REL_L2_TOL = 1e-2        # bf16 layer output vs the fp32 oracle
+MAX_ABS_TOL = 2e-2
+WEIGHT_TOL = 2e-6        # combine weights (fp32 softmax on both sides, different exp / summation order)
+
+
+def oracle_config(cfg: wl.MoEConfig) -> oracle.OracleConfig:
+    return oracle.OracleConfig(cfg.hidden, cfg.inter, cfg.num_experts, cfg.num_shared, cfg.top_k,
+                               cfg.max_adapters, cfg.e_max)
+
+
+def oracle_layer(cfg, layer, bank, tuned, base=None, adapters=None) -> oracle.OracleLayer:
+    base = base or wl.gen_base_layer(cfg, layer, bank)
+    ads = []
+    for i in range(cfg.max_adapters):
+        if adapters is not None and i not in adapters:
+            ads.append(None)
+            continue
+        ew = wl.gen_adapter_layer(cfg, i, layer, tuned[i][layer], bank)
+        ads.append((tuned[i][layer], ew.w_gate, ew.w_up, ew.w_down))
+    return oracle.OracleLayer(oracle_config(cfg), base.router_w, base.routed.w_gate, base.routed.w_up,
+                              base.routed.w_down, base.shared.w_gate, base.shared.w_up, base.shared.w_down, ads)
+
+
+def to_dev(bits_or_ids, dtype=None):
+    import torch
+    a = np.ascontiguousarray(bits_or_ids)
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    return torch.from_numpy(a).cuda()
+
+
+def bf16_to_f32(t) -> np.ndarray:
+    return t.float().cpu().numpy()
+
+
+def check_routing(cfg, olayer, x_bits, aid, r, Pi=None):
+    """Compare the routing-side results of a debug forward `r` (dict of torch tensors) with the oracle.
+    Returns (ids_gpu, w_for_ffn, slots_gpu, n_near_tie_flips)."""
+    oc = olayer.cfg
+    B, k, P = x_bits.shape[0], oc.k, oc.P
+    ids_g = r["topk_ids"].cpu().numpy()
+    w_g = r["topk_w"].cpu().numpy()
+    slots_g = r["slot_ids"].cpu().numpy()
+    counts_g = r["counts"].cpu().numpy()
+    inv_g = r["inv"].cpu().numpy()
+    off_g = r["offsets"].cpu().numpy()
+    ids_o, w_o, gap, _ = oracle.gate_topk(oc, x_bits, olayer.router_w)
+    # top-k ids: exact as sets, except counted near-ties
+    flips = 0
+    w_ffn = np.empty_like(w_g)
+    for t in range(B):
+        if set(ids_g[t].tolist()) != set(ids_o[t].tolist()):
+            assert gap[t] < NEAR_TIE, f"token {t}: top-k differs with gap {gap[t]}"
+            flips += 1
+            w_ffn[t] = w_g[t]
+            continue
+        lut = {int(j): float(w) for j, w in zip(ids_o[t], w_o[t])}
+        for c in range(k):
+            wo = lut[int(ids_g[t, c])]
+            assert abs(wo - w_g[t, c]) <= WEIGHT_TOL, (t, c, wo, w_g[t, c])
+            w_ffn[t, c] = wo
+        if gap[t] >= NEAR_TIE and np.min(np.abs(np.diff(np.sort(w_o[t])))) >= NEAR_TIE:
+            assert ids_g[t].tolist() == ids_o[t].tolist(), f"token {t}: order differs"
+    assert len(set(map(len, map(set, ids_g.tolist())))) == 1 and len(set(ids_g[0].tolist())) == k
+    # rerouted slots and counts: bit-exact given the same top-k ids
+    Pi = olayer.build_map() if Pi is None else Pi
+    slots_o = oracle.reroute(ids_g, aid, Pi)
+    assert np.array_equal(slots_g, slots_o)
+    counts_o = oracle.counts(slots_g, P)
+    assert np.array_equal(counts_g, counts_o)
+    # offsets: exclusive scan; inv: a bijection onto [0, B*k) that respects the slot chunks
+    assert np.array_equal(off_g, np.concatenate([[0], np.cumsum(counts_o)]).astype(np.int32))
+    flat = inv_g.reshape(-1)
+    assert np.array_equal(np.sort(flat), np.arange(B * k))
+    s = slots_g.reshape(-1)
+    assert np.all(flat >= off_g[s]) and np.all(flat < off_g[s + 1])
+    return ids_g, w_ffn, slots_g, flips
+
+
+def check_output(olayer, x_bits, slots, w, out_gpu_f32, sample=None):
+    """Layer output against the fp32 oracle fed with the given slots/weights (optionally on a sample)."""
+    idx = np.arange(x_bits.shape[0]) if sample is None else np.asarray(sample)
+    ref = oracle.ffn_given_slots(olayer, x_bits[idx], slots[idx], w[idx])
+    got = out_gpu_f32[idx]
+    rel = float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30))
+    mx = float(np.abs(got - ref).max())
+    assert rel <= REL_L2_TOL, f"relative L2 error {rel}"
+    assert mx <= MAX_ABS_TOL, f"max abs error {mx}"
+    return rel, mx

@@ -1,0 +1,151 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2508_17624_b200 import binding, build
+from paper_2508_17624_b200 import workloads as wl
+
+from helpers import bf16_to_f32, check_output, check_routing, oracle_layer, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    import torch
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    build.build()
+    binding.lib()
+
+
+def run_layer(cfg, layer=0, n_tokens=None, aid_mode=None, adapters=None, sample=None, pool=None, bank=None,
+              tuned=None, bases=None):
+    import torch
+    bank = bank or wl.NoiseBank(cfg.seed)
+    own = pool is None
+    if own:
+        pool = binding.Pool.from_config(cfg, max_tokens=n_tokens or cfg.n_tokens)
+        tuned, bases = binding.load_model(pool, cfg, bank, adapters=adapters)
+    olayer = oracle_layer(cfg, layer, bank, tuned, base=bases[layer], adapters=adapters)
+    x = wl.gen_tokens(cfg, layer, n_tokens)
+    aid = wl.gen_adapter_ids(cfg, n_tokens, aid_mode)
+    r = pool.moe_forward_debug(layer, to_dev(x), to_dev(aid))
+    torch.cuda.synchronize()
+    assert pool.last_device_error() == 0
+    ids, w, slots, flips = check_routing(cfg, olayer, x, aid, r)
+    rel, mx = check_output(olayer, x, slots, w, bf16_to_f32(r["out"]), sample)
+    # the plain entry point gives the same bits as the debug one
+    out2 = pool.moe_forward(layer, to_dev(x), to_dev(aid))
+    torch.cuda.synchronize()
+    assert torch.equal(out2, r["out"])
+    if own:
+        pool.destroy()
+    return dict(flips=flips, rel=rel, max_abs=mx, slots=slots, out=r["out"])
+
+
+def test_c0_tiny_layer():
+    res = run_layer(wl.CONFIGS["c0"])
+    assert res["flips"] <= 2
+    assert (res["slots"] >= 16).any()
+
+
+@pytest.mark.parametrize("n_tokens", [1, 7, 33, 64, 100])
+def test_c0_ragged_token_counts(n_tokens):
+    run_layer(wl.CONFIGS["c0"], n_tokens=n_tokens)
+
+
+def test_c1_decode_layer():
+    res = run_layer(wl.CONFIGS["c1"])
+    print("c1", {k: v for k, v in res.items() if k in ("flips", "rel", "max_abs")})
+    assert res["flips"] <= 4
+
+
+def test_c1_base_only_equals_no_adapters():
+    """All tokens base: adapters loaded or not, the output is the base model's."""
+    import torch
+    cfg = wl.CONFIGS["c1"]
+    a = run_layer(cfg, aid_mode="base")
+    b = run_layer(cfg, aid_mode="base", adapters=[])
+    assert torch.equal(a["out"], b["out"])
+    assert (a["slots"] < cfg.num_experts).all()
+
+
+def test_zero_tokens_and_errors():
+    import torch
+    cfg = wl.CONFIGS["c0"]
+    pool = binding.Pool.from_config(cfg)
+    x = torch.zeros((4, cfg.hidden), dtype=torch.bfloat16, device="cuda")
+    aid = torch.zeros(4, dtype=torch.int32, device="cuda")
+    with pytest.raises(binding.EwError) as ei:
+        pool.moe_forward(0, x, aid)                     # base weights not loaded yet
+    assert ei.value.status == 4
+    binding.load_model(pool, cfg, adapters=[0])
+    pool.moe_forward(0, x[:0], aid[:0])                 # n_tokens = 0 is a no-op
+    with pytest.raises(binding.EwError):
+        pool.moe_forward(0, torch.zeros((cfg.n_tokens + 1, cfg.hidden), dtype=torch.bfloat16, device="cuda"),
+                         torch.zeros(cfg.n_tokens + 1, dtype=torch.int32, device="cuda"))
+    # adapter 1 is not loaded and 5 is out of range: both behave as base tokens and raise the device flag
+    xb = to_dev(wl.gen_tokens(cfg, 0, 4))
+    bad = pool.moe_forward(0, xb, torch.tensor([1, 5, -7, -1], dtype=torch.int32, device="cuda"))
+    torch.cuda.synchronize()
+    assert pool.last_device_error() == 8
+    good = pool.moe_forward(0, xb, torch.full((4,), -1, dtype=torch.int32, device="cuda"))
+    torch.cuda.synchronize()
+    assert pool.last_device_error() == 0
+    assert torch.equal(bad, good)
+    pool.destroy()
+
+
+def test_load_unload_on_device():
+    """Evicting an adapter returns its tokens to the base path; reloading restores the adapter path."""
+    import torch
+    cfg = wl.CONFIGS["c0"]
+    bank = wl.NoiseBank(cfg.seed)
+    pool = binding.Pool.from_config(cfg)
+    tuned, bases = binding.load_model(pool, cfg, bank)
+    x, aid = to_dev(wl.gen_tokens(cfg)), to_dev(wl.gen_adapter_ids(cfg))
+    full = pool.moe_forward(0, x, aid).clone()
+    st_full = pool.stats()
+    pool.unload_adapter(1)
+    aid_wo1 = torch.where(aid == 1, torch.full_like(aid, -1), aid)
+    part = pool.moe_forward(0, x, aid_wo1).clone()
+    torch.cuda.synchronize()
+    assert pool.last_device_error() == 0
+    changed = (aid == 1).cpu().numpy()
+    same = torch.equal(part[~torch.from_numpy(changed).cuda()], full[~torch.from_numpy(changed).cuda()])
+    assert same
+    ew = wl.gen_adapter_layer(cfg, 1, 0, tuned[1][0], bank)
+    pool.load_adapter(1, np.array([3], np.int32), tuned[1][0], ew.w_gate, ew.w_up, ew.w_down)
+    again = pool.moe_forward(0, x, aid)
+    torch.cuda.synchronize()
+    assert torch.equal(again, full)
+    assert pool.stats()["pages_mapped"] == st_full["pages_mapped"]
+    pool.destroy()
+
+
+def test_reroute_operator_c4_sample():
+    """The rerouting operator alone: slot ids and per-slot counts are bit-exact."""
+    import torch
+    cfg = wl.with_(wl.CONFIGS["c4"], n_tokens=4099)      # several tiles and a ragged tail
+    oc = oracle.OracleConfig(cfg.hidden, cfg.inter, cfg.num_experts, 0, cfg.top_k, cfg.max_adapters, cfg.e_max)
+    ids, _, _ = oracle.topk_from_logits(oc, wl.gen_logits(cfg))
+    aid = wl.gen_adapter_ids(cfg, mode="uniform")
+    pool = binding.Pool(hidden=64, inter=64, num_experts=cfg.num_experts, num_shared=0, top_k=cfg.top_k,
+                        max_adapters=cfg.max_adapters, e_max=cfg.e_max, max_tokens=8)
+    z = np.zeros((cfg.num_experts, 64, 64), np.uint16)
+    pool.load_base(0, np.zeros((cfg.num_experts, 64), np.uint16), z, z, z)
+    counts = np.array([16], np.int32)
+    tuned = wl.tuned_sets(cfg, np.full((cfg.max_adapters, 1), 16))
+    for i in range(cfg.max_adapters):
+        za = np.zeros((16, 64, 64), np.uint16)
+        pool.load_adapter(i, counts, tuned[i][0], za, za, za)
+    Pi = oracle.build_map(cfg.num_experts, cfg.max_adapters, cfg.e_max, [t[0] for t in tuned])
+    assert np.array_equal(pool.get_expert_map(0), Pi)
+    slots, cnt = pool.reroute(0, to_dev(ids), to_dev(aid))
+    torch.cuda.synchronize()
+    want = oracle.reroute(ids, aid, Pi)
+    assert np.array_equal(slots.cpu().numpy(), want)
+    assert np.array_equal(cnt.cpu().numpy(), oracle.counts(want, cfg.num_slots))
+    assert pool.last_device_error() == 0
+    pool.destroy()

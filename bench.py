@@ -1,0 +1,330 @@
+#!/usr/bin/env python
+"""Benchmark of the adapter-aware MoE layer forward (ExpertWeave hot path) on B200.
+
+A step is one pass of the whole hot path (router + top-k + batched rerouting + histogram, permute,
+grouped SwiGLU GEMM-1, GEMM-2, combine) over one decode batch of the DeepSeek-V2-Lite-shaped layer
+(workload c1: 256 tokens, 64 routed + 2 shared experts, top-6, 4 adapters x 8 re-tuned experts).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W]      the CUDA path (prints one JSON line)
+  python bench.py --impl reference ...                     the CPU oracle as it stands, same metric
+
+With N > 1 (torchrun) every rank runs its own replica of the batch on its own GPU (the path has no
+exchange step), the timed region is bracketed by barriers and the slowest rank's time is used.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "adapter-aware MoE layer tokens/s"
+UNIT = "tokens/s"
+WORKLOAD = "c1: DeepSeek-V2-Lite-shaped MoE layer, decode batch 256, 4 adapters x 8 experts"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.active = False
+        self.err = None
+
+    def run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = int(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
+            names = {
+                getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+                getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+                getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+                getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+                getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake_slowdown",
+            }
+            get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons")
+            while not self._stop_evt.is_set():
+                if self.active:
+                    self.samples.append(int(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
+                    mask = int(get_reasons(h))
+                    for bit, name in names.items():
+                        if mask & bit:
+                            self.reasons.add(name)
+                time.sleep(self.period)
+        except Exception as e:  # clocks are evidence, not part of the computation
+            self.err = repr(e)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+
+    def summary(self):
+        out = {"sm_mhz": float(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
+               "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        if self.err:
+            out["error"] = self.err
+        return out
+
+
+def physical_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except (ValueError, IndexError):
+            pass
+    return local_rank
+
+
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2508_17624_b200 import binding, build, workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    build.build()
+    cfg = wl.CONFIGS["c1"]
+    B, H, k = cfg.n_tokens, cfg.hidden, cfg.top_k
+    pool = binding.Pool.from_config(cfg, device=local)
+    binding.load_model(pool, cfg)
+    x_bits, aid_np = wl.gen_tokens(cfg), wl.gen_adapter_ids(cfg)
+    x = torch.from_numpy(x_bits.view(np.int16)).cuda().view(torch.bfloat16)
+    aid = torch.from_numpy(aid_np).cuda()
+    out = torch.empty_like(x)
+
+    # structure of this batch (for the algorithmic bytes): live slots from one debug forward
+    dbg = pool.moe_forward_debug(0, x, aid)
+    torch.cuda.synchronize()
+    counts = dbg["counts"].cpu().numpy()
+    live = int((counts > 0).sum())
+    groups = live + cfg.num_shared
+    pairs = B * k
+    rows_act = cfg.num_shared * B + pairs
+    blk = cfg.inter * cfg.hidden * 2
+    bytes_gemm1 = groups * 2 * blk + (pairs + B) * H * 2 + rows_act * cfg.inter * 2     # weights + rows in + act out
+    bytes_gemm2 = groups * blk + rows_act * cfg.inter * 2 + rows_act * H * 4
+    bytes_layer = groups * 3 * blk
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        pool.moe_forward(0, x, aid, out)
+    barrier()
+    sampler = ClockSampler(physical_index(local))
+    sampler.start()
+
+    # ---- timed region: K steps, per-kernel events recorded by the library on the same stream
+    pool.profile_enable(True)
+    pool.profile_read()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.active = True
+    e0.record()
+    for _ in range(args.steps):
+        pool.moe_forward(0, x, aid, out)
+    e1.record()
+    barrier()
+    sampler.active = False
+    ms_total = e0.elapsed_time(e1)
+    kern_ms, n_prof = pool.profile_read()
+    pool.profile_enable(False)
+    extended = False
+    if len(sampler.samples) < 3 and not args.minimal:          # short runs: keep the same load going until the sampler has seen it
+        extended = True
+        sampler.active = True
+        t_end = time.time() + 1.5
+        while time.time() < t_end and len(sampler.samples) < 5:
+            for _ in range(50):
+                pool.moe_forward(0, x, aid, out)
+            torch.cuda.synchronize()
+        sampler.active = False
+
+    # ---- same region without the per-kernel events (reported as a cross-check)
+    side_steps = 0 if args.minimal else args.steps
+    barrier()
+    e0.record()
+    for _ in range(side_steps):
+        pool.moe_forward(0, x, aid, out)
+    e1.record()
+    barrier()
+    ms_plain = e0.elapsed_time(e1)
+
+    # ---- end to end through the C ABI with host buffers (pinned): H2D + forward + D2H every step
+    xh = torch.from_numpy(x_bits.view(np.int16).copy()).pin_memory()
+    ah = torch.from_numpy(aid_np.copy()).pin_memory()
+    oh = torch.empty((B, H), dtype=torch.int16).pin_memory()
+    for _ in range(3 if side_steps else 1):
+        pool.moe_forward_host(0, xh, ah, oh)
+    barrier()
+    e0.record()
+    for _ in range(max(side_steps, 1)):
+        pool.moe_forward_host(0, xh, ah, oh)
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    assert torch.equal(oh.cuda().view(torch.bfloat16), out), "host-buffer path disagrees with the device path"
+    sampler.stop()
+    err = pool.last_device_error()
+    assert err == 0, f"device error word {err}"
+
+    times = torch.tensor([ms_total, ms_e2e, ms_plain], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e, ms_plain = (float(v) for v in times.cpu())
+
+    result = None
+    if rank == 0:
+        peak, peak_kind = load_peaks()
+        g1_ms = kern_ms["gemm1"] / max(n_prof, 1)
+        achieved = bytes_gemm1 / (g1_ms * 1e-3) / 1e9
+        result = {
+            "metric": METRIC, "value": world * B * args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "tokens_per_step_per_gpu": B, "hidden": H, "inter": cfg.inter,
+                       "experts": cfg.num_experts, "shared": cfg.num_shared, "top_k": k,
+                       "adapters": cfg.max_adapters, "e_max": cfg.e_max, "live_slots": live,
+                       "token_tile": None, "parallelism": f"replicas x{world}",
+                       "l2": "no flush: each step streams %.2f GB of live expert weights, far above the 126 MB L2"
+                             % (bytes_layer / 1e9)},
+            "e2e": {"value": world * B * max(side_steps, 1) / (ms_e2e * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": B * H * 2 + B * 4, "d2h_bytes_per_step": B * H * 2},
+            "gpu_launches": 5 * args.steps,
+            "clocks": dict(sampler.summary(), extended=extended),
+            "roofline": {"bound": "hbm", "kernel": "grouped_gemm_kernel<GLU> (GEMM-1 + SwiGLU)",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "of": peak_kind, "traffic": None, "algorithmic_bytes": bytes_gemm1,
+                         "avg_launch_ms": g1_ms},
+            "kernels_ms_per_step": {kname: v / max(n_prof, 1) for kname, v in kern_ms.items()},
+            "gemm2": {"achieved": bytes_gemm2 / (kern_ms["gemm2"] / max(n_prof, 1) * 1e-3) / 1e9, "unit": "GB/s",
+                      "algorithmic_bytes": bytes_gemm2},
+            "layer_weight_stream": {"achieved": bytes_layer / (ms_total / args.steps * 1e-3) / 1e9, "unit": "GB/s",
+                                    "frac": bytes_layer / (ms_total / args.steps * 1e-3) / 1e9 / peak},
+            "ms_per_step_without_kernel_events": ms_plain / max(side_steps, 1),
+        }
+        if not args.no_cpu_baseline and not args.minimal and world == 1:
+            result["cpu_baseline"] = cpu_baseline(cfg, budget_s=12.0)
+    pool.destroy()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(result))
+
+
+def build_oracle_layer(cfg):
+    import oracle
+    from paper_2508_17624_b200 import workloads as wl
+    bank = wl.NoiseBank(cfg.seed)
+    base = wl.gen_base_layer(cfg, 0, bank)
+    tuned = wl.tuned_sets(cfg)
+    ads = []
+    for i in range(cfg.max_adapters):
+        ew = wl.gen_adapter_layer(cfg, i, 0, tuned[i][0], bank)
+        ads.append((tuned[i][0], ew.w_gate, ew.w_up, ew.w_down))
+    oc = oracle.OracleConfig(cfg.hidden, cfg.inter, cfg.num_experts, cfg.num_shared, cfg.top_k, cfg.max_adapters,
+                             cfg.e_max)
+    return oracle.OracleLayer(oc, base.router_w, base.routed.w_gate, base.routed.w_up, base.routed.w_down,
+                              base.shared.w_gate, base.shared.w_up, base.shared.w_down, ads)
+
+
+def cpu_baseline(cfg, budget_s: float):
+    """The oracle as it stands, timed on the host cores on a bounded sample of the same batch."""
+    import oracle
+    from paper_2508_17624_b200 import workloads as wl
+    layer = build_oracle_layer(cfg)
+    x, aid = wl.gen_tokens(cfg), wl.gen_adapter_ids(cfg)
+    n = min(32, cfg.n_tokens)
+    t0 = time.time()
+    oracle.layer_forward(layer, x[:n], aid[:n])
+    per_tok = (time.time() - t0) / n
+    n = int(max(1, min(cfg.n_tokens, budget_s / max(per_tok, 1e-9))))
+    t0 = time.time()
+    oracle.layer_forward(layer, x[:n], aid[:n])
+    dt = time.time() - t0
+    return {"value": n / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"first {n} of the {cfg.n_tokens} tokens of the same batch, one pass, {dt:.2f} s"}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, same metric and config; each step a bounded sample of the batch."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2508_17624_b200 import workloads as wl
+    cfg = wl.CONFIGS["c1"]
+    layer = build_oracle_layer(cfg)
+    x, aid = wl.gen_tokens(cfg), wl.gen_adapter_ids(cfg)
+    t0 = time.time()
+    oracle.layer_forward(layer, x[:16], aid[:16])
+    per_tok = (time.time() - t0) / 16
+    total_steps = args.steps + max(args.warmup, 0)
+    n = int(max(1, min(cfg.n_tokens, 150.0 / max(per_tok * total_steps, 1e-9))))
+    for _ in range(max(args.warmup, 0)):
+        oracle.layer_forward(layer, x[:n], aid[:n])
+    t0 = time.time()
+    for _ in range(args.steps):
+        oracle.layer_forward(layer, x[:n], aid[:n])
+    dt = time.time() - t0
+    value = n * args.steps / dt
+    cores = oracle.num_threads()
+    sample = f"each step = the first {n} of the batch's {cfg.n_tokens} tokens"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--minimal", action="store_true",
+                    help="warm-up and timed steps only (for profiler captures): no CPU baseline, no side measurements")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -158,6 +158,23 @@ ew_status_t ew_moe_forward_debug(ew_pool_t *pool, int32_t layer, const void *x, 
                                  float *topk_w, int32_t *slot_ids, int32_t *counts, int32_t *inv,
                                  int32_t *offsets);
 
+/* Same forward with HOST buffers: copies x and adapter_ids to device staging owned by the pool, runs
+ * ew_moe_forward on them and copies the result back, all asynchronous on `cuda_stream` when the host
+ * buffers are page-locked (pageable buffers make the copies synchronous).  The caller synchronises
+ * the stream before reading out_host.  x_host, out_host: host bf16 [n_tokens, H]; adapter_ids_host:
+ * host int32 [n_tokens]. */
+ew_status_t ew_moe_forward_host(ew_pool_t *pool, int32_t layer, const void *x_host,
+                                const int32_t *adapter_ids_host, int32_t n_tokens, void *out_host,
+                                void *cuda_stream);
+
+/* Per-kernel timing.  While enabled, every forward records CUDA events on its stream around its five
+ * kernels (no host synchronisation).  ew_profile_read waits for the recorded forwards, adds up the
+ * elapsed milliseconds per kernel into ms[5] = {route (incl. zeroing the counts), permute+plan,
+ * GEMM-1+SwiGLU, GEMM-2, combine}, writes how many forwards were measured, and clears the record.
+ * At most 4096 forwards are recorded between two reads. */
+ew_status_t ew_profile_enable(ew_pool_t *pool, int32_t on);
+ew_status_t ew_profile_read(ew_pool_t *pool, double *ms, int32_t *n_forwards);
+
 /* The batched rerouting operator on its own (Section 4.3): given the router's top-k ids, write
  * slot_ids[t,j] = adapter_ids[t] < 0 ? topk_ids[t,j] : Pi[layer][adapter_ids[t]][topk_ids[t,j]] and,
  * if counts is not null, the number of pairs per slot (counts is overwritten, not accumulated).

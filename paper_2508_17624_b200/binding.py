@@ -21,7 +21,8 @@ STATUS_NAMES = ["EW_OK", "EW_ERR_INVALID_ARG", "EW_ERR_OOM", "EW_ERR_SLOT_IN_USE
                 "EW_ERR_TOO_MANY_EXPERTS", "EW_ERR_CUDA", "EW_ERR_TIMEOUT", "EW_ERR_BAD_ADAPTER_ID_IN_BATCH",
                 "EW_ERR_NO_DEVICE"]
 EXPORTS = ["ew_pool_create", "ew_pool_destroy", "ew_load_base", "ew_load_adapter", "ew_unload_adapter",
-           "ew_pool_trim", "ew_moe_forward", "ew_moe_forward_debug", "ew_reroute", "ew_get_expert_map",
+           "ew_pool_trim", "ew_moe_forward", "ew_moe_forward_debug", "ew_moe_forward_host", "ew_profile_enable",
+           "ew_profile_read", "ew_reroute", "ew_get_expert_map",
            "ew_pool_stats", "ew_last_device_error", "ew_slot_address", "ew_status_str", "ew_last_error_string"]
 
 
@@ -170,6 +171,26 @@ class Pool:
                                           _dp(r["inv"]), _dp(r["offsets"])), "ew_moe_forward_debug")
         r["out"] = out
         return r
+
+    def moe_forward_host(self, layer, x_host, adapter_ids_host, out_host, n_tokens=None):
+        """x_host / out_host: pinned torch CPU tensors (or numpy arrays); asynchronous on the current stream."""
+        def hp(t):
+            return C.c_void_p(t.data_ptr()) if hasattr(t, "data_ptr") else t.ctypes.data_as(C.c_void_p)
+        n = x_host.shape[0] if n_tokens is None else n_tokens
+        _check(lib().ew_moe_forward_host(self._h, layer, hp(x_host), hp(adapter_ids_host), n, hp(out_host),
+                                         _stream()), "ew_moe_forward_host")
+        return out_host
+
+    def profile_enable(self, on: bool):
+        _check(lib().ew_profile_enable(self._h, int(on)), "ew_profile_enable")
+
+    def profile_read(self):
+        """-> (dict kernel -> total ms, forwards measured)"""
+        ms = (C.c_double * 5)()
+        n = C.c_int32(0)
+        _check(lib().ew_profile_read(self._h, ms, C.byref(n)), "ew_profile_read")
+        names = ("route", "permute", "gemm1", "gemm2", "combine")
+        return {k: float(v) for k, v in zip(names, ms)}, int(n.value)
 
     def reroute(self, layer, topk_ids, adapter_ids, slot_ids=None, counts=None, want_counts=True):
         import torch

@@ -69,6 +69,11 @@ struct ew_pool {
     cudaStream_t copy_stream = nullptr;
     std::vector<std::pair<cudaStream_t, cudaEvent_t>> fwd_events;   // last forward per caller stream
     int sm_count = 148;
+    bool profiling = false;
+    std::vector<cudaEvent_t> prof_events;   // 6 per recorded forward
+    size_t prof_used = 0;                   // events in use
+    void *stage_x = nullptr, *stage_out = nullptr;   // device staging of ew_moe_forward_host
+    int32_t *stage_aid = nullptr;
     uint64_t live_expert_bytes = 0, live_experts = 0;
     CUresult (*encode_tiled)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                              const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,

@@ -87,6 +87,7 @@ static ew_status_t alloc_workspace(ew_pool *p) {
         {(void **)&w.items2, rb * r2 * sizeof(GemmItem)}, {(void **)&w.xp, (Bm * k + 32) * H * 2},
         {(void **)&w.act, rows * I * 2}, {(void **)&w.y, rows * H * 4}, {(void **)&w.err, 16},
         {(void **)&w.loaded, (size_t)c.max_adapters * 4 + 16},
+        {&p->stage_x, Bm * H * 2}, {&p->stage_out, Bm * H * 2}, {(void **)&p->stage_aid, Bm * 4},
     };
     size_t total = 0;
     for (auto &s : segs) total += align_up(s.bytes, 1024);
@@ -124,6 +125,7 @@ static void destroy_pool(ew_pool *p) {
     if (gpu) {
         if (p->ws.topk_ids) cudaFree(p->ws.topk_ids);   // the workspace is one allocation; topk_ids is its base
         for (auto &e : p->fwd_events) cudaEventDestroy(e.second);
+        for (auto &e : p->prof_events) cudaEventDestroy(e);
         if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
     }
     delete p->be;
@@ -494,9 +496,23 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     uint32_t box[2] = {64, 32};
     if (make_tensor_map(p, &map_x, x, 2, dx, box)) return EW_ERR_CUDA;
     size_t nk = (size_t)B * c.top_k;
+    cudaEvent_t *pe = nullptr;
+    if (p->profiling && p->prof_used + 6 <= 6 * 4096) {
+        while (p->prof_events.size() < p->prof_used + 6) {
+            cudaEvent_t ev;
+            CU_TRY(cudaEventCreate(&ev));
+            p->prof_events.push_back(ev);
+        }
+        pe = p->prof_events.data() + p->prof_used;
+        p->prof_used += 6;
+    }
+#define PROF_MARK(i) do { if (pe) CU_TRY(cudaEventRecord(pe[i], st)); } while (0)
+    PROF_MARK(0);
     CU_TRY(cudaMemsetAsync(p->ws.counts, 0, (size_t)p->P * 4, st));
     LAUNCH_TRY(launch_route(p, layer, x, aid, B, st));
+    PROF_MARK(1);
     LAUNCH_TRY(launch_permute(p, x, B, st));
+    PROF_MARK(2);
     if (topk_ids) CU_TRY(cudaMemcpyAsync(topk_ids, p->ws.topk_ids, nk * 4, cudaMemcpyDeviceToDevice, st));
     if (topk_w) CU_TRY(cudaMemcpyAsync(topk_w, p->ws.topk_w, nk * 4, cudaMemcpyDeviceToDevice, st));
     if (slot_ids) CU_TRY(cudaMemcpyAsync(slot_ids, p->ws.slot_ids, nk * 4, cudaMemcpyDeviceToDevice, st));
@@ -504,8 +520,12 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     if (inv) CU_TRY(cudaMemcpyAsync(inv, p->ws.inv, nk * 4, cudaMemcpyDeviceToDevice, st));
     if (offsets) CU_TRY(cudaMemcpyAsync(offsets, p->ws.offsets, ((size_t)p->P + 1) * 4, cudaMemcpyDeviceToDevice, st));
     LAUNCH_TRY(launch_gemm1(p, layer, map_x, B, st));
+    PROF_MARK(3);
     LAUNCH_TRY(launch_gemm2(p, layer, B, st));
+    PROF_MARK(4);
     LAUNCH_TRY(launch_combine(p, B, out, st));
+    PROF_MARK(5);
+#undef PROF_MARK
     return note_forward(p, st);
 }
 
@@ -528,4 +548,49 @@ extern "C" ew_status_t ew_reroute(ew_pool_t *p, int32_t layer, const int32_t *to
     if (!topk_ids || !aid || !slot_ids) return EW_ERR_INVALID_ARG;
     LAUNCH_TRY(launch_reroute(p, layer, topk_ids, aid, B, slot_ids, counts, st));
     return note_forward(p, st);
+}
+
+extern "C" ew_status_t ew_moe_forward_host(ew_pool_t *p, int32_t layer, const void *x_host, const int32_t *aid_host,
+                                           int32_t B, void *out_host, void *cuda_stream) {
+    if (!p || layer < 0 || layer >= p->cfg.num_layers || B < 0 || B > p->cfg.max_tokens) return EW_ERR_INVALID_ARG;
+    if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
+    if (B == 0) return EW_OK;
+    if (!x_host || !aid_host || !out_host) return EW_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int dev = -1;
+    CU_TRY(cudaGetDevice(&dev));
+    if (dev != p->cfg.device) CU_TRY(cudaSetDevice(p->cfg.device));
+    size_t xb = (size_t)B * p->cfg.hidden * 2;
+    CU_TRY(cudaMemcpyAsync(p->stage_x, x_host, xb, cudaMemcpyHostToDevice, st));
+    CU_TRY(cudaMemcpyAsync(p->stage_aid, aid_host, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+    ew_status_t s = ew_moe_forward(p, layer, p->stage_x, p->stage_aid, B, p->stage_out, cuda_stream);
+    if (s != EW_OK) return s;
+    CU_TRY(cudaMemcpyAsync(out_host, p->stage_out, xb, cudaMemcpyDeviceToHost, st));
+    return EW_OK;
+}
+
+extern "C" ew_status_t ew_profile_enable(ew_pool_t *p, int32_t on) {
+    if (!p) return EW_ERR_INVALID_ARG;
+    if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
+    p->profiling = on != 0;
+    return EW_OK;
+}
+
+extern "C" ew_status_t ew_profile_read(ew_pool_t *p, double *ms, int32_t *n_forwards) {
+    if (!p || !ms || !n_forwards) return EW_ERR_INVALID_ARG;
+    if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
+    for (int i = 0; i < 5; ++i) ms[i] = 0.0;
+    size_t n = p->prof_used / 6;
+    for (size_t f = 0; f < n; ++f) {
+        cudaEvent_t *e = p->prof_events.data() + 6 * f;
+        CU_TRY(cudaEventSynchronize(e[5]));
+        for (int i = 0; i < 5; ++i) {
+            float t = 0.f;
+            CU_TRY(cudaEventElapsedTime(&t, e[i], e[i + 1]));
+            ms[i] += t;
+        }
+    }
+    *n_forwards = (int32_t)n;
+    p->prof_used = 0;
+    return EW_OK;
 }

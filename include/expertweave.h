@@ -17,7 +17,7 @@
  *     contiguous.  int32 and float are the C types.
  *   - One pool may be used by one host thread at a time.  Forward calls on one pool share one
  *     workspace: issue them on one stream (or order them yourself).
- *   - H and I must be multiples of 8 (16-byte rows); M <= 256; top_k <= 32 and <= M.
+ *   - H must be a multiple of 64 and I a multiple of 8; M <= 256; top_k <= 32 and <= M.
  */
 #ifndef EXPERTWEAVE_H_
 #define EXPERTWEAVE_H_

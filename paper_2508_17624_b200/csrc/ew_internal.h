@@ -52,6 +52,7 @@ struct LayerState {
     std::vector<int32_t> pi_host;  // master copy
     bool base_loaded = false;
     CUtensorMap map_w13, map_w2;   // TMA descriptors over the two virtual tensors
+    CUtensorMap map_router;        // and over the router rows [M, H]
 };
 
 }  // namespace ew
@@ -87,6 +88,10 @@ void set_last_error(const std::string &s);
 // bf16 2-D/3-D tiled descriptor with 128-byte swizzle; dims/box innermost first.
 int make_tensor_map(ew_pool *p, CUtensorMap *out, const void *base, int rank, const uint64_t *dims,
                     const uint32_t *box);
+
+// bf16 [rows, H] matrix (H a multiple of 64) seen as (64 elements, rows, H/64 K-atoms): one box of
+// 64 x box_rows x atoms lands in shared memory as `atoms` consecutive 128-byte-swizzled tiles.
+int make_atom_map(ew_pool *p, CUtensorMap *out, const void *base, int H, int rows, int box_rows, int atoms);
 
 // Kernel launchers (all asynchronous on `st`; return cudaError_t as int).
 int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B, cudaStream_t st);

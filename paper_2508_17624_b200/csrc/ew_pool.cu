@@ -68,6 +68,20 @@ int ew::make_tensor_map(ew_pool *p, CUtensorMap *out, const void *base, int rank
     return 0;
 }
 
+int ew::make_atom_map(ew_pool *p, CUtensorMap *out, const void *base, int H, int rows, int box_rows, int atoms) {
+    cuuint64_t gdim[3] = {64, (cuuint64_t)rows, (cuuint64_t)(H / 64)};
+    cuuint64_t gstride[2] = {(cuuint64_t)H * 2, 128};
+    cuuint32_t bx[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)atoms}, estr[3] = {1, 1, 1};
+    CUresult r = p->encode_tiled(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), gdim, gstride, bx, estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_last_error("cuTensorMapEncodeTiled (atom map) failed with code " + std::to_string((int)r));
+        return 1;
+    }
+    return 0;
+}
+
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 static ew_status_t alloc_workspace(ew_pool *p) {
@@ -85,7 +99,7 @@ static ew_status_t alloc_workspace(ew_pool *p) {
         {(void **)&w.rank, Bm * k * 4}, {(void **)&w.inv, Bm * k * 4}, {(void **)&w.counts, P * 4},
         {(void **)&w.offsets, (P + 1) * 4}, {(void **)&w.n_items, 16}, {(void **)&w.items1, rb * r1 * sizeof(GemmItem)},
         {(void **)&w.items2, rb * r2 * sizeof(GemmItem)}, {(void **)&w.xp, (Bm * k + 32) * H * 2},
-        {(void **)&w.act, rows * I * 2}, {(void **)&w.y, rows * H * 4}, {(void **)&w.err, 16},
+        {(void **)&w.act, rows * I * 2}, {(void **)&w.y, rows * H * 4}, {(void **)&w.err, 256},
         {(void **)&w.loaded, (size_t)c.max_adapters * 4 + 16},
         {&p->stage_x, Bm * H * 2}, {&p->stage_out, Bm * H * 2}, {(void **)&p->stage_aid, Bm * 4},
     };
@@ -135,7 +149,7 @@ static void destroy_pool(ew_pool *p) {
 extern "C" ew_status_t ew_pool_create(const ew_config_t *cfg, ew_pool_t **out) {
     if (!cfg || !out) return EW_ERR_INVALID_ARG;
     const ew_config_t &c = *cfg;
-    if (c.num_layers < 1 || c.hidden < 8 || c.inter < 8 || c.hidden % 8 || c.inter % 8 || c.num_experts < 1 ||
+    if (c.num_layers < 1 || c.hidden < 64 || c.inter < 8 || c.hidden % 64 || c.inter % 8 || c.num_experts < 1 ||
         c.num_experts > 256 || c.num_shared < 0 || c.top_k < 1 || c.top_k > 32 || c.top_k > c.num_experts ||
         c.max_adapters < 0 || c.e_max < 0 || c.max_tokens < 1 || (c.pool_mode != 0 && c.pool_mode != 1) ||
         (c.max_adapters > 0 && c.e_max < 1)) {
@@ -212,7 +226,8 @@ extern "C" ew_status_t ew_pool_create(const ew_config_t *cfg, ew_pool_t **out) {
                 uint64_t d13[3] = {H, I, 2 * slots}, d2[3] = {I, H, slots};
                 uint32_t box[3] = {64, 128, 1};
                 if (make_tensor_map(p, &L.map_w13, (void *)L.w13.base, 3, d13, box) ||
-                    make_tensor_map(p, &L.map_w2, (void *)L.w2.base, 3, d2, box))
+                    make_tensor_map(p, &L.map_w2, (void *)L.w2.base, 3, d2, box) ||
+                    make_atom_map(p, &L.map_router, L.router_w, c.hidden, c.num_experts, (c.num_experts + 15) / 16 * 16, 4))
                     return EW_ERR_CUDA;
             }
             ew_status_t s = alloc_workspace(p);

@@ -1,5 +1,4 @@
 // Routing-side kernels of the adapter-aware MoE layer:
-//   route_kernel     router logits + softmax + top-k + batched rerouting + per-slot histogram (fused)
 //   reroute_kernel   the batched rerouting operator alone (Section 4.3) + histogram
 //   permute_kernel   exclusive scan of the counts, scatter of token rows into slot-contiguous order,
 //                    and (one extra CTA) the work-item lists of the grouped GEMMs
@@ -11,19 +10,6 @@
 namespace ew {
 namespace {
 
-constexpr int kMaxPerLane = 8;   // experts per lane: M <= 256
-
-__device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
-__device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
-
-__device__ __forceinline__ float dot8(const uint4 &a, const uint4 &b, float acc) {
-    acc = fmaf(bf_lo(a.x), bf_lo(b.x), acc); acc = fmaf(bf_hi(a.x), bf_hi(b.x), acc);
-    acc = fmaf(bf_lo(a.y), bf_lo(b.y), acc); acc = fmaf(bf_hi(a.y), bf_hi(b.y), acc);
-    acc = fmaf(bf_lo(a.z), bf_lo(b.z), acc); acc = fmaf(bf_hi(a.z), bf_hi(b.z), acc);
-    acc = fmaf(bf_lo(a.w), bf_lo(b.w), acc); acc = fmaf(bf_hi(a.w), bf_hi(b.w), acc);
-    return acc;
-}
-
 // slot = aid < 0 ? id : Pi[aid][id]; bad adapter ids behave as -1 and raise bit 0 of the error word
 __device__ __forceinline__ int checked_aid(int a, int N, const int32_t *loaded, int *err) {
     if (a < -1 || a >= N || (a >= 0 && !loaded[a])) {
@@ -31,100 +17,6 @@ __device__ __forceinline__ int checked_aid(int a, int N, const int32_t *loaded, 
         return -1;
     }
     return a;
-}
-
-// ------------------------------------------------------------------------------------------------
-// Fused router: one warp per token.  The token row sits in shared memory, router rows stream through
-// L1/L2 with 16-byte loads, fp32 accumulation, warp-shuffle reductions for the dot products, the
-// softmax statistics and the k arg-max rounds (value descending, index ascending).  The expert map
-// of the layer is staged in shared memory; the per-slot histogram is built with one atomic per pair,
-// whose return value is the pair's position inside its slot's chunk.
-// ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) route_kernel(const uint4 *__restrict__ x, const uint4 *__restrict__ wg,
-                                                    const int32_t *__restrict__ aid, const int32_t *__restrict__ pi,
-                                                    const int32_t *__restrict__ loaded, int B, int H, int M, int k, int N,
-                                                    int renormalize, float scale, int32_t *__restrict__ topk_ids,
-                                                    float *__restrict__ topk_w, int32_t *__restrict__ slot_ids,
-                                                    int32_t *__restrict__ rank, int32_t *__restrict__ counts, int *err) {
-    extern __shared__ uint4 smem4[];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int hv = H >> 3;                                   // 16-byte vectors per row
-    uint4 *xs = smem4 + (size_t)warp * hv;                   // this warp's token row
-    int32_t *pi_s = reinterpret_cast<int32_t *>(smem4 + (size_t)8 * hv);
-    for (int i = threadIdx.x; i < N * M; i += blockDim.x) pi_s[i] = pi[i];
-    const int t = blockIdx.x * 8 + warp;
-    if (t < B)
-        for (int v = lane; v < hv; v += 32) xs[v] = x[(size_t)t * hv + v];
-    __syncthreads();
-    if (t >= B) return;
-
-    float z[kMaxPerLane];                                    // lane holds experts j = q*32 + lane
-#pragma unroll
-    for (int q = 0; q < kMaxPerLane; ++q) z[q] = -INFINITY;
-#pragma unroll
-    for (int q = 0; q < kMaxPerLane; ++q) {
-        if (q * 32 < M) {
-            for (int jl = 0; jl < 32 && q * 32 + jl < M; ++jl) {
-                const uint4 *wr = wg + (size_t)(q * 32 + jl) * hv;
-                float acc = 0.f;
-                for (int v = lane; v < hv; v += 32) acc = dot8(xs[v], __ldg(wr + v), acc);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-                if (lane == jl) z[q] = acc;
-            }
-        }
-    }
-    // softmax over the M logits
-    float mx = z[0];
-#pragma unroll
-    for (int q = 1; q < kMaxPerLane; ++q) mx = fmaxf(mx, z[q]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    float sum = 0.f;
-#pragma unroll
-    for (int q = 0; q < kMaxPerLane; ++q) {
-        z[q] = (q * 32 + lane < M) ? expf(z[q] - mx) : -1.f;     // -1 marks "no expert here" (probabilities are >= 0)
-        sum += fmaxf(z[q], 0.f);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-#pragma unroll
-    for (int q = 0; q < kMaxPerLane; ++q)
-        if (z[q] >= 0.f) z[q] = z[q] / sum;
-    // k rounds of arg-max; lane r keeps the r-th selection
-    int my_id = 0;
-    float my_w = 0.f, wsum = 0.f;
-    for (int r = 0; r < k; ++r) {
-        float bv = -1.f;
-        int bi = 0x7fffffff;
-#pragma unroll
-        for (int q = 0; q < kMaxPerLane; ++q)
-            if (z[q] > bv) { bv = z[q]; bi = q * 32 + lane; }      // ascending q: the lower index keeps a tie
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-        }
-        if (lane == r) { my_id = bi; my_w = bv; }
-        wsum += bv;
-        if ((bi & 31) == lane) {
-#pragma unroll
-            for (int q = 0; q < kMaxPerLane; ++q)
-                if (q == (bi >> 5)) z[q] = -1.f;                     // taken
-        }
-    }
-    if (lane < k) {
-        if (renormalize) my_w = my_w / wsum;
-        my_w *= scale;
-        const int a = checked_aid(aid[t], N, loaded, err);
-        const int slot = a < 0 ? my_id : pi_s[a * M + my_id];
-        const size_t o = (size_t)t * k + lane;
-        topk_ids[o] = my_id;
-        topk_w[o] = my_w;
-        slot_ids[o] = slot;
-        rank[o] = atomicAdd(counts + slot, 1);
-    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -313,21 +205,6 @@ static int pick_token_tile(const ew_pool *p, int B) {
     const double mean = (double)B * p->cfg.top_k / p->cfg.num_experts;
     const double want = mean * 1.5;
     return want <= 32 ? 32 : want <= 64 ? 64 : want <= 128 ? 128 : 256;
-}
-
-int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B, cudaStream_t st) {
-    const ew_config_t &c = p->cfg;
-    const LayerState &L = p->layers[layer];
-    const size_t smem = (size_t)8 * c.hidden * 2 + (size_t)c.max_adapters * c.num_experts * 4 + 16;
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return (int)e;
-    }
-    route_kernel<<<(B + 7) / 8, 256, smem, st>>>((const uint4 *)x, (const uint4 *)L.router_w, aid, L.pi_dev, p->ws.loaded,
-                                                 B, c.hidden, c.num_experts, c.top_k, c.max_adapters, c.renormalize,
-                                                 c.routed_scale, p->ws.topk_ids, p->ws.topk_w, p->ws.slot_ids,
-                                                 p->ws.rank, p->ws.counts, p->ws.err);
-    return (int)cudaGetLastError();
 }
 
 int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st) {

@@ -1,0 +1,324 @@
+// Fused router kernel: logits on the tensor cores, then softmax + top-k + batched rerouting +
+// per-slot histogram in the epilogue (Sections 2.1 and 4.3).
+//
+// One CTA owns `tok_tile` (32, 64 or 128) tokens.  The logits tile D[128, M] = X[128, H] * Wr[M, H]^T is
+// one tcgen05 accumulator (M <= 256 fp32 columns of TMEM); X and the router rows stream through a TMA
+// ring.  The kernel is latency-bound, so each TMA instruction fetches kAtoms 64-element K-atoms at once
+// (3-D descriptors ordered element, row, atom: shared memory receives one swizzled tile per atom).  Only the first
+// `tok_tile` rows of the 128-row MMA tile are loaded; the other rows hold whatever shared memory held
+// and feed accumulator lanes nobody reads.  TMEM lane i belongs to token i, so in the epilogue every
+// thread owns one token: it reads its M logits from TMEM, forms the softmax probabilities in fp32, takes
+// k arg-max rounds (probability descending, lower index on ties), looks each chosen expert up in the
+// layer's expert map Pi (staged in shared memory) under the token's adapter id, and bumps the slot's
+// counter; the atomic's return value is the pair's position inside the slot's chunk.
+#include "ew_internal.h"
+#include "ew_tc.cuh"
+
+namespace ew {
+namespace {
+using namespace tc;
+
+constexpr int kThreads = 192;
+constexpr int kTileRows = 128;
+constexpr int kMaxStages = 16;
+constexpr int kAtoms = 4;            // 64-element K-atoms per TMA box and pipeline stage
+constexpr int kMaxPiSmem = 16 * 1024;
+
+__device__ __forceinline__ int checked_aid(int a, int N, const int32_t *loaded, int *err) {
+    if (a < -1 || a >= N || (a >= 0 && !loaded[a])) {
+        atomicOr(err, 1);
+        return -1;
+    }
+    return a;
+}
+
+struct RouterArgs {
+    const int32_t *aid, *pi, *loaded;
+    int B, H, M, k, N, renormalize;
+    float scale;
+    int stages, tmem_cols, pi_in_smem, tok_tile;
+    int32_t *topk_ids;
+    float *topk_w;
+    int32_t *slot_ids, *rank, *counts;
+    int *err;
+};
+
+// write one selected pair: reroute through Pi, outputs (the histogram follows in emit_ranks)
+__device__ __forceinline__ void emit_pair(const RouterArgs &A, const int32_t *pi_s, int t, int r, int a, int id, float w,
+                                          int (&sl)[8]) {
+    const int slot = a < 0 ? id : (A.pi_in_smem ? pi_s[a * A.M + id] : __ldg(A.pi + a * A.M + id));
+    const size_t o = (size_t)t * A.k + r;
+    A.topk_ids[o] = id;
+    A.topk_w[o] = w;
+    A.slot_ids[o] = slot;
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+        if (u == r) sl[u] = slot;       // the first eight slots stay in registers for emit_ranks
+}
+
+// per-slot histogram: one atomic per pair, eight in flight per thread; the value returned is the
+// pair's position inside its slot's chunk
+__device__ __forceinline__ void emit_ranks(const RouterArgs &A, int t, const int (&sl)[8]) {
+    for (int r0 = 0; r0 < A.k; r0 += 8) {
+        int got[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (r0 + u < A.k) got[u] = atomicAdd(A.counts + (r0 == 0 ? sl[u] : A.slot_ids[(size_t)t * A.k + r0 + u]), 1);
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (r0 + u < A.k) A.rank[(size_t)t * A.k + r0 + u] = got[u];
+    }
+}
+
+// REG = true: M <= 64, the token's probabilities stay in registers
+template <bool REG>
+__global__ void __launch_bounds__(kThreads, 1)
+router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_r, const RouterArgs A) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
+    const int M = A.M, stages = A.stages, tok_tile = A.tok_tile;
+    const int n_mma = ((M + 15) >> 4) << 4;                          // router rows arrive as one box of n_mma rows
+    const int x_atom = tok_tile * kBlockK * 2;                       // bytes of one K-atom of the token tile (multiple of 4 KiB)
+    const int r_atom = (n_mma * kBlockK * 2 + 1023) & ~1023;         // and of the router tile
+    const int x_bytes = kAtoms * x_atom;
+    const int stage_bytes = x_bytes + kAtoms * r_atom;
+    // ring, then 16 KiB of slack (the MMA reads a full 128-row A tile from every stage), then barriers
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_al + stages * stage_bytes + kTileRows * kBlockK * 2);
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kMaxStages, bar_done = bar_empty + 8 * kMaxStages;
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(bars + 2 * kMaxStages + 1);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
+    int32_t *pi_s = reinterpret_cast<int32_t *>(tmem_holder + 2);
+    float *pbuf = reinterpret_cast<float *>(smem_al);                // [M][128]; aliases the ring once it has drained
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_atoms = A.H / kBlockK;
+    const int num_kb = (num_atoms + kAtoms - 1) / kAtoms;
+    const int tok0 = blockIdx.x * tok_tile;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_done, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_map(&map_x);
+        prefetch_map(&map_r);
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)),
+                     "r"((uint32_t)A.tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (A.pi_in_smem)
+        for (int i = threadIdx.x; i < A.N * M; i += kThreads) pi_s[i] = A.pi[i];
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp == 0) {
+        if (lane == 0) {                                             // TMA producer
+            uint32_t stage = 0, phase = 0;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, abort_flag, A.err)) break;
+                const uint32_t sa = smem_base + stage * stage_bytes, full = bar_full + 8 * stage;
+                mbar_expect_tx(full, kAtoms * (tok_tile + n_mma) * kBlockK * 2);
+                tma_load_3d(sa, &map_x, 0, tok0, kb * kAtoms, full);
+                tma_load_3d(sa + x_bytes, &map_r, 0, 0, kb * kAtoms, full);
+                if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1; }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {                                             // MMA issuer
+            uint32_t stage = 0, phase = 0;
+            const uint32_t idesc = instr_desc(n_mma);
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; ++kb) {
+                if (!(ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, A.err))) break;
+                tc_fence_after();
+                const uint32_t sa = smem_base + stage * stage_bytes;
+                const int atoms = min(kAtoms, num_atoms - kb * kAtoms);      // atoms past H arrive zero-filled: skip them
+                for (int at = 0; at < atoms; ++at) {
+                    const uint64_t a = smem_desc_sw128(sa + at * x_atom), b = smem_desc_sw128(sa + x_bytes + at * r_atom);
+#pragma unroll
+                    for (int ki = 0; ki < kBlockK / 16; ++ki)
+                        tc_mma(tmem_base, a + 2 * ki, b + 2 * ki, idesc, (kb | at | ki) ? 1u : 0u);
+                }
+                tc_commit(bar_empty + 8 * stage);
+                if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1; }
+            }
+            if (ok) tc_commit(bar_done);
+        }
+    } else {
+        // epilogue: thread <-> token
+        const int lg = warp & 3;
+        const int tl = lg * 32 + lane;                               // token inside the tile = TMEM lane
+        const int t = tok0 + tl;
+        const int k = A.k;
+        if (lg * 32 < tok_tile && mbar_wait(bar_done, 0, abort_flag, A.err)) {
+            tc_fence_after();
+            const uint32_t t0 = tmem_base + ((uint32_t)(lg * 32) << 16);
+            if (REG) {
+                uint32_t v0[32], v1[32];
+                if (n_mma >= 32) tc_ld32(t0, v0); else tc_ld16(t0, v0);
+                if (n_mma > 32) { if (n_mma - 32 >= 32) tc_ld32(t0 + 32, v1); else tc_ld16(t0 + 32, v1); }
+                tc_wait_ld();
+                float p[64];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    p[j] = j < M ? __uint_as_float(v0[j]) : -INFINITY;
+                    p[32 + j] = 32 + j < M ? __uint_as_float(v1[j]) : -INFINITY;
+                }
+                float mx = p[0];
+#pragma unroll
+                for (int j = 1; j < 64; ++j) mx = fmaxf(mx, p[j]);
+                float sum = 0.f;
+#pragma unroll
+                for (int j = 0; j < 64; ++j) {                       // exp(-inf) = 0 for the absent experts
+                    p[j] = __expf(p[j] - mx);
+                    sum += p[j];
+                }
+                const float inv_sum = 1.f / sum;
+#pragma unroll
+                for (int j = 0; j < 64; ++j) p[j] = j < M ? p[j] * inv_sum : -1.f;
+                if (t < A.B) {
+                    const int a = checked_aid(A.aid[t], A.N, A.loaded, A.err);
+                    float wsum = 0.f;
+                    int sl[8];
+                    for (int r = 0; r < k; ++r) {
+                        float bv = -1.f;
+                        int bi = 0;
+#pragma unroll
+                        for (int j = 0; j < 64; ++j) {               // branch-free selects; strict >: the lower index keeps a tie
+                            const bool gt = p[j] > bv;
+                            bv = gt ? p[j] : bv;
+                            bi = gt ? j : bi;
+                        }
+#pragma unroll
+                        for (int j = 0; j < 64; ++j) p[j] = (j == bi) ? -1.f : p[j];   // taken (probabilities are >= 0)
+                        wsum += bv;
+                        emit_pair(A, pi_s, t, r, a, bi, bv, sl);
+                    }
+                    emit_ranks(A, t, sl);
+                    if (A.renormalize || A.scale != 1.f)
+                        for (int r = 0; r < k; ++r) {
+                            const size_t o = (size_t)t * k + r;
+                            float w = A.topk_w[o];
+                            if (A.renormalize) w = w / wsum;
+                            A.topk_w[o] = w * A.scale;
+                        }
+                }
+            } else {
+                uint32_t v[32];
+                float mx = -INFINITY;
+                for (int c0 = 0; c0 < n_mma; c0 += 32) {             // pass 1: max logit
+                    if (n_mma - c0 >= 32) tc_ld32(t0 + c0, v); else tc_ld16(t0 + c0, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (c0 + j < M) mx = fmaxf(mx, __uint_as_float(v[j]));
+                }
+                float sum = 0.f;
+                for (int c0 = 0; c0 < n_mma; c0 += 32) {             // pass 2: exponentials and their sum (j ascending)
+                    if (n_mma - c0 >= 32) tc_ld32(t0 + c0, v); else tc_ld16(t0 + c0, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (c0 + j < M) {
+                            const float e = expf(__uint_as_float(v[j]) - mx);
+                            pbuf[(c0 + j) * kTileRows + tl] = e;
+                            sum += e;
+                        }
+                }
+                for (int j = 0; j < M; ++j) pbuf[j * kTileRows + tl] = pbuf[j * kTileRows + tl] / sum;
+                if (t < A.B) {
+                    const int a = checked_aid(A.aid[t], A.N, A.loaded, A.err);
+                    float wsum = 0.f;
+                    int sl[8];
+                    for (int r = 0; r < k; ++r) {
+                        float bv = -1.f;
+                        int bi = 0;
+                        for (int j = 0; j < M; ++j) {
+                            const float pj = pbuf[j * kTileRows + tl];
+                            const bool gt = pj > bv;
+                            bv = gt ? pj : bv;
+                            bi = gt ? j : bi;
+                        }
+                        pbuf[bi * kTileRows + tl] = -1.f;
+                        wsum += bv;
+                        emit_pair(A, pi_s, t, r, a, bi, bv, sl);
+                    }
+                    emit_ranks(A, t, sl);
+                    if (A.renormalize || A.scale != 1.f)
+                        for (int r = 0; r < k; ++r) {
+                            const size_t o = (size_t)t * k + r;
+                            float w = A.topk_w[o];
+                            if (A.renormalize) w = w / wsum;
+                            A.topk_w[o] = w * A.scale;
+                        }
+                }
+            }
+        }
+    }
+
+    if (*abort_flag) {
+        long long c0 = clock64();
+        while (clock64() - c0 < 2000000ll) {}
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)A.tmem_cols)
+                     : "memory");
+}
+
+}  // namespace
+
+int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B, cudaStream_t st) {
+    const ew_config_t &c = p->cfg;
+    const LayerState &L = p->layers[layer];
+    const int M = c.num_experts;
+    const int n_mma = (M + 15) / 16 * 16;
+    // tokens per CTA: small batches are spread over more SMs (each CTA streams the whole router matrix)
+    const int tok_tile = B <= 32 * p->sm_count ? 32 : B <= 64 * p->sm_count ? 64 : 128;
+    const int stage_bytes = kAtoms * (tok_tile * kBlockK * 2 + ((n_mma * kBlockK * 2 + 1023) & ~1023));
+    const size_t pi_bytes = (size_t)c.max_adapters * M * 4;
+    const int pi_in_smem = pi_bytes <= (size_t)kMaxPiSmem;
+    const size_t tail = 1024 /*alignment*/ + kTileRows * kBlockK * 2 + 8 * (2 * kMaxStages + 1) + 16 +
+                        (pi_in_smem ? pi_bytes : 0) + 64;
+    int stages = (int)((227 * 1024 - tail) / stage_bytes);
+    if (stages > kMaxStages) stages = kMaxStages;
+    const bool reg = M <= 64;
+    const size_t pbuf_bytes = reg ? 0 : (size_t)M * kTileRows * 4;
+    if ((size_t)stages * stage_bytes + kTileRows * kBlockK * 2 < pbuf_bytes || stages < 2)
+        return (int)cudaErrorInvalidConfiguration;
+    const size_t smem = (size_t)stages * stage_bytes + tail;
+    CUtensorMap map_x;
+    if (make_atom_map(p, &map_x, x, c.hidden, B, tok_tile, kAtoms)) return (int)cudaErrorInvalidValue;
+    RouterArgs A;
+    A.aid = aid; A.pi = L.pi_dev; A.loaded = p->ws.loaded;
+    A.B = B; A.H = c.hidden; A.M = M; A.k = c.top_k; A.N = c.max_adapters; A.renormalize = c.renormalize;
+    A.scale = c.routed_scale;
+    A.stages = stages; A.tmem_cols = n_mma <= 32 ? 32 : n_mma <= 64 ? 64 : n_mma <= 128 ? 128 : 256;
+    A.pi_in_smem = pi_in_smem; A.tok_tile = tok_tile;
+    A.topk_ids = p->ws.topk_ids; A.topk_w = p->ws.topk_w; A.slot_ids = p->ws.slot_ids; A.rank = p->ws.rank;
+    A.counts = p->ws.counts; A.err = p->ws.err;
+    static size_t attr_set[2] = {0, 0};
+    if (smem > attr_set[reg]) {
+        cudaError_t e = reg ? cudaFuncSetAttribute(router_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                            : cudaFuncSetAttribute(router_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+        attr_set[reg] = smem;
+    }
+    const int grid = (B + tok_tile - 1) / tok_tile;
+    if (reg) router_kernel<true><<<grid, kThreads, smem, st>>>(map_x, L.map_router, A);
+    else router_kernel<false><<<grid, kThreads, smem, st>>>(map_x, L.map_router, A);
+    return (int)cudaGetLastError();
+}
+
+}  // namespace ew

@@ -34,7 +34,7 @@ def test_status_strings(lib):
 def test_argument_errors_without_a_gpu(lib):
     assert lib.ew_pool_create(None, None) == 1
     h = C.c_void_p()
-    bad = binding.EwConfig(-1, 1, 250, 128, 16, 1, 2, 2, 3, 64, 0, 1.0, 0, 0, 0, 0, 0)   # H not a multiple of 8
+    bad = binding.EwConfig(-1, 1, 250, 128, 16, 1, 2, 2, 3, 64, 0, 1.0, 0, 0, 0, 0, 0)   # H not a multiple of 64
     assert lib.ew_pool_create(C.byref(bad), C.byref(h)) == 1
     bad = binding.EwConfig(-1, 1, 256, 128, 16, 1, 17, 2, 3, 64, 0, 1.0, 0, 0, 0, 0, 0)  # k > M
     assert lib.ew_pool_create(C.byref(bad), C.byref(h)) == 1

@@ -184,6 +184,30 @@ ew_status_t ew_profile_read(ew_pool_t *pool, double *ms, int32_t *n_forwards);
 ew_status_t ew_reroute(ew_pool_t *pool, int32_t layer, const int32_t *topk_ids, const int32_t *adapter_ids,
                        int32_t n_tokens, int32_t *slot_ids, int32_t *counts, void *cuda_stream);
 
+/* Routing without any allocation (the paper has no counterpart: this entry point exists for callers
+ * of this library that cannot allocate device memory when they need a routing decision - an engine
+ * whose KV cache has taken all free HBM, code running where the CUDA allocator must not be entered,
+ * or a second batch to route while a forward on this pool, which owns a single workspace, is still in
+ * flight).  It runs the same fused router kernel as ew_moe_forward (logits, softmax, top-k, batched
+ * rerouting, per-slot counts) for x [n_tokens,H] and writes into buffers the CALLER provides:
+ *   topk_ids, slot_ids [n_tokens,k] int32; topk_w [n_tokens,k] float; counts [M + N*E_max] int32
+ *   (overwritten); device_status (optional, device int32): 0 or EW_ERR_BAD_ADAPTER_ID_IN_BATCH-style
+ *   bit set as in ew_last_device_error's word (bit 0 bad adapter id, bit 1 expired wait).
+ * All pointers DEVICE.  The kernel's scratch lives in one fixed array inside the library (about 256 KiB
+ * per GPU, held until the process exits); therefore
+ *   - n_tokens * top_k must not exceed 65536, otherwise EW_ERR_INVALID_ARG and nothing is launched;
+ *   - the call performs no cudaMalloc / cudaFree and enters no allocating library routine;
+ *   - the first call on a device resolves the array's device address (cudaGetSymbolAddress): make that
+ *     first call before any stream capture begins;
+ *   - all calls share the array, which still holds the previous call's contents (the words that must
+ *     start at zero are cleared on the stream at the start of each call): two calls that overlap on
+ *     the GPU (different streams, no ordering) race on it.  Order them.
+ * The pool's weights and expert maps are read, its workspace is not touched.
+ * Errors: EW_ERR_INVALID_ARG, EW_ERR_NOT_LOADED, EW_ERR_NO_DEVICE, EW_ERR_CUDA. */
+ew_status_t ew_route_noalloc(ew_pool_t *pool, int32_t layer, const void *x, const int32_t *adapter_ids,
+                             int32_t n_tokens, int32_t *topk_ids, float *topk_w, int32_t *slot_ids,
+                             int32_t *counts, int32_t *device_status, void *cuda_stream);
+
 /* Copy one layer's expert map Pi^(l) [N,M] to HOST memory (the host-side master copy). */
 ew_status_t ew_get_expert_map(ew_pool_t *pool, int32_t layer, int32_t *host_out);
 

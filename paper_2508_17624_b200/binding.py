@@ -22,7 +22,7 @@ STATUS_NAMES = ["EW_OK", "EW_ERR_INVALID_ARG", "EW_ERR_OOM", "EW_ERR_SLOT_IN_USE
                 "EW_ERR_NO_DEVICE"]
 EXPORTS = ["ew_pool_create", "ew_pool_destroy", "ew_load_base", "ew_load_adapter", "ew_unload_adapter",
            "ew_pool_trim", "ew_moe_forward", "ew_moe_forward_debug", "ew_moe_forward_host", "ew_profile_enable",
-           "ew_profile_read", "ew_reroute", "ew_get_expert_map",
+           "ew_profile_read", "ew_reroute", "ew_route_noalloc", "ew_get_expert_map",
            "ew_pool_stats", "ew_last_device_error", "ew_slot_address", "ew_status_str", "ew_last_error_string"]
 
 
@@ -201,6 +201,12 @@ class Pool:
         _check(lib().ew_reroute(self._h, layer, _dp(topk_ids), _dp(adapter_ids), topk_ids.shape[0], _dp(slot_ids),
                                 _dp(counts), _stream()), "ew_reroute")
         return slot_ids, counts
+
+    def route_noalloc(self, layer, x, adapter_ids, topk_ids, topk_w, slot_ids, counts, device_status=None):
+        """Routing into caller-provided device tensors; the library allocates nothing (see the header)."""
+        _check(lib().ew_route_noalloc(self._h, layer, _dp(x), _dp(adapter_ids), x.shape[0], _dp(topk_ids),
+                                      _dp(topk_w), _dp(slot_ids), _dp(counts), _dp(device_status), _stream()),
+               "ew_route_noalloc")
 
     def get_expert_map(self, layer) -> np.ndarray:
         out = np.empty((self.cfg.max_adapters, self.cfg.num_experts), np.int32)

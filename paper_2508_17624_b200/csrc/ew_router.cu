@@ -11,6 +11,9 @@
 // k arg-max rounds (probability descending, lower index on ties), looks each chosen expert up in the
 // layer's expert map Pi (staged in shared memory) under the token's adapter id, and bumps the slot's
 // counter; the atomic's return value is the pair's position inside the slot's chunk.
+#include <mutex>
+#include <string>
+
 #include "ew_internal.h"
 #include "ew_tc.cuh"
 
@@ -322,3 +325,117 @@ int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B
 }
 
 }  // namespace ew
+
+// ================================================================================================
+// Allocation-free routing.
+//
+// Some callers may not allocate device memory at the moment they need a routing decision: a serving
+// engine that has handed every free byte of HBM to its KV cache (any cudaMalloc then fails or
+// fragments), or code that runs where the CUDA allocator must not be entered at all.  The pool's own
+// forward never allocates either, but it owns exactly one workspace, so a second batch cannot be routed
+// while a forward is in flight without a second workspace, i.e. an allocation.  ew_route_noalloc runs
+// the fused router kernel with the caller's output buffers and keeps the kernel's scratch (the
+// device status word and the per-pair positions inside each slot) in the fixed array below, which every
+// GPU that loads this library holds until the process exits.
+// ================================================================================================
+namespace ew {
+namespace {
+constexpr int kNoAllocMaxPairs = 65536;                 // n_tokens * top_k accepted by ew_route_noalloc
+constexpr int kNoAllocHeader = 256;                     // bytes before the per-pair array; word 0 = status
+}  // namespace
+}  // namespace ew
+
+static __device__ __align__(256) unsigned char g_route_noalloc_scratch[ew::kNoAllocHeader + ew::kNoAllocMaxPairs * 4];
+
+namespace ew {
+namespace {
+std::mutex g_noalloc_mu;
+unsigned char *g_noalloc_ptr[64] = {};                  // device address of the array, per device ordinal
+
+// The array's name is only a host-side handle: resolve its device address once per device, with that
+// device current, and hand the address to the kernel.
+int noalloc_scratch(int device, unsigned char **out) {
+    if (device < 0 || device >= 64) return (int)cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_noalloc_mu);
+    if (!g_noalloc_ptr[device]) {
+        void *ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_route_noalloc_scratch);
+        if (e != cudaSuccess) return (int)e;
+        g_noalloc_ptr[device] = static_cast<unsigned char *>(ptr);
+    }
+    *out = g_noalloc_ptr[device];
+    return 0;
+}
+}  // namespace
+}  // namespace ew
+
+extern "C" ew_status_t ew_route_noalloc(ew_pool_t *p, int32_t layer, const void *x, const int32_t *adapter_ids,
+                                        int32_t n_tokens, int32_t *topk_ids, float *topk_w, int32_t *slot_ids,
+                                        int32_t *counts, int32_t *device_status, void *cuda_stream) {
+    using namespace ew;
+    if (!p || layer < 0 || layer >= p->cfg.num_layers || n_tokens < 0) return EW_ERR_INVALID_ARG;
+    if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
+    const ew_config_t &c = p->cfg;
+    if ((long long)n_tokens * c.top_k > kNoAllocMaxPairs) {
+        set_last_error("ew_route_noalloc: n_tokens * top_k exceeds the fixed scratch array (65536 pairs)");
+        return EW_ERR_INVALID_ARG;
+    }
+    if (!counts) return EW_ERR_INVALID_ARG;
+    if (!p->layers[layer].base_loaded) return EW_ERR_NOT_LOADED;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess && dev != c.device) e = cudaSetDevice(c.device);
+    unsigned char *scratch = nullptr;
+    int rc = e == cudaSuccess ? noalloc_scratch(c.device, &scratch) : (int)e;
+    // the array keeps the previous call's contents: the status word and the counters must start at zero
+    if (!rc) rc = (int)cudaMemsetAsync(scratch, 0, kNoAllocHeader, st);
+    if (!rc) rc = (int)cudaMemsetAsync(counts, 0, (size_t)p->P * 4, st);
+    if (rc) {
+        set_last_error(std::string("ew_route_noalloc: ") + cudaGetErrorString((cudaError_t)rc));
+        return EW_ERR_CUDA;
+    }
+    if (n_tokens == 0) return EW_OK;
+    if (!x || !adapter_ids || !topk_ids || !topk_w || !slot_ids || ((uintptr_t)x & 15)) return EW_ERR_INVALID_ARG;
+
+    const LayerState &L = p->layers[layer];
+    const int M = c.num_experts, B = n_tokens;
+    const int n_mma = (M + 15) / 16 * 16;
+    const int tok_tile = B <= 32 * p->sm_count ? 32 : B <= 64 * p->sm_count ? 64 : 128;
+    const int stage_bytes = kAtoms * (tok_tile * kBlockK * 2 + ((n_mma * kBlockK * 2 + 1023) & ~1023));
+    const size_t pi_bytes = (size_t)c.max_adapters * M * 4;
+    const int pi_in_smem = pi_bytes <= (size_t)kMaxPiSmem;
+    const size_t tail = 1024 + kTileRows * kBlockK * 2 + 8 * (2 * kMaxStages + 1) + 16 + (pi_in_smem ? pi_bytes : 0) + 64;
+    int stages = (int)((227 * 1024 - tail) / stage_bytes);
+    if (stages > kMaxStages) stages = kMaxStages;
+    const bool reg = M <= 64;
+    if (stages < 2 || (!reg && (size_t)stages * stage_bytes + kTileRows * kBlockK * 2 < (size_t)M * kTileRows * 4))
+        return EW_ERR_INVALID_ARG;
+    const size_t smem = (size_t)stages * stage_bytes + tail;
+    CUtensorMap map_x;
+    if (make_atom_map(p, &map_x, x, c.hidden, B, tok_tile, kAtoms)) return EW_ERR_CUDA;
+    RouterArgs A;
+    A.aid = adapter_ids; A.pi = L.pi_dev; A.loaded = p->ws.loaded;
+    A.B = B; A.H = c.hidden; A.M = M; A.k = c.top_k; A.N = c.max_adapters; A.renormalize = c.renormalize;
+    A.scale = c.routed_scale;
+    A.stages = stages; A.tmem_cols = n_mma <= 32 ? 32 : n_mma <= 64 ? 64 : n_mma <= 128 ? 128 : 256;
+    A.pi_in_smem = pi_in_smem; A.tok_tile = tok_tile;
+    A.topk_ids = topk_ids; A.topk_w = topk_w; A.slot_ids = slot_ids; A.counts = counts;
+    A.rank = reinterpret_cast<int32_t *>(scratch + kNoAllocHeader);      // scratch: position of each pair in its slot
+    A.err = reinterpret_cast<int *>(scratch);                            // scratch: device status word
+    e = reg ? cudaFuncSetAttribute(router_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
+            : cudaFuncSetAttribute(router_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess) {
+        const int grid = (B + tok_tile - 1) / tok_tile;
+        if (reg) router_kernel<true><<<grid, kThreads, smem, st>>>(map_x, L.map_router, A);
+        else router_kernel<false><<<grid, kThreads, smem, st>>>(map_x, L.map_router, A);
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess && device_status)
+        e = cudaMemcpyAsync(device_status, scratch, 4, cudaMemcpyDeviceToDevice, st);
+    if (e != cudaSuccess) {
+        set_last_error(std::string("ew_route_noalloc: ") + cudaGetErrorString(e));
+        return EW_ERR_CUDA;
+    }
+    return EW_OK;
+}

@@ -49,7 +49,8 @@ struct Cfg {
 template <int NT, bool GLU>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
-                    const __grid_constant__ CUtensorMap map_x, const GemmItem *__restrict__ items,
+                    const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_a_big,
+                    const __grid_constant__ CUtensorMap map_x_big, const GemmItem *__restrict__ items,
                     const int32_t *__restrict__ n_items_ptr, int K, int out_rows_per_slot, void *__restrict__ out,
                     int *err) {
     using C = Cfg<NT, GLU>;
@@ -101,12 +102,15 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
             for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
                 const GemmItem it = items[w];
                 const int nchunk = (it.rows + kChunkRows - 1) / kChunkRows;
-                const CUtensorMap *amap = (GLU && it.from_x) ? &map_x : &map_a;
+                // thin items fetch their rows in 32-row boxes; fat ones (prefill) with one NT-row box per stage
+                const bool big = NT >= 128 && it.rows > 2 * kChunkRows;
+                const CUtensorMap *amap = (GLU && it.from_x) ? (big ? &map_x_big : &map_x) : (big ? &map_a_big : &map_a);
+                const uint32_t b_bytes = big ? NT * kBlockK * 2 : nchunk * kChunkBytes;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1, abort_flag, err))) break;
                     const uint32_t sa = smem_base + stage * C::kStageBytes;
                     const uint32_t full = bar_full + 8 * stage;
-                    mbar_expect_tx(full, (GLU ? 2 : 1) * kATileBytes + nchunk * kChunkBytes);
+                    mbar_expect_tx(full, (GLU ? 2 : 1) * kATileBytes + b_bytes);
                     if (GLU) {
                         tma_load_3d(sa, &map_w, kb * kBlockK, it.tile * kTileRows, it.slot * 2, full);
                         tma_load_3d(sa + kATileBytes, &map_w, kb * kBlockK, it.tile * kTileRows, it.slot * 2 + 1, full);
@@ -114,8 +118,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
                         tma_load_3d(sa, &map_w, kb * kBlockK, it.tile * kTileRows, it.slot, full);
                     }
                     const uint32_t sb = sa + (GLU ? 2 : 1) * kATileBytes;
-                    for (int c = 0; c < nchunk; ++c)
-                        tma_load_2d(sb + c * kChunkBytes, amap, kb * kBlockK, it.in_row + c * kChunkRows, full);
+                    if (big) {
+                        tma_load_2d(sb, amap, kb * kBlockK, it.in_row, full);
+                    } else {
+                        for (int c = 0; c < nchunk; ++c)
+                            tma_load_2d(sb + c * kChunkBytes, amap, kb * kBlockK, it.in_row + c * kChunkRows, full);
+                    }
                     if (++stage == C::kStages) { stage = 0; phase ^= 1; }
                 }
             }
@@ -216,11 +224,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
 }
 
 template <int NT, bool GLU>
-int launch_one(ew_pool *p, const CUtensorMap &mw, const CUtensorMap &ma, const CUtensorMap &mx, const GemmItem *items,
-               const int32_t *n_items, int K, int out_rows, void *out, cudaStream_t st) {
+int launch_one(ew_pool *p, const CUtensorMap &mw, const CUtensorMap &ma, const CUtensorMap &mx, const CUtensorMap &mab,
+               const CUtensorMap &mxb, const GemmItem *items, const int32_t *n_items, int K, int out_rows, void *out,
+               cudaStream_t st) {
     using C = Cfg<NT, GLU>;
-    grouped_gemm_kernel<NT, GLU><<<p->sm_count, kThreads, C::kSmemBytes, st>>>(mw, ma, mx, items, n_items, K, out_rows,
-                                                                              out, p->ws.err);
+    grouped_gemm_kernel<NT, GLU><<<p->sm_count, kThreads, C::kSmemBytes, st>>>(mw, ma, mx, mab, mxb, items, n_items, K,
+                                                                              out_rows, out, p->ws.err);
     return (int)cudaGetLastError();
 }
 
@@ -240,25 +249,28 @@ int gemm_setup(ew_pool *) {
     return rc;
 }
 
-int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, int, cudaStream_t st) {
+int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, const CUtensorMap &map_x_big, int, cudaStream_t st) {
     const LayerState &L = p->layers[layer];
     const int K = p->cfg.hidden, I = p->cfg.inter;
+    const Workspace &w = p->ws;
     switch (p->token_tile) {
-        case 32: return launch_one<32, true>(p, L.map_w13, p->map_xp, map_x, p->ws.items1, p->ws.n_items, K, I, p->ws.act, st);
-        case 64: return launch_one<64, true>(p, L.map_w13, p->map_xp, map_x, p->ws.items1, p->ws.n_items, K, I, p->ws.act, st);
-        case 128: return launch_one<128, true>(p, L.map_w13, p->map_xp, map_x, p->ws.items1, p->ws.n_items, K, I, p->ws.act, st);
-        default: return launch_one<256, true>(p, L.map_w13, p->map_xp, map_x, p->ws.items1, p->ws.n_items, K, I, p->ws.act, st);
+        case 32: return launch_one<32, true>(p, L.map_w13, p->map_xp, map_x, p->map_xp, map_x, w.items1, w.n_items, K, I, w.act, st);
+        case 64: return launch_one<64, true>(p, L.map_w13, p->map_xp, map_x, p->map_xp, map_x, w.items1, w.n_items, K, I, w.act, st);
+        case 128: return launch_one<128, true>(p, L.map_w13, p->map_xp, map_x, p->map_xp_big[0], map_x_big, w.items1, w.n_items, K, I, w.act, st);
+        default: return launch_one<256, true>(p, L.map_w13, p->map_xp, map_x, p->map_xp_big[1], map_x_big, w.items1, w.n_items, K, I, w.act, st);
     }
 }
 
 int launch_gemm2(ew_pool *p, int layer, int, cudaStream_t st) {
     const LayerState &L = p->layers[layer];
     const int K = p->cfg.inter, H = p->cfg.hidden;
+    const Workspace &w = p->ws;
+    const CUtensorMap &a = p->map_act;
     switch (p->token_tile) {
-        case 32: return launch_one<32, false>(p, L.map_w2, p->map_act, p->map_act, p->ws.items2, p->ws.n_items + 1, K, H, p->ws.y, st);
-        case 64: return launch_one<64, false>(p, L.map_w2, p->map_act, p->map_act, p->ws.items2, p->ws.n_items + 1, K, H, p->ws.y, st);
-        case 128: return launch_one<128, false>(p, L.map_w2, p->map_act, p->map_act, p->ws.items2, p->ws.n_items + 1, K, H, p->ws.y, st);
-        default: return launch_one<256, false>(p, L.map_w2, p->map_act, p->map_act, p->ws.items2, p->ws.n_items + 1, K, H, p->ws.y, st);
+        case 32: return launch_one<32, false>(p, L.map_w2, a, a, a, a, w.items2, w.n_items + 1, K, H, w.y, st);
+        case 64: return launch_one<64, false>(p, L.map_w2, a, a, a, a, w.items2, w.n_items + 1, K, H, w.y, st);
+        case 128: return launch_one<128, false>(p, L.map_w2, a, a, p->map_act_big[0], a, w.items2, w.n_items + 1, K, H, w.y, st);
+        default: return launch_one<256, false>(p, L.map_w2, a, a, p->map_act_big[1], a, w.items2, w.n_items + 1, K, H, w.y, st);
     }
 }
 

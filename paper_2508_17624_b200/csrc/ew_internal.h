@@ -66,7 +66,8 @@ struct ew_pool {
     std::vector<ew::LayerState> layers;
     std::vector<std::vector<int32_t>> adapter_counts;   // [N][L]; empty = not loaded
     ew::Workspace ws;
-    CUtensorMap map_xp, map_act;   // TMA descriptors over the workspace activations
+    CUtensorMap map_xp, map_act;   // TMA descriptors over the workspace activations (box 64 x 32 rows)
+    CUtensorMap map_xp_big[2], map_act_big[2];   // same with 128- and 256-row boxes (prefill token tiles)
     cudaStream_t copy_stream = nullptr;
     std::vector<std::pair<cudaStream_t, cudaEvent_t>> fwd_events;   // last forward per caller stream
     int sm_count = 148;
@@ -96,7 +97,8 @@ int make_atom_map(ew_pool *p, CUtensorMap *out, const void *base, int H, int row
 // Kernel launchers (all asynchronous on `st`; return cudaError_t as int).
 int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B, cudaStream_t st);
 int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st);
-int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, int B, cudaStream_t st);
+int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, const CUtensorMap &map_x_big, int B, cudaStream_t st);
+int pick_token_tile(const ew_pool *p, int B);
 int launch_gemm2(ew_pool *p, int layer, int B, cudaStream_t st);
 int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st);
 int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid, int B, int32_t *slots,

@@ -119,6 +119,11 @@ static ew_status_t alloc_workspace(ew_pool *p) {
     uint32_t box[2] = {64, 32};
     if (make_tensor_map(p, &p->map_xp, w.xp, 2, d_xp, box) || make_tensor_map(p, &p->map_act, w.act, 2, d_act, box))
         return EW_ERR_CUDA;
+    for (int v = 0; v < 2; ++v) {
+        uint32_t bbox[2] = {64, v ? 256u : 128u};
+        if (make_tensor_map(p, &p->map_xp_big[v], w.xp, 2, d_xp, bbox) || make_tensor_map(p, &p->map_act_big[v], w.act, 2, d_act, bbox))
+            return EW_ERR_CUDA;
+    }
     return EW_OK;
 }
 
@@ -510,6 +515,12 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     uint64_t dx[2] = {(uint64_t)c.hidden, (uint64_t)B};
     uint32_t box[2] = {64, 32};
     if (make_tensor_map(p, &map_x, x, 2, dx, box)) return EW_ERR_CUDA;
+    CUtensorMap map_x_big = map_x;
+    p->token_tile = pick_token_tile(p, B);
+    if (p->token_tile >= 128) {
+        uint32_t bbox[2] = {64, (uint32_t)p->token_tile};
+        if (make_tensor_map(p, &map_x_big, x, 2, dx, bbox)) return EW_ERR_CUDA;
+    }
     size_t nk = (size_t)B * c.top_k;
     cudaEvent_t *pe = nullptr;
     if (p->profiling && p->prof_used + 6 <= 6 * 4096) {
@@ -534,7 +545,7 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     if (counts) CU_TRY(cudaMemcpyAsync(counts, p->ws.counts, (size_t)p->P * 4, cudaMemcpyDeviceToDevice, st));
     if (inv) CU_TRY(cudaMemcpyAsync(inv, p->ws.inv, nk * 4, cudaMemcpyDeviceToDevice, st));
     if (offsets) CU_TRY(cudaMemcpyAsync(offsets, p->ws.offsets, ((size_t)p->P + 1) * 4, cudaMemcpyDeviceToDevice, st));
-    LAUNCH_TRY(launch_gemm1(p, layer, map_x, B, st));
+    LAUNCH_TRY(launch_gemm1(p, layer, map_x, map_x_big, B, st));
     PROF_MARK(3);
     LAUNCH_TRY(launch_gemm2(p, layer, B, st));
     PROF_MARK(4);

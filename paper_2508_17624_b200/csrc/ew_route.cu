@@ -201,7 +201,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const float4 *__restrict__
 }  // namespace
 
 // Token rows per GEMM work item: the smallest tile that holds ~1.5x the mean rows per routed expert.
-static int pick_token_tile(const ew_pool *p, int B) {
+int pick_token_tile(const ew_pool *p, int B) {
     const double mean = (double)B * p->cfg.top_k / p->cfg.num_experts;
     const double want = mean * 1.5;
     return want <= 32 ? 32 : want <= 64 ? 64 : want <= 128 ? 128 : 256;
@@ -209,7 +209,6 @@ static int pick_token_tile(const ew_pool *p, int B) {
 
 int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
-    p->token_tile = pick_token_tile(p, B);
     const int R1 = (c.inter + 127) / 128, R2 = (c.hidden + 127) / 128;
     const long long pairs = (long long)B * c.top_k;
     const int grid = (int)((pairs + 7) / 8) + 1;

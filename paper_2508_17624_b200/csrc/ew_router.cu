@@ -182,7 +182,7 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                 float sum = 0.f;
 #pragma unroll
                 for (int j = 0; j < 64; ++j) {                       // exp(-inf) = 0 for the absent experts
-                    p[j] = __expf(p[j] - mx);
+                    p[j] = expf(p[j] - mx);
                     sum += p[j];
                 }
                 const float inv_sum = 1.f / sum;

@@ -10,7 +10,11 @@ from paper_2508_17624_b200 import workloads as wl
 NEAR_TIE = 1e-5          # a token whose k-th and (k+1)-th probabilities differ by less is a near-tie
 REL_L2_TOL = 1e-2        # bf16 layer output vs the fp32 oracle
 MAX_ABS_TOL = 2e-2
-WEIGHT_TOL = 2e-6        # combine weights (fp32 softmax on both sides, different exp / summation order)
+# Combine weights: both sides accumulate the H-term logit in fp32 but in a different order (sequential
+# vs the tensor core's tree), which moves a logit by up to ~1e-5 (sqrt(H) * 2^-24 * sum|x_h w_h| with
+# H = 2048, sum|x w| ~ 26); d p = p (1 - p) d z, so the weights agree to a relative 2e-5.
+WEIGHT_RTOL = 2e-5
+WEIGHT_TOL = 1e-7        # absolute floor
 
 
 def oracle_config(cfg: wl.MoEConfig) -> oracle.OracleConfig:
@@ -67,7 +71,7 @@ def check_routing(cfg, olayer, x_bits, aid, r, Pi=None):
         lut = {int(j): float(w) for j, w in zip(ids_o[t], w_o[t])}
         for c in range(k):
             wo = lut[int(ids_g[t, c])]
-            assert abs(wo - w_g[t, c]) <= WEIGHT_TOL, (t, c, wo, w_g[t, c])
+            assert abs(wo - w_g[t, c]) <= WEIGHT_TOL + WEIGHT_RTOL * wo, (t, c, wo, w_g[t, c])
             w_ffn[t, c] = wo
         if gap[t] >= NEAR_TIE and np.min(np.abs(np.diff(np.sort(w_o[t])))) >= NEAR_TIE:
             assert ids_g[t].tolist() == ids_o[t].tolist(), f"token {t}: order differs"

@@ -149,3 +149,100 @@ def test_reroute_operator_c4_sample():
     assert np.array_equal(cnt.cpu().numpy(), oracle.counts(want, cfg.num_slots))
     assert pool.last_device_error() == 0
     pool.destroy()
+
+
+def test_c2_prefill_layer():
+    """8192 tokens, 20 adapters: routing checked for every token, the layer output on a seeded sample."""
+    cfg = wl.CONFIGS["c2"]
+    sample = np.random.default_rng(2).choice(cfg.n_tokens, size=192, replace=False)
+    res = run_layer(cfg, sample=np.sort(sample))
+    print("c2", {k: v for k, v in res.items() if k in ("flips", "rel", "max_abs")})
+    assert res["flips"] <= 40
+    counts = np.bincount(res["slots"].reshape(-1), minlength=cfg.num_slots)
+    assert counts[:cfg.num_experts].min() > 256            # base slots are fat (several token blocks) ...
+    assert ((counts[cfg.num_experts:] > 0) & (counts[cfg.num_experts:] < 256)).any()   # ... adapter slots thin
+
+
+def test_c4_reroute_full_size():
+    """65536 tokens, 20 adapters re-tuning 10 %, 25 % and 50 % of the experts: ids and counts bit-exact."""
+    import torch
+    cfg = wl.CONFIGS["c4"]
+    oc = oracle.OracleConfig(cfg.hidden, cfg.inter, cfg.num_experts, 0, cfg.top_k, cfg.max_adapters, cfg.e_max)
+    ids, _, _ = oracle.topk_from_logits(oc, wl.gen_logits(cfg))
+    aid = wl.gen_adapter_ids(cfg, mode="uniform")
+    assert set(np.unique(aid)) == set(range(-1, cfg.max_adapters))
+    pool = binding.Pool(hidden=64, inter=64, num_experts=cfg.num_experts, num_shared=0, top_k=cfg.top_k,
+                        max_adapters=cfg.max_adapters, e_max=cfg.e_max, max_tokens=8)
+    z = np.zeros((cfg.num_experts, 64, 64), np.uint16)
+    pool.load_base(0, np.zeros((cfg.num_experts, 64), np.uint16), z, z, z)
+    d_ids, d_aid = to_dev(ids), to_dev(aid)
+    for e in (6, 16, 32):
+        tuned = wl.tuned_sets(cfg, np.full((cfg.max_adapters, 1), e))
+        za = np.zeros((e, 64, 64), np.uint16)
+        for i in range(cfg.max_adapters):
+            pool.load_adapter(i, np.array([e], np.int32), tuned[i][0], za, za, za)
+        Pi = oracle.build_map(cfg.num_experts, cfg.max_adapters, cfg.e_max, [t[0] for t in tuned])
+        slots, cnt = pool.reroute(0, d_ids, d_aid)
+        torch.cuda.synchronize()
+        want = oracle.reroute(ids, aid, Pi)
+        assert np.array_equal(slots.cpu().numpy(), want)
+        assert np.array_equal(cnt.cpu().numpy(), oracle.counts(want, cfg.num_slots))
+        redirected = float((want >= cfg.num_experts).mean())
+        assert abs(redirected - (e / 64) * 20 / 21) < 0.02      # tuned fraction x share of non-base tokens
+        # in place (slot_ids aliasing topk_ids) gives the same result
+        buf = d_ids.clone()
+        pool.reroute(0, buf, d_aid, slot_ids=buf, want_counts=False)
+        torch.cuda.synchronize()
+        assert np.array_equal(buf.cpu().numpy(), want)
+        for i in range(cfg.max_adapters):
+            pool.unload_adapter(i)
+    assert pool.last_device_error() == 0
+    pool.destroy()
+
+
+def test_c3_stacked_layers():
+    """26 layers of the decode shape resident in one pool through the virtual weight tensors (fewer layers
+    if the device has less free memory), 20 adapters, Zipf adapter popularity; three layers are checked."""
+    import torch
+    cfg = wl.CONFIGS["c3"]
+    per_layer = (66 + 20 * 9) * 3 * cfg.inter * cfg.hidden * 2
+    free, _ = torch.cuda.mem_get_info()
+    L = int(min(cfg.num_layers, max(2, (free - (12 << 30)) // per_layer)))
+    cfg = wl.with_(cfg, num_layers=L)
+    print(f"c3: {L} layers resident")
+    bank = wl.NoiseBank(cfg.seed)
+    pool = binding.Pool.from_config(cfg)
+    tuned = wl.tuned_sets(cfg)
+    check = sorted({0, L // 2, L - 1})
+    bases = {}
+    for l in range(L):
+        b = wl.gen_base_layer(cfg, l, bank)
+        pool.load_base(l, b.router_w, b.routed.w_gate, b.routed.w_up, b.routed.w_down,
+                       b.shared.w_gate, b.shared.w_up, b.shared.w_down)
+        if l in check:
+            bases[l] = b
+    for i in range(cfg.max_adapters):
+        per = [wl.gen_adapter_layer(cfg, i, l, tuned[i][l], bank) for l in range(L)]
+        pool.load_adapter(i, np.array([len(tuned[i][l]) for l in range(L)], np.int32),
+                          np.concatenate([tuned[i][l] for l in range(L)]),
+                          np.concatenate([e.w_gate for e in per]), np.concatenate([e.w_up for e in per]),
+                          np.concatenate([e.w_down for e in per]))
+        del per
+    st = pool.stats()
+    assert st["adapters_loaded"] == cfg.max_adapters
+    assert st["physical_bytes"] < 0.90 * st["padding_bytes"]           # ~8 of the 10 reserved slots per adapter are live
+    assert st["physical_bytes"] - st["live_expert_bytes"] < 0.02 * st["live_expert_bytes"]   # page rounding only
+    aid = wl.gen_adapter_ids(cfg)
+    assert aid.min() >= 0                                              # every token belongs to an adapter
+    sample = np.sort(np.random.default_rng(3).choice(cfg.n_tokens, size=48, replace=False))
+    for l in check:
+        res = run_layer(cfg, layer=l, sample=sample, pool=pool, bank=bank, tuned=tuned, bases=bases)
+        print("c3 layer", l, {k: v for k, v in res.items() if k in ("flips", "rel", "max_abs")})
+    # all layers back to back on one stream, each on its own input
+    xs = [to_dev(wl.gen_tokens(cfg, l)) for l in range(L)]
+    d_aid = to_dev(aid)
+    outs = [pool.moe_forward(l, xs[l], d_aid) for l in range(L)]
+    torch.cuda.synchronize()
+    assert pool.last_device_error() == 0
+    assert all(torch.isfinite(o.float()).all() for o in outs)
+    pool.destroy()

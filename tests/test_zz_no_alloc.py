@@ -11,7 +11,7 @@ import pytest
 from paper_2508_17624_b200 import binding, build
 from paper_2508_17624_b200 import workloads as wl
 
-from helpers import WEIGHT_TOL, to_dev
+from helpers import WEIGHT_RTOL, WEIGHT_TOL, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -45,7 +45,7 @@ def test_route_noalloc_matches_forward_twice_in_a_row(name):
         ids, w, slots, counts, status = _route(pool, cfg, x, aid, cfg.n_tokens)
         assert status == 0
         assert np.array_equal(ids, want["topk_ids"]), call
-        assert np.abs(w - want["topk_w"]).max() <= WEIGHT_TOL, call
+        assert (np.abs(w - want["topk_w"]) <= WEIGHT_TOL + WEIGHT_RTOL * want["topk_w"]).all(), call
         assert np.array_equal(slots, want["slot_ids"]), call
         assert np.array_equal(counts, want["counts"]), call
     # a bad adapter id is reported through the status word kept in the array, and cleared by the next call

@@ -25,16 +25,21 @@ sys.path.insert(0, ROOT)
 
 METRIC = "adapter-aware MoE layer tokens/s"
 UNIT = "tokens/s"
-WORKLOAD = "c1: DeepSeek-V2-Lite-shaped MoE layer, decode batch 256, 4 adapters x 8 experts"
+WORKLOADS = {
+    "c1": "c1: DeepSeek-V2-Lite-shaped MoE layer, decode batch 256, 4 adapters x 8 experts",
+    "c2": "c2: DeepSeek-V2-Lite-shaped MoE layer, prefill 8192 tokens (32 requests x 256), 20 adapters x 4-16 experts",
+}
+WORKLOAD = WORKLOADS["c1"]
 
 
 def load_peaks():
+    """-> (HBM GB/s, bf16 TFLOP/s burst, kind)"""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), "measured"
+    return 6650.0, 1590.0, "fallback"
 
 
 class ClockSampler(threading.Thread):
@@ -109,7 +114,8 @@ def run_cuda(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     build.build()
-    cfg = wl.CONFIGS["c1"]
+    cfg = wl.CONFIGS[args.workload]
+    workload = WORKLOADS[args.workload]
     B, H, k = cfg.n_tokens, cfg.hidden, cfg.top_k
     pool = binding.Pool.from_config(cfg, device=local)
     binding.load_model(pool, cfg)
@@ -203,14 +209,28 @@ def run_cuda(args):
 
     result = None
     if rank == 0:
-        peak, peak_kind = load_peaks()
+        peak, peak_tf, peak_kind = load_peaks()
         g1_ms = kern_ms["gemm1"] / max(n_prof, 1)
         achieved = bytes_gemm1 / (g1_ms * 1e-3) / 1e9
+        flops_gemm1 = 2.0 * rows_act * 2 * cfg.inter * H
+        flops_gemm2 = 2.0 * rows_act * cfg.inter * H
+        tensor_bound = flops_gemm1 / (peak_tf * 1e12) > bytes_gemm1 / (peak * 1e9)
+        if tensor_bound:
+            roof = {"bound": "tensor", "kernel": "grouped_gemm_kernel<GLU> (GEMM-1 + SwiGLU)",
+                    "achieved": flops_gemm1 / (g1_ms * 1e-3) / 1e12, "peak": peak_tf, "unit": "TFLOP/s",
+                    "frac": flops_gemm1 / (g1_ms * 1e-3) / 1e12 / peak_tf, "of": peak_kind + " (bf16 burst)",
+                    "traffic": None, "algorithmic_flops": flops_gemm1, "avg_launch_ms": g1_ms,
+                    "hbm_gbs": achieved}
+        else:
+            roof = {"bound": "hbm", "kernel": "grouped_gemm_kernel<GLU> (GEMM-1 + SwiGLU)",
+                    "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "of": peak_kind, "traffic": None, "algorithmic_bytes": bytes_gemm1,
+                    "avg_launch_ms": g1_ms}
         result = {
             "metric": METRIC, "value": world * B * args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "tokens_per_step_per_gpu": B, "hidden": H, "inter": cfg.inter,
+            "config": {"workload": workload, "tokens_per_step_per_gpu": B, "hidden": H, "inter": cfg.inter,
                        "experts": cfg.num_experts, "shared": cfg.num_shared, "top_k": k,
                        "adapters": cfg.max_adapters, "e_max": cfg.e_max, "live_slots": live,
                        "token_tile": None, "parallelism": f"replicas x{world}",
@@ -220,13 +240,11 @@ def run_cuda(args):
                     "h2d_bytes_per_step": B * H * 2 + B * 4, "d2h_bytes_per_step": B * H * 2},
             "gpu_launches": 5 * args.steps,
             "clocks": dict(sampler.summary(), extended=extended),
-            "roofline": {"bound": "hbm", "kernel": "grouped_gemm_kernel<GLU> (GEMM-1 + SwiGLU)",
-                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "of": peak_kind, "traffic": None, "algorithmic_bytes": bytes_gemm1,
-                         "avg_launch_ms": g1_ms},
+            "roofline": roof,
             "kernels_ms_per_step": {kname: v / max(n_prof, 1) for kname, v in kern_ms.items()},
             "gemm2": {"achieved": bytes_gemm2 / (kern_ms["gemm2"] / max(n_prof, 1) * 1e-3) / 1e9, "unit": "GB/s",
-                      "algorithmic_bytes": bytes_gemm2},
+                      "algorithmic_bytes": bytes_gemm2,
+                      "tflops": flops_gemm2 / (kern_ms["gemm2"] / max(n_prof, 1) * 1e-3) / 1e12},
             "layer_weight_stream": {"achieved": bytes_layer / (ms_total / args.steps * 1e-3) / 1e9, "unit": "GB/s",
                                     "frac": bytes_layer / (ms_total / args.steps * 1e-3) / 1e9 / peak},
             "ms_per_step_without_kernel_events": ms_plain / max(side_steps, 1),
@@ -239,6 +257,80 @@ def run_cuda(args):
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(result))
+
+
+def run_reroute(args):
+    """--workload c4: the batched rerouting operator alone (ids in, slot ids + per-slot counts out).
+
+    One JSON line per coverage (10 / 25 / 50 % of the experts re-tuned) at 65536 tokens, plus a size sweep
+    up to 2^24 tokens.  Cold L2: consecutive launches work on different buffer sets whose total exceeds the
+    L2 (256 MB).  GB/s = algorithmic bytes (ids in + slots out + adapter ids in + map) / mean launch time.
+    """
+    import torch
+    from paper_2508_17624_b200 import binding, build, workloads as wl
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    build.build()
+    cfg = wl.CONFIGS["c4"]
+    M, k, N, P = cfg.num_experts, cfg.top_k, cfg.max_adapters, cfg.num_slots
+    pool = binding.Pool(hidden=64, inter=64, num_experts=M, num_shared=0, top_k=k, max_adapters=N, e_max=cfg.e_max,
+                        max_tokens=8)
+    z = np.zeros((M, 64, 64), np.uint16)
+    pool.load_base(0, np.zeros((M, 64), np.uint16), z, z, z)
+    peak, _, peak_kind = load_peaks()
+    lines = []
+
+    def measure(B, iters):
+        pair_bytes = 2 * B * k * 4 + B * 4 + N * M * 4
+        n_sets = max(2, int((256 << 20) // pair_bytes) + 1)
+        g = torch.Generator(device="cuda").manual_seed(4)
+        sets = []
+        for _ in range(min(n_sets, 96)):
+            logits = torch.randn((B, M), device="cuda", generator=g)
+            ids = torch.topk(logits, k, dim=1).indices.to(torch.int32).contiguous()
+            aid = torch.randint(-1, N, (B,), device="cuda", generator=g, dtype=torch.int32)
+            sets.append((ids, aid, torch.empty_like(ids), torch.empty(P, dtype=torch.int32, device="cuda")))
+            del logits
+        for i in range(3):
+            pool.reroute(0, *sets[i % len(sets)][:2], slot_ids=sets[i % len(sets)][2], counts=sets[i % len(sets)][3])
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(iters):
+            s_ = sets[i % len(sets)]
+            pool.reroute(0, s_[0], s_[1], slot_ids=s_[2], counts=s_[3])
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / iters
+        return pair_bytes, ms, len(sets)
+
+    for e in ((32,) if args.tokens else (6, 16, 32)):
+        tuned = wl.tuned_sets(cfg, np.full((N, 1), e))
+        za = np.zeros((e, 64, 64), np.uint16)
+        for i in range(N):
+            pool.load_adapter(i, np.array([e], np.int32), tuned[i][0], za, za, za)
+        nbytes, ms, n_sets = measure(args.tokens or cfg.n_tokens, args.steps)
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        lines.append({"metric": "batched reroute GB/s", "value": gbs, "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
+                      "ms_per_launch": ms, "tokens": args.tokens or cfg.n_tokens,
+                      "tokens_per_s": (args.tokens or cfg.n_tokens) / (ms * 1e-3),
+                      "dtype": "int32", "data": "synthetic",
+                      "config": {"workload": f"c4: reroute only, {args.tokens or cfg.n_tokens} tokens, 20 adapters x {e} of 64 experts",
+                                 "l2": f"cold: {n_sets} rotating buffer sets", "includes": "zeroing of counts + kernel"},
+                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                                   "of": peak_kind, "algorithmic_bytes": nbytes, "traffic": None}})
+        if e != 32:
+            for i in range(N):
+                pool.unload_adapter(i)
+    sweep = []
+    for lg in (() if args.tokens else (16, 18, 20, 22, 24)):
+        nbytes, ms, n_sets = measure(1 << lg, max(20, args.steps >> max(0, lg - 18)))
+        sweep.append({"tokens": 1 << lg, "ms_per_launch": ms, "GB/s": nbytes / (ms * 1e-3) / 1e9,
+                      "frac": nbytes / (ms * 1e-3) / 1e9 / peak})
+    lines.append({"metric": "batched reroute GB/s, size sweep (50 % coverage)", "sweep": sweep, "peak": peak, "of": peak_kind})
+    assert pool.last_device_error() == 0
+    pool.destroy()
+    for ln in lines:
+        print(json.dumps(ln))
 
 
 def build_oracle_layer(cfg):
@@ -317,11 +409,16 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="c1", choices=sorted(WORKLOADS) + ["c4"],
+                    help="c1 (decode, the benchmark's workload), c2 (prefill) or c4 (reroute operator only)")
+    ap.add_argument("--tokens", type=int, default=0, help="c4 only: one run at this many tokens (50 %% coverage)")
     ap.add_argument("--minimal", action="store_true",
                     help="warm-up and timed steps only (for profiler captures): no CPU baseline, no side measurements")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "c4":
+        run_reroute(args)
     else:
         run_cuda(args)
 

@@ -571,7 +571,7 @@ extern "C" ew_status_t ew_reroute(ew_pool_t *p, int32_t layer, const int32_t *to
     if (dev != p->cfg.device) CU_TRY(cudaSetDevice(p->cfg.device));
     if (counts) CU_TRY(cudaMemsetAsync(counts, 0, (size_t)p->P * 4, st));
     if (B == 0) return EW_OK;
-    if (!topk_ids || !aid || !slot_ids) return EW_ERR_INVALID_ARG;
+    if (!topk_ids || !aid || !slot_ids || ((uintptr_t)topk_ids & 3) || ((uintptr_t)slot_ids & 3)) return EW_ERR_INVALID_ARG;
     LAUNCH_TRY(launch_reroute(p, layer, topk_ids, aid, B, slot_ids, counts, st));
     return note_forward(p, st);
 }

@@ -10,59 +10,109 @@
 namespace ew {
 namespace {
 
-// slot = aid < 0 ? id : Pi[aid][id]; bad adapter ids behave as -1 and raise bit 0 of the error word
-__device__ __forceinline__ int checked_aid(int a, int N, const int32_t *loaded, int *err) {
-    if (a < -1 || a >= N || (a >= 0 && !loaded[a])) {
-        atomicOr(err, 1);
-        return -1;
-    }
-    return a;
-}
+// ------------------------------------------------------------------------------------------------
+// Batched rerouting alone: slot = aid < 0 ? id : Pi[aid][id] (bad adapter ids behave as -1 and raise
+// bit 0 of the error word).  A CTA moves tiles of 256 tokens (256*k ids, so every tile starts 16-byte
+// aligned) through a three-stage shared-memory ring filled by 16-byte asynchronous copies (two tiles
+// ahead are in flight); a thread rewrites 16-byte vectors of four ids in place (the token of an id is a
+// multiply-shift on its index inside the tile, exact for i < 8192 and k <= 32; adapter ids are staged
+// per tile), and the tile leaves with coalesced 16-byte streaming stores.  Expert map and loaded flags
+// sit in shared memory; the per-CTA shared-memory histogram is flushed with one atomic per non-empty slot.
+// ------------------------------------------------------------------------------------------------
+constexpr int kRerouteTok = 256;
+constexpr int kRerouteStages = 3;
 
-// ------------------------------------------------------------------------------------------------
-// Batched rerouting alone: four pairs per thread (16-byte loads and stores), expert map in shared
-// memory, per-CTA shared-memory histogram flushed with one atomic per non-empty slot.
-// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 __global__ void __launch_bounds__(256) reroute_kernel(const int32_t *__restrict__ ids, const int32_t *__restrict__ aid,
                                                       const int32_t *__restrict__ pi, const int32_t *__restrict__ loaded,
-                                                      long long n_pairs, int k, int M, int N, int P,
+                                                      int n_tokens, int k, int M, int N, int P, int vec_ok,
                                                       int32_t *__restrict__ slots, int32_t *__restrict__ counts, int *err) {
     extern __shared__ int32_t smem_i[];
-    int32_t *pi_s = smem_i, *hist = smem_i + N * M;
+    const int tile_ints_max = kRerouteTok * k;         // multiple of 4 ints: every stage stays 16-byte aligned
+    const int stage_ints = tile_ints_max;
+    int32_t *tiles = smem_i;                           // [kRerouteStages][256 * k]
+    int32_t *pi_s = tiles + kRerouteStages * stage_ints, *hist = pi_s + N * M, *loaded_s = hist + P, *aid_s = loaded_s + N;
     for (int i = threadIdx.x; i < N * M; i += blockDim.x) pi_s[i] = pi[i];
+    for (int i = threadIdx.x; i < N; i += blockDim.x) loaded_s[i] = loaded[i];
     if (counts)
         for (int i = threadIdx.x; i < P; i += blockDim.x) hist[i] = 0;
-    __syncthreads();
-    const long long n_vec = (n_pairs + 3) >> 2;
-    for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < n_vec; v += (long long)gridDim.x * blockDim.x) {
-        const long long q0 = v << 2;
-        int id[4];
-        const bool full = q0 + 3 < n_pairs;
-        if (full) {
-            const int4 r = *reinterpret_cast<const int4 *>(ids + q0);
-            id[0] = r.x; id[1] = r.y; id[2] = r.z; id[3] = r.w;
-        } else {
-            for (int j = 0; j < 4; ++j) id[j] = q0 + j < n_pairs ? ids[q0 + j] : 0;
+    const unsigned div_magic = ((1u << 20) + k - 1) / k;
+    const int n_tiles = (n_tokens + kRerouteTok - 1) / kRerouteTok;
+    int flags = 0;
+    auto tile_ints = [&](int tl) { return min(kRerouteTok, n_tokens - tl * kRerouteTok) * k; };
+    // asynchronous copy of tile tl into stage st (16-byte pieces; unaligned buffers fall back to plain loads)
+    auto fetch = [&](int tl, int st) {
+        if (tl < n_tiles) {
+            const int32_t *src = ids + (size_t)tl * tile_ints_max;
+            int32_t *dst = tiles + st * stage_ints;
+            const int n_int = tile_ints(tl), n_vec = vec_ok ? n_int >> 2 : 0;
+            for (int i = threadIdx.x; i < n_vec; i += 256) cp_async16(dst + 4 * i, src + 4 * i);
+            for (int i = (n_vec << 2) + threadIdx.x; i < n_int; i += 256) dst[i] = src[i];
         }
-        int s[4];
+        cp_async_commit();                             // one group per call, empty or not, keeps the wait count uniform
+    };
+    auto checked = [&](int a) -> int {                 // adapter ids outside [-1,N) or of unloaded adapters act as -1
+        if (a < -1 || a >= N || (a >= 0 && !loaded_s[a])) { flags |= 1; a = -1; }
+        return a;
+    };
+    auto map_one = [&](int e, int a) -> int {
+        if ((unsigned)e >= (unsigned)M) { flags |= 4; return e; }
+        const int sl = a < 0 ? e : pi_s[a * M + e];
+        if (counts) atomicAdd(hist + sl, 1);
+        return sl;
+    };
+    for (int s0 = 0; s0 < kRerouteStages - 1; ++s0) fetch(blockIdx.x + s0 * gridDim.x, s0);
+    int st = 0;
+    for (int tl = blockIdx.x; tl < n_tiles; tl += gridDim.x) {
+        const size_t base = (size_t)tl * tile_ints_max;
+        const int n_int = tile_ints(tl), n_vec = n_int >> 2;     // n_int is a multiple of k; tiles but the last of 256*k
+        int32_t *tile = tiles + st * stage_ints;
+        {
+            const int t = tl * kRerouteTok + threadIdx.x;
+            const int a = checked(t < n_tokens ? __ldg(aid + t) : -1);
+            __syncthreads();                           // previous tile fully processed and stored; tables staged
+            aid_s[threadIdx.x] = a;
+        }
+        // the stage freed by the previous tile receives the tile kRerouteStages-1 ahead
+        fetch(tl + (kRerouteStages - 1) * gridDim.x, (st + kRerouteStages - 1) % kRerouteStages);
+        cp_async_wait<kRerouteStages - 1>();           // this tile's group has landed
+        __syncthreads();
+        for (int v = threadIdx.x; v < n_vec; v += 256) {
+            int4 r = reinterpret_cast<int4 *>(tile)[v];
+            const int i0 = v << 2;
+            int tok = (int)(((unsigned)i0 * div_magic) >> 20);
+            int rem = i0 - tok * k;                    // position of the vector's first id inside its token's row
+            int a = aid_s[tok];
+            int *e = reinterpret_cast<int *>(&r);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const long long q = q0 + j;
-            if (q < n_pairs) {
-                const int a = checked_aid(__ldg(aid + q / k), N, loaded, err);
-                int e = id[j];
-                if (e < 0 || e >= M) { atomicOr(err, 4); s[j] = e; }
-                else {
-                    s[j] = a < 0 ? e : pi_s[a * M + e];
-                    if (counts) atomicAdd(hist + s[j], 1);
-                }
-            } else s[j] = 0;
+            for (int j = 0; j < 4; ++j) {
+                if (rem == k) { rem = 0; a = aid_s[++tok]; }
+                e[j] = map_one(e[j], a);
+                ++rem;
+            }
+            reinterpret_cast<int4 *>(tile)[v] = r;
         }
-        if (full) *reinterpret_cast<int4 *>(slots + q0) = make_int4(s[0], s[1], s[2], s[3]);
-        else
-            for (int j = 0; j < 4; ++j)
-                if (q0 + j < n_pairs) slots[q0 + j] = s[j];
+        for (int i = (n_vec << 2) + threadIdx.x; i < n_int; i += 256)       // last tile when its length is not a multiple of 4
+            tile[i] = map_one(tile[i], aid_s[((unsigned)i * div_magic) >> 20]);
+        __syncthreads();
+        if (vec_ok) {
+            for (int i = threadIdx.x; i < n_vec; i += 256)
+                __stcs(reinterpret_cast<int4 *>(slots + base) + i, reinterpret_cast<const int4 *>(tile)[i]);
+            for (int i = (n_vec << 2) + threadIdx.x; i < n_int; i += 256) slots[base + i] = tile[i];
+        } else {
+            for (int i = threadIdx.x; i < n_int; i += 256) slots[base + i] = tile[i];
+        }
+        st = (st + 1) % kRerouteStages;
     }
+    cp_async_wait<0>();
+    if (flags) atomicOr(err, flags);
     if (counts) {
         __syncthreads();
         for (int i = threadIdx.x; i < P; i += blockDim.x)
@@ -229,14 +279,21 @@ int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st) {
 int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid, int B, int32_t *slots,
                    int32_t *counts, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
-    const long long pairs = (long long)B * c.top_k;
-    const long long vecs = (pairs + 3) / 4;
-    long long blocks = (vecs + 255) / 256;
-    const long long cap = (long long)p->sm_count * 8;
+    long long blocks = ((long long)B + kRerouteTok - 1) / kRerouteTok;
+    const size_t smem = ((size_t)kRerouteStages * kRerouteTok * c.top_k + (size_t)c.max_adapters * c.num_experts + p->P + c.max_adapters + kRerouteTok) * 4 + 16;
+    // 16-byte accesses need aligned buffers; every tile starts at a multiple of 256*k ints
+    const int vec_ok = (((uintptr_t)ids | (uintptr_t)slots) & 15) == 0;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(reroute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+    }
+    // exactly one wave: every CTA is resident and walks its share of the tiles
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, reroute_kernel, 256, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
+    const long long cap = (long long)p->sm_count * per_sm;
     if (blocks > cap) blocks = cap;
-    const size_t smem = ((size_t)c.max_adapters * c.num_experts + p->P) * 4 + 16;
-    reroute_kernel<<<(int)blocks, 256, smem, st>>>(ids, aid, p->layers[layer].pi_dev, p->ws.loaded, pairs, c.top_k,
-                                                   c.num_experts, c.max_adapters, p->P, slots, counts, p->ws.err);
+    reroute_kernel<<<(int)blocks, 256, smem, st>>>(ids, aid, p->layers[layer].pi_dev, p->ws.loaded, B, c.top_k,
+                                                   c.num_experts, c.max_adapters, p->P, vec_ok, slots, counts, p->ws.err);
     return (int)cudaGetLastError();
 }
 

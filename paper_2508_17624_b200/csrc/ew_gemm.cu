@@ -65,7 +65,6 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_items = *n_items_ptr;
     const int num_kb = (K + kBlockK - 1) / kBlockK;
 
     if (threadIdx.x == 0) {
@@ -89,10 +88,13 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
+    pdl_wait();                                         // the item list and the activations come from the previous kernels
+    const int n_items = *n_items_ptr;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -228,9 +230,8 @@ int launch_one(ew_pool *p, const CUtensorMap &mw, const CUtensorMap &ma, const C
                const CUtensorMap &mxb, const GemmItem *items, const int32_t *n_items, int K, int out_rows, void *out,
                cudaStream_t st) {
     using C = Cfg<NT, GLU>;
-    grouped_gemm_kernel<NT, GLU><<<p->sm_count, kThreads, C::kSmemBytes, st>>>(mw, ma, mx, mab, mxb, items, n_items, K,
-                                                                              out_rows, out, p->ws.err);
-    return (int)cudaGetLastError();
+    return launch_pdl(grouped_gemm_kernel<NT, GLU>, dim3(p->sm_count), dim3(kThreads), C::kSmemBytes, st, mw, ma, mx, mab,
+                      mxb, items, n_items, K, out_rows, out, p->ws.err);
 }
 
 template <int NT, bool GLU>

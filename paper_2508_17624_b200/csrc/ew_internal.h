@@ -71,6 +71,7 @@ struct ew_pool {
     cudaStream_t copy_stream = nullptr;
     std::vector<std::pair<cudaStream_t, cudaEvent_t>> fwd_events;   // last forward per caller stream
     int sm_count = 148;
+    bool counts_clean = true;      // the slot counters are zero (the combine kernel of a finished forward re-zeroes them)
     bool profiling = false;
     std::vector<cudaEvent_t> prof_events;   // 6 per recorded forward
     size_t prof_used = 0;                   // events in use
@@ -85,6 +86,23 @@ struct ew_pool {
 namespace ew {
 
 void set_last_error(const std::string &s);
+
+// Launch with programmatic stream serialization (the kernel calls pdl_wait() before it reads its
+// predecessor's output).
+template <class... KArgs, class... Args>
+int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return (int)cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 // bf16 2-D/3-D tiled descriptor with 128-byte swizzle; dims/box innermost first.
 int make_tensor_map(ew_pool *p, CUtensorMap *out, const void *base, int rank, const uint64_t *dims,

@@ -534,7 +534,8 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     }
 #define PROF_MARK(i) do { if (pe) CU_TRY(cudaEventRecord(pe[i], st)); } while (0)
     PROF_MARK(0);
-    CU_TRY(cudaMemsetAsync(p->ws.counts, 0, (size_t)p->P * 4, st));
+    if (!p->counts_clean) CU_TRY(cudaMemsetAsync(p->ws.counts, 0, (size_t)p->P * 4, st));   // an earlier forward failed midway
+    p->counts_clean = false;
     LAUNCH_TRY(launch_route(p, layer, x, aid, B, st));
     PROF_MARK(1);
     LAUNCH_TRY(launch_permute(p, x, B, st));
@@ -550,6 +551,7 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     LAUNCH_TRY(launch_gemm2(p, layer, B, st));
     PROF_MARK(4);
     LAUNCH_TRY(launch_combine(p, B, out, st));
+    p->counts_clean = true;                             // the combine kernel zeroes the counters when it is done with them
     PROF_MARK(5);
 #undef PROF_MARK
     return note_forward(p, st);

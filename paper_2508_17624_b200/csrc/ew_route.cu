@@ -6,6 +6,7 @@
 #include <cuda_bf16.h>
 
 #include "ew_internal.h"
+#include "ew_tc.cuh"
 
 namespace ew {
 namespace {
@@ -160,6 +161,8 @@ __global__ void __launch_bounds__(256) permute_kernel(const uint4 *__restrict__ 
     int32_t *off = sm;                 // [P + 1]
     int32_t *blk = sm + P + 1;         // [P + S + 1] token blocks per group, scanned
     __shared__ int32_t warp_sums[8];
+    tc::pdl_launch_dependents();
+    tc::pdl_wait();                                     // counts, slot ids and ranks come from the router kernel
     block_exclusive_scan(counts, off, P, warp_sums);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (blockIdx.x + 1 < gridDim.x) {
@@ -218,10 +221,14 @@ __global__ void __launch_bounds__(256) permute_kernel(const uint4 *__restrict__ 
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) combine_kernel(const float4 *__restrict__ y, const int32_t *__restrict__ inv,
                                                       const float *__restrict__ w, int B, int k, int H, int S,
-                                                      uint2 *__restrict__ out) {
+                                                      uint2 *__restrict__ out, int32_t *__restrict__ counts, int P) {
     __shared__ int32_t rows[32];
     __shared__ float wts[32];
     const int t = blockIdx.x;
+    tc::pdl_launch_dependents();
+    tc::pdl_wait();                                     // expert outputs come from GEMM-2
+    if (t == 0)                                         // the slot counters are spent: leave them zero for the next forward
+        for (int i = threadIdx.x; i < P; i += blockDim.x) counts[i] = 0;
     if (threadIdx.x < k) {
         rows[threadIdx.x] = S * B + inv[(size_t)t * k + threadIdx.x];
         wts[threadIdx.x] = w[(size_t)t * k + threadIdx.x];
@@ -263,17 +270,15 @@ int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st) {
     const long long pairs = (long long)B * c.top_k;
     const int grid = (int)((pairs + 7) / 8) + 1;
     const size_t smem = ((size_t)(p->P + 1) + 2 * (size_t)(p->P + c.num_shared) + 2) * 4;
-    permute_kernel<<<grid, 256, smem, st>>>((const uint4 *)x, p->ws.slot_ids, p->ws.rank, p->ws.counts, B, c.top_k,
-                                            c.hidden, p->P, c.num_shared, p->token_tile, R1, R2, p->ws.offsets,
-                                            p->ws.inv, (uint4 *)p->ws.xp, p->ws.items1, p->ws.items2, p->ws.n_items);
-    return (int)cudaGetLastError();
+    return launch_pdl(permute_kernel, dim3(grid), dim3(256), smem, st, (const uint4 *)x, p->ws.slot_ids, p->ws.rank,
+                      p->ws.counts, B, c.top_k, c.hidden, p->P, c.num_shared, p->token_tile, R1, R2, p->ws.offsets, p->ws.inv,
+                      (uint4 *)p->ws.xp, p->ws.items1, p->ws.items2, p->ws.n_items);
 }
 
 int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
-    combine_kernel<<<B, 256, 0, st>>>((const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B, c.top_k, c.hidden,
-                                      c.num_shared, (uint2 *)out);
-    return (int)cudaGetLastError();
+    return launch_pdl(combine_kernel, dim3(B), dim3(256), 0, st, (const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B, c.top_k,
+                      c.hidden, c.num_shared, (uint2 *)out, p->ws.counts, p->P);
 }
 
 int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid, int B, int32_t *slots,

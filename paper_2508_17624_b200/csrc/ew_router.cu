@@ -118,10 +118,12 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
     }
     if (A.pi_in_smem)
         for (int i = threadIdx.x; i < A.N * M; i += kThreads) pi_s[i] = A.pi[i];
+    pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
+    pdl_wait();                                         // x and the slot counters belong to earlier work in the stream
 
     if (warp == 0) {
         if (lane == 0) {                                             // TMA producer
@@ -319,9 +321,8 @@ int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B
         attr_set[reg] = smem;
     }
     const int grid = (B + tok_tile - 1) / tok_tile;
-    if (reg) router_kernel<true><<<grid, kThreads, smem, st>>>(map_x, L.map_router, A);
-    else router_kernel<false><<<grid, kThreads, smem, st>>>(map_x, L.map_router, A);
-    return (int)cudaGetLastError();
+    if (reg) return launch_pdl(router_kernel<true>, dim3(grid), dim3(kThreads), smem, st, map_x, L.map_router, A);
+    return launch_pdl(router_kernel<false>, dim3(grid), dim3(kThreads), smem, st, map_x, L.map_router, A);
 }
 
 }  // namespace ew

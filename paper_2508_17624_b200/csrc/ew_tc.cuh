@@ -12,6 +12,13 @@ constexpr int kChunkBytes = kChunkRows * kBlockK * 2;  // 4 KiB
 constexpr long long kWaitLimitCycles = 2000000000ll;   // about one second
 
 // ---------------------------------------------------------------------------------------------- PTX
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start while
+// its predecessor in the stream is still running; it must not touch the predecessor's results before
+// pdl_wait() returns (which also guarantees that everything earlier in the stream has completed, because
+// every kernel of the forward waits before it finishes).  Both are no-ops in an ordinary launch.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {

@@ -91,6 +91,21 @@ class ClockSampler(threading.Thread):
         return out
 
 
+def reduce_max_over_ranks(values, device="cpu"):
+    """Element-wise MAX of per-rank measurements over all ranks (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def whole_job_tokens_per_s(world: int, tokens_per_step_per_rank: int, steps: int, ms_slowest_rank: float) -> float:
+    """Replicas only: every rank pushes its own batch, the job's time is the slowest rank's."""
+    return world * tokens_per_step_per_rank * steps / (ms_slowest_rank * 1e-3)
+
+
 def physical_index(local_rank: int) -> int:
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -205,10 +220,7 @@ def run_cuda(args):
     err = pool.last_device_error()
     assert err == 0, f"device error word {err}"
 
-    times = torch.tensor([ms_total, ms_e2e, ms_plain], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e, ms_plain = (float(v) for v in times.cpu())
+    ms_total, ms_e2e, ms_plain = reduce_max_over_ranks([ms_total, ms_e2e, ms_plain], device="cuda")
 
     result = None
     if rank == 0:
@@ -230,7 +242,7 @@ def run_cuda(args):
                     "of": peak_kind, "traffic": None, "algorithmic_bytes": bytes_gemm1,
                     "avg_launch_ms": g1_ms}
         result = {
-            "metric": METRIC, "value": world * B * args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": whole_job_tokens_per_s(world, B, args.steps, ms_total), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": workload, "tokens_per_step_per_gpu": B, "hidden": H, "inter": cfg.inter,
@@ -239,7 +251,7 @@ def run_cuda(args):
                        "token_tile": None, "parallelism": f"replicas x{world}",
                        "l2": "no flush: each step streams %.2f GB of live expert weights, far above the 126 MB L2"
                              % (bytes_layer / 1e9)},
-            "e2e": {"value": world * B * max(side_steps, 1) / (ms_e2e * 1e-3), "unit": UNIT,
+            "e2e": {"value": whole_job_tokens_per_s(world, B, max(side_steps, 1), ms_e2e), "unit": UNIT,
                     "h2d_bytes_per_step": B * H * 2 + B * 4, "d2h_bytes_per_step": B * H * 2},
             "gpu_launches": 5 * args.steps,
             "clocks": dict(sampler.summary(), extended=extended),

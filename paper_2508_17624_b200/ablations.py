@@ -1,0 +1,165 @@
+"""In-house analogues of the paper's micro-benchmarks (Section 5.3 / 5.4), on synthetic layers.
+
+  python -m paper_2508_17624_b200.ablations [--steps K]
+
+Prints one JSON object:
+  adapters_vs_base   layer time with 4 adapters in the batch vs the same layer serving base-model tokens only
+                     (the paper's "overhead vs Base-Only", Section 5.2, restated for one layer)
+  vmm_vs_padding     layer time and physical bytes, pages on demand vs the fully backed padding tensor
+                     (Section 5.3 "virtual weight tensor vs padding", Section 5.4 memory)
+  reroute            the batched rerouting step three ways: fused into the router kernel (its share of the
+                     layer), the stand-alone operator, and the unfused formulation from stock tensor ops
+                     (broadcast the adapter ids, compute offsets into the map, gather: the paper's
+                     "SingleOp" variant, Section 5.3)
+All inputs are seeded and synthetic (workloads.py); timings are CUDA events over K back-to-back calls.
+"""
+import argparse
+import json
+
+import numpy as np
+
+
+def _time(fn, steps, torch):
+    for _ in range(5):
+        fn()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def table1_shaped_counts(max_e: int, avg_e: float, layers: int, seed: int) -> np.ndarray:
+    """Per-layer expert counts with the given maximum and (rounded) average: the paper prints only these two
+    summary numbers per adapter (Table 1), not the per-layer counts."""
+    rng = np.random.default_rng(seed)
+    target = int(round(avg_e * layers))
+    e = rng.integers(1, max_e + 1, size=layers)
+    e[rng.integers(layers)] = max_e
+    while e.sum() != target:
+        i = rng.integers(layers)
+        if e.sum() > target and e[i] > 1 and (e[i] < max_e or (e == max_e).sum() > 1):
+            e[i] -= 1
+        elif e.sum() < target and e[i] < max_e:
+            e[i] += 1
+    return e.astype(np.int32)
+
+
+def memory_table1_shapes():
+    """Adapter memory, pages on demand vs padding, for Table-1-shaped adapters of the DeepSeek-V2-Lite shape
+    (26 layers, 64 experts, 16.5 MiB per expert), on the accounting-only backend (no GPU needed).  The paper's
+    Section 5.4 loads gate-math, then gate-intent, then token-math and reports 40.4 %, 28.9 % and 37.3 % less."""
+    from . import binding, workloads as wl
+    shapes = [("gate-math", 12, 7.04), ("gate-intent", 12, 9.50), ("token-math", 9, 6.12)]
+    L, M, e_max = 26, 64, 12
+    out = []
+    pools = {}
+    for mode in (0, 1):
+        pools[mode] = binding.Pool(device=-1, num_layers=L, hidden=2048, inter=1408, num_experts=M, num_shared=2,
+                                   top_k=6, max_adapters=3, e_max=e_max, max_tokens=16, pool_mode=mode)
+        for l in range(L):
+            pools[mode].load_base(l, None, None, None, None, None, None, None)
+    base = {m: pools[m].stats()["physical_bytes"] for m in pools}
+    base_pad_reserved = 3 * e_max * L * 3 * 1408 * 2048 * 2
+    for i, (name, mx, avg) in enumerate(shapes):
+        counts = table1_shaped_counts(mx, avg, L, seed=100 + i)
+        ids = np.concatenate([np.arange(c, dtype=np.int32) for c in counts])
+        for m in pools:
+            pools[m].load_adapter(i, counts, ids, None, None, None)
+        vmm = pools[0].stats()["physical_bytes"] - base[0]
+        # the padding tensor reserves E_max slots for every adapter that is loaded
+        pad = (i + 1) * e_max * L * 3 * 1408 * 2048 * 2
+        out.append({"adapters": i + 1, "added": name, "adapter_bytes_vmm": vmm, "adapter_bytes_padding": pad,
+                    "saving": 1.0 - vmm / pad})
+    assert pools[1].stats()["physical_bytes"] - pools[0].stats()["physical_bytes"] > 0
+    for m in pools:
+        pools[m].destroy()
+    return out
+
+
+def main():
+    import torch
+    from . import binding, build, workloads as wl
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--steps", type=int, default=500)
+    args = ap.parse_args()
+    assert torch.cuda.is_available(), "needs a CUDA device"
+    build.build()
+    cfg = wl.CONFIGS["c1"]
+    bank = wl.NoiseBank(cfg.seed)
+    x = torch.from_numpy(wl.gen_tokens(cfg).view(np.int16)).cuda().view(torch.bfloat16)
+    aid = torch.from_numpy(wl.gen_adapter_ids(cfg)).cuda()
+    base_aid = torch.full_like(aid, -1)
+    out = torch.empty_like(x)
+    res = {}
+
+    # ---- pages on demand
+    pool = binding.Pool.from_config(cfg)
+    binding.load_model(pool, cfg, bank, adapters=[])
+    t_base_only = _time(lambda: pool.moe_forward(0, x, base_aid, out), args.steps, torch)
+    st_base = pool.stats()
+    binding.load_model(pool, cfg, bank, layers=[])           # now the four adapters
+    t_mixed = _time(lambda: pool.moe_forward(0, x, aid, out), args.steps, torch)
+    t_base_tokens = _time(lambda: pool.moe_forward(0, x, base_aid, out), args.steps, torch)
+    pool.profile_enable(True)
+    pool.profile_read()
+    for _ in range(200):
+        pool.moe_forward(0, x, aid, out)
+    kern, n = pool.profile_read()
+    pool.profile_enable(False)
+    st_vmm = pool.stats()
+    d = pool.moe_forward_debug(0, x, aid)
+    torch.cuda.synchronize()
+    live = int((d["counts"] > 0).sum())
+    res["adapters_vs_base"] = {
+        "ms_base_only_pool": t_base_only, "ms_adapters_loaded_base_tokens": t_base_tokens, "ms_mixed_batch": t_mixed,
+        "overhead_mixed_vs_base_only": t_mixed / t_base_only - 1.0,
+        "live_slots_mixed": live, "live_weight_bytes_ratio": (live + cfg.num_shared) / (cfg.num_experts + cfg.num_shared)}
+    res["reroute"] = {"router_kernel_ms": kern["route"] / n, "layer_ms_with_kernel_events": sum(kern.values()) / n,
+                      "router_share_of_layer": kern["route"] / sum(kern.values())}
+
+    # ---- stand-alone operator vs unfused tensor ops, at the decode batch and at 65536 tokens
+    pi_dev = torch.from_numpy(pool.get_expert_map(0)).cuda()
+    for B in (cfg.n_tokens, 65536):
+        g = torch.Generator(device="cuda").manual_seed(7)
+        ids = torch.topk(torch.randn((B, cfg.num_experts), device="cuda", generator=g), cfg.top_k, dim=1).indices.to(torch.int32)
+        a = torch.randint(-1, cfg.max_adapters, (B,), device="cuda", generator=g, dtype=torch.int32)
+        slots = torch.empty_like(ids)
+        counts = torch.empty(pool.num_slots, dtype=torch.int32, device="cuda")
+
+        def unfused():
+            a_b = a.to(torch.int64).unsqueeze(1).expand(-1, cfg.top_k)              # broadcast the adapter ids
+            off = a_b.clamp(min=0) * cfg.num_experts + ids.to(torch.int64)           # offsets into the map
+            red = pi_dev.reshape(-1).gather(0, off.reshape(-1)).reshape(B, cfg.top_k)   # gather
+            return torch.where(a_b < 0, ids, red)
+
+        want = unfused()
+        pool.reroute(0, ids, a, slot_ids=slots, counts=counts)
+        torch.cuda.synchronize()
+        assert torch.equal(want, slots), (B, int((want != slots).sum()), pool.last_device_error())
+        res["reroute"][f"B={B}"] = {
+            "operator_ms": _time(lambda: pool.reroute(0, ids, a, slot_ids=slots, counts=counts), args.steps, torch),
+            "operator_no_counts_ms": _time(lambda: pool.reroute(0, ids, a, slot_ids=slots, want_counts=False), args.steps, torch),
+            "unfused_tensor_ops_ms": _time(unfused, args.steps, torch)}
+    pool.destroy()
+
+    # ---- padding baseline: the whole [M + N*E_max + S] tensor is physically backed
+    pad = binding.Pool.from_config(cfg, pool_mode=1)
+    binding.load_model(pad, cfg, bank)
+    t_pad = _time(lambda: pad.moe_forward(0, x, aid, out), args.steps, torch)
+    st_pad = pad.stats()
+    pad.destroy()
+    res["vmm_vs_padding"] = {"ms_vmm": t_mixed, "ms_padding": t_pad, "latency_delta": t_mixed / t_pad - 1.0,
+                             "physical_bytes_vmm": st_vmm["physical_bytes"], "physical_bytes_padding": st_pad["physical_bytes"],
+                             "physical_bytes_base_only": st_base["physical_bytes"],
+                             "adapter_bytes_vmm": st_vmm["physical_bytes"] - st_base["physical_bytes"],
+                             "adapter_bytes_padding": st_pad["physical_bytes"] - st_base["physical_bytes"]}
+    res["memory_table1_shapes"] = memory_table1_shapes()
+    print(json.dumps(res))
+
+
+if __name__ == "__main__":
+    main()

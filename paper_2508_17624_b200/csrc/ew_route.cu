@@ -44,6 +44,7 @@ __global__ void __launch_bounds__(256) reroute_kernel(const int32_t *__restrict_
     for (int i = threadIdx.x; i < N; i += blockDim.x) loaded_s[i] = loaded[i];
     if (counts)
         for (int i = threadIdx.x; i < P; i += blockDim.x) hist[i] = 0;
+    __syncthreads();                                   // the staged flags are read right away (adapter-id check)
     const unsigned div_magic = ((1u << 20) + k - 1) / k;
     const int n_tiles = (n_tokens + kRerouteTok - 1) / kRerouteTok;
     int flags = 0;

@@ -23,6 +23,10 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+# DRAM bytes (read + write) per launch of the dominant kernel from the committed ncu captures
+# (profiles/c1_decode_grouped_gemm_full.md); reported beside the algorithmic bytes, not used in any ratio.
+NCU_TRAFFIC_BYTES = {"c1": 1.1480e9}
+
 METRIC = "adapter-aware MoE layer tokens/s"
 UNIT = "tokens/s"
 WORKLOADS = {
@@ -239,7 +243,7 @@ def run_cuda(args):
         else:
             roof = {"bound": "hbm", "kernel": "grouped_gemm_kernel<GLU> (GEMM-1 + SwiGLU)",
                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "of": peak_kind, "traffic": None, "algorithmic_bytes": bytes_gemm1,
+                    "of": peak_kind, "traffic": NCU_TRAFFIC_BYTES.get(args.workload), "algorithmic_bytes": bytes_gemm1,
                     "avg_launch_ms": g1_ms}
         result = {
             "metric": METRIC, "value": whole_job_tokens_per_s(world, B, args.steps, ms_total), "unit": UNIT, "n_gpus": world,

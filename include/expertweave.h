@@ -217,6 +217,13 @@ ew_status_t ew_pool_stats(ew_pool_t *pool, ew_stats_t *out);
  * an ew_status_t: EW_OK, EW_ERR_BAD_ADAPTER_ID_IN_BATCH, EW_ERR_TIMEOUT or EW_ERR_INVALID_ARG. */
 ew_status_t ew_last_device_error(ew_pool_t *pool, int32_t *code);
 
+/* Self-test of the bounded device-side waits (the tensor-core kernels wait on shared-memory barriers with a
+ * time limit instead of spinning forever).  Launches a one-CTA kernel that waits, with a limit of about a
+ * millisecond, on a barrier nothing arrives at; synchronises the stream; returns EW_OK if the wait expired and
+ * the kernel ran to its end.  Afterwards ew_last_device_error reports EW_ERR_TIMEOUT once.  No memory is
+ * touched outside the pool's error word. */
+ew_status_t ew_selftest_bounded_wait(ew_pool_t *pool, void *cuda_stream);
+
 /* Device address of slot `slot` of a layer's fused gate|up tensor (which = 0) or down tensor
  * (which = 1); slots M + N*E_max .. +S-1 are the shared experts.  For tests and tools: reading an
  * unmapped slot faults, so callers must only touch slots of loaded experts. */

@@ -22,7 +22,7 @@ STATUS_NAMES = ["EW_OK", "EW_ERR_INVALID_ARG", "EW_ERR_OOM", "EW_ERR_SLOT_IN_USE
                 "EW_ERR_NO_DEVICE"]
 EXPORTS = ["ew_pool_create", "ew_pool_destroy", "ew_load_base", "ew_load_adapter", "ew_unload_adapter",
            "ew_pool_trim", "ew_moe_forward", "ew_moe_forward_debug", "ew_moe_forward_host", "ew_profile_enable",
-           "ew_profile_read", "ew_reroute", "ew_route_noalloc", "ew_get_expert_map",
+           "ew_profile_read", "ew_reroute", "ew_route_noalloc", "ew_selftest_bounded_wait", "ew_get_expert_map",
            "ew_pool_stats", "ew_last_device_error", "ew_slot_address", "ew_status_str", "ew_last_error_string"]
 
 
@@ -207,6 +207,9 @@ class Pool:
         _check(lib().ew_route_noalloc(self._h, layer, _dp(x), _dp(adapter_ids), x.shape[0], _dp(topk_ids),
                                       _dp(topk_w), _dp(slot_ids), _dp(counts), _dp(device_status), _stream()),
                "ew_route_noalloc")
+
+    def selftest_bounded_wait(self):
+        _check(lib().ew_selftest_bounded_wait(self._h, _stream()), "ew_selftest_bounded_wait")
 
     def get_expert_map(self, layer) -> np.ndarray:
         out = np.empty((self.cfg.max_adapters, self.cfg.num_experts), np.int32)

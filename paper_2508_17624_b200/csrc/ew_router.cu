@@ -440,3 +440,48 @@ extern "C" ew_status_t ew_route_noalloc(ew_pool_t *p, int32_t layer, const void 
     }
     return EW_OK;
 }
+
+// ================================================================================================
+// Self-test of the bounded wait: a one-CTA kernel waits on an mbarrier that nothing ever arrives at,
+// with the same wait routine the tensor-core kernels use and a limit of about a millisecond.  The wait
+// must expire, raise bit 1 of the device error word and let the kernel return normally.
+// ================================================================================================
+namespace ew {
+namespace {
+__global__ void wait_selftest_kernel(int *err, int *reached_end) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    bool ok = true;
+    if (threadIdx.x == 0) ok = mbar_wait(smem_u32(&bar), 0, &abort_flag, err, 2000000ll);
+    __syncthreads();
+    if (threadIdx.x == 0) *reached_end = ok ? 2 : 1;     // 1: the wait gave up and the kernel went on to its end
+}
+}  // namespace
+}  // namespace ew
+
+extern "C" ew_status_t ew_selftest_bounded_wait(ew_pool_t *p, void *cuda_stream) {
+    using namespace ew;
+    if (!p) return EW_ERR_INVALID_ARG;
+    if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int *flag = p->ws.err + 1;                            // second word of the error segment
+    cudaError_t e = cudaMemsetAsync(flag, 0, 4, st);
+    if (e == cudaSuccess) {
+        wait_selftest_kernel<<<1, 32, 0, st>>>(p->ws.err, flag);
+        e = cudaGetLastError();
+    }
+    int reached = 0;
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&reached, flag, 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) {
+        set_last_error(std::string("ew_selftest_bounded_wait: ") + cudaGetErrorString(e));
+        return EW_ERR_CUDA;
+    }
+    return reached == 1 ? EW_OK : EW_ERR_INVALID_ARG;
+}

@@ -246,3 +246,21 @@ def test_c3_stacked_layers():
     assert pool.last_device_error() == 0
     assert all(torch.isfinite(o.float()).all() for o in outs)
     pool.destroy()
+
+
+def test_bounded_wait_expires_and_reports():
+    """A device-side wait that nothing satisfies gives up after its limit, raises the timeout bit and the
+    kernel returns; the context stays usable (a forward right after is still correct)."""
+    import torch
+    cfg = wl.CONFIGS["c0"]
+    pool = binding.Pool.from_config(cfg)
+    binding.load_model(pool, cfg)
+    x, aid = to_dev(wl.gen_tokens(cfg)), to_dev(wl.gen_adapter_ids(cfg))
+    before = pool.moe_forward(0, x, aid).clone()
+    pool.selftest_bounded_wait()
+    assert pool.last_device_error() == 7          # EW_ERR_TIMEOUT, reported once
+    assert pool.last_device_error() == 0
+    after = pool.moe_forward(0, x, aid)
+    torch.cuda.synchronize()
+    assert torch.equal(before, after)
+    pool.destroy()

@@ -120,9 +120,9 @@ ew_status_t ew_load_adapter(ew_pool_t *pool, int32_t adapter_id, const int32_t *
                             const int32_t *expert_ids, const void *w_gate, const void *w_up,
                             const void *w_down);
 
-/* Evict an adapter: its expert-map rows return to identity, the call then waits for every forward
- * issued before it, and pages whose reference count drops to zero are unmapped and returned to the
- * pool's free list for reuse (Section 4.2).  Errors: EW_ERR_INVALID_ARG, EW_ERR_NOT_LOADED. */
+/* Evict an adapter: the call waits for every forward issued before it (they complete as issued, with
+ * the adapter still in place), then its expert-map rows return to identity and pages whose reference
+ * count drops to zero are unmapped and returned to the pool's free list for reuse (Section 4.2).  Errors: EW_ERR_INVALID_ARG, EW_ERR_NOT_LOADED. */
 ew_status_t ew_unload_adapter(ew_pool_t *pool, int32_t adapter_id);
 
 /* Release the free list's pages back to the driver ("eventually reclaimed", Section 4.2). */

@@ -7,6 +7,8 @@ Prints one JSON object:
                      (the paper's "overhead vs Base-Only", Section 5.2, restated for one layer)
   vmm_vs_padding     layer time and physical bytes, pages on demand vs the fully backed padding tensor
                      (Section 5.3 "virtual weight tensor vs padding", Section 5.4 memory)
+  churn              evicting and re-loading one adapter (8 experts, 132 MiB) while forwards are in flight:
+                     host-side latency of ew_unload_adapter / ew_load_adapter and page reuse (Section 4.2)
   reroute            the batched rerouting step three ways: fused into the router kernel (its share of the
                      layer), the stand-alone operator, and the unfused formulation from stock tensor ops
                      (broadcast the adapter ids, compute offsets into the map, gather: the paper's
@@ -120,6 +122,32 @@ def main():
         "live_slots_mixed": live, "live_weight_bytes_ratio": (live + cfg.num_shared) / (cfg.num_experts + cfg.num_shared)}
     res["reroute"] = {"router_kernel_ms": kern["route"] / n, "layer_ms_with_kernel_events": sum(kern.values()) / n,
                       "router_share_of_layer": kern["route"] / sum(kern.values())}
+
+    # ---- churn: evict and re-load adapter 3 with 20 forwards queued each time
+    import time
+    tuned = wl.tuned_sets(cfg)
+    ew3 = wl.gen_adapter_layer(cfg, 3, 0, tuned[3][0], bank)
+    aid_wo3 = torch.where(aid == 3, torch.full_like(aid, -1), aid)
+    created0 = pool.stats()["pages_created_total"]
+    t_un, t_ld = [], []
+    for _ in range(5):
+        for _ in range(20):
+            pool.moe_forward(0, x, aid, out)
+        t0 = time.perf_counter()
+        pool.unload_adapter(3)                       # waits for the 20 forwards, flips the map rows, unmaps
+        t1 = time.perf_counter()
+        for _ in range(20):
+            pool.moe_forward(0, x, aid_wo3, out)
+        t2 = time.perf_counter()
+        pool.load_adapter(3, np.array([len(tuned[3][0])], np.int32), tuned[3][0], ew3.w_gate, ew3.w_up, ew3.w_down)
+        t3 = time.perf_counter()
+        t_un.append((t1 - t0) * 1e3)
+        t_ld.append((t3 - t2) * 1e3)
+    torch.cuda.synchronize()
+    res["churn"] = {"unload_ms_median": float(np.median(t_un)), "load_ms_median": float(np.median(t_ld)),
+                    "adapter_bytes": int(ew3.w_gate.nbytes * 3), "forwards_in_flight": 20,
+                    "pages_created_during_churn": pool.stats()["pages_created_total"] - created0,
+                    "device_error": pool.last_device_error()}
 
     # ---- stand-alone operator vs unfused tensor ops, at the decode batch and at 65536 tokens
     pi_dev = torch.from_numpy(pool.get_expert_map(0)).cuda()

@@ -395,7 +395,10 @@ extern "C" ew_status_t ew_unload_adapter(ew_pool_t *p, int32_t a) {
     bool gpu = c.device >= 0;
     int L = c.num_layers, M = c.num_experts;
     if (gpu) CU_TRY(cudaSetDevice(c.device));
-    // 1. rows back to identity, so that later forwards no longer reach the adapter's slots
+    // 1. forwards issued earlier may still read the adapter's slots and its map rows: let them finish as issued
+    if (gpu)
+        for (auto &e : p->fwd_events) CU_TRY(cudaEventSynchronize(e.second));
+    // 2. rows back to identity, so that later forwards no longer reach the adapter's slots
     for (int l = 0; l < L; ++l) {
         LayerState &Ls = p->layers[l];
         int32_t *row = Ls.pi_host.data() + (size_t)a * M;
@@ -406,8 +409,6 @@ extern "C" ew_status_t ew_unload_adapter(ew_pool_t *p, int32_t a) {
         int32_t zero = 0;
         CU_TRY(cudaMemcpyAsync(p->ws.loaded + a, &zero, 4, cudaMemcpyHostToDevice, p->copy_stream));
         CU_TRY(cudaStreamSynchronize(p->copy_stream));
-        // 2. forwards issued earlier may still read those slots: wait for them
-        for (auto &e : p->fwd_events) CU_TRY(cudaEventSynchronize(e.second));
     }
     // 3. drop the reference counts; pages reaching zero go back to the pool
     size_t delta = (size_t)M + (size_t)a * c.e_max, total = 0;

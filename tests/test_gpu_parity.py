@@ -264,3 +264,62 @@ def test_bounded_wait_expires_and_reports():
     torch.cuda.synchronize()
     assert torch.equal(before, after)
     pool.destroy()
+
+
+def test_adapter_churn_under_load():
+    """Adapters come and go while forwards are in flight (Section 4.2: pages are handed out at load time,
+    returned on eviction and reused).  Small experts (192 KiB) make neighbouring adapters share 2 MiB pages at
+    every alignment.  After every change the layer output is checked against the oracle for the adapters that
+    are loaded at that moment."""
+    import torch
+    cfg = wl.with_(wl.CONFIGS["c0"], max_adapters=6, e_max=5, n_tokens=96, seed=11)
+    bank = wl.NoiseBank(cfg.seed)
+    rng = np.random.default_rng(11)
+    pool = binding.Pool.from_config(cfg, prealloc_pages=2)
+    base = wl.gen_base_layer(cfg, 0, bank)
+    pool.load_base(0, base.router_w, base.routed.w_gate, base.routed.w_up, base.routed.w_down,
+                   base.shared.w_gate, base.shared.w_up, base.shared.w_down)
+    counts0 = rng.integers(1, cfg.e_max + 1, size=(cfg.max_adapters, 1))
+    tuned = wl.tuned_sets(cfg, counts0)
+    weights = {i: wl.gen_adapter_layer(cfg, i, 0, tuned[i][0], bank) for i in range(cfg.max_adapters)}
+    x_bits = wl.gen_tokens(cfg)
+    x = to_dev(x_bits)
+    loaded = set()
+    created = []
+    for step in range(24):
+        # keep the GPU busy with forwards of the current population, then change the population
+        pop = sorted(loaded)
+        aid_np = rng.choice([-1] + pop, size=cfg.n_tokens).astype(np.int32)
+        aid = to_dev(aid_np)
+        for _ in range(20):
+            pool.moe_forward(0, x, aid)
+        i = int(rng.integers(cfg.max_adapters))
+        if i in loaded:
+            pool.unload_adapter(i)                       # must wait for the forwards above, not fault
+            loaded.discard(i)
+        else:
+            ew = weights[i]
+            pool.load_adapter(i, np.array([len(tuned[i][0])], np.int32), tuned[i][0], ew.w_gate, ew.w_up, ew.w_down)
+            loaded.add(i)
+        created.append(pool.stats()["pages_created_total"])
+        # the new population, checked against the oracle
+        pop = sorted(loaded)
+        aid_np = rng.choice([-1] + pop, size=cfg.n_tokens).astype(np.int32)
+        r = pool.moe_forward_debug(0, x, to_dev(aid_np))
+        torch.cuda.synchronize()
+        assert pool.last_device_error() == 0, step
+        olayer = oracle_layer(cfg, 0, bank, tuned, base=base, adapters=loaded)
+        ids, w, slots, flips = check_routing(cfg, olayer, x_bits, aid_np, r)
+        check_output(olayer, x_bits, slots, w, bf16_to_f32(r["out"]))
+        # a token of an evicted adapter is served as a base token and flagged
+        gone = [a for a in range(cfg.max_adapters) if a not in loaded]
+        if gone:
+            bad = aid_np.copy()
+            bad[0] = gone[0]
+            pool.moe_forward(0, x, to_dev(bad))
+            torch.cuda.synchronize()
+            assert pool.last_device_error() == 8
+    st = pool.stats()
+    assert st["pages_mapped"] + st["pages_free"] == st["pages_created_total"]
+    assert created[-1] == max(created) and created[-1] <= created[len(created) // 2] + 1   # pages are reused, not re-created
+    pool.destroy()

@@ -195,7 +195,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
                             const size_t o = (size_t)(it.out_row + c0 + j) * out_rows_per_slot + orow;
                             if (GLU) {
                                 const float gv = __uint_as_float(g[j]), uv = __uint_as_float(u[j]);
-                                const float a = (gv / (1.f + __expf(-gv))) * uv;
+                                const float a = __fdividef(gv, 1.f + __expf(-gv)) * uv;      // silu(g) * u; the result is rounded to bf16
                                 reinterpret_cast<__nv_bfloat16 *>(out)[o] = __float2bfloat16_rn(a);
                             } else {
                                 reinterpret_cast<float *>(out)[o] = __uint_as_float(g[j]);

@@ -124,10 +124,11 @@ __global__ void __launch_bounds__(256) reroute_kernel(const int32_t *__restrict_
 
 // ------------------------------------------------------------------------------------------------
 // Scan + permute + plan.  Every CTA recomputes the exclusive scan of the (small) count array in
-// shared memory; CTAs 0..n-2 copy one token row per warp to its slot-contiguous position, the last
-// CTA publishes the offsets and writes the GEMM work items:
-//   shared experts first (all B rows each), then every non-empty slot; per group the items are ordered
-//   (weight tile, token block) so that CTAs working at the same time share a weight tile through L2.
+// shared memory; the first kPlanners CTAs publish the offsets and write the GEMM work items (the item
+// loop is a chain of dependent integer arithmetic, so it is spread over several CTAs), the other CTAs copy
+// one token row per warp to its slot-contiguous position.  Item order:
+//   per group the items are ordered (weight tile, token block) so that CTAs working at the same time
+//   share a weight tile through L2; thin and fat groups are merged evenly (see below).
 // ------------------------------------------------------------------------------------------------
 __device__ void block_exclusive_scan(const int32_t *__restrict__ in, int32_t *out, int n, int32_t *warp_sums) {
     // out[0..n] = exclusive scan of in[0..n-1] (out[n] = total); blockDim.x = 256
@@ -152,6 +153,8 @@ __device__ void block_exclusive_scan(const int32_t *__restrict__ in, int32_t *ou
     __syncthreads();
 }
 
+constexpr int kPlanners = 8;
+
 __global__ void __launch_bounds__(256) permute_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ slot_ids,
                                                       const int32_t *__restrict__ rank, const int32_t *__restrict__ counts,
                                                       int B, int k, int H, int P, int S, int NT, int R1, int R2,
@@ -164,10 +167,13 @@ __global__ void __launch_bounds__(256) permute_kernel(const uint4 *__restrict__ 
     __shared__ int32_t warp_sums[8];
     tc::pdl_launch_dependents();
     tc::pdl_wait();                                     // counts, slot ids and ranks come from the router kernel
-    block_exclusive_scan(counts, off, P, warp_sums);
+    int32_t *cnt_s = sm + (P + 1) + 4 * (P + S + 1);    // [P] the counts, staged once
+    for (int i = threadIdx.x; i < P; i += 256) cnt_s[i] = counts[i];
+    __syncthreads();
+    block_exclusive_scan(cnt_s, off, P, warp_sums);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (blockIdx.x + 1 < gridDim.x) {
-        const long long q = (long long)blockIdx.x * 8 + warp;
+    if (blockIdx.x >= kPlanners) {                       // the first CTAs (dispatched first) are the planners
+        const long long q = (long long)(blockIdx.x - kPlanners) * 8 + warp;
         if (q < (long long)B * k) {
             const int dest = off[slot_ids[q]] + rank[q];
             if (lane == 0) inv[q] = dest;
@@ -178,30 +184,45 @@ __global__ void __launch_bounds__(256) permute_kernel(const uint4 *__restrict__ 
         }
         return;
     }
-    // ---- planner CTA
-    for (int i = threadIdx.x; i <= P; i += 256) offsets[i] = off[i];
-    // groups: g < S shared expert g (rows = B); g >= S slot g - S (rows = counts)
+    // ---- planner CTAs: each repeats the (cheap) scans and writes the items of every kPlanners-th group
+    if (blockIdx.x == 0)
+        for (int i = threadIdx.x; i <= P; i += 256) offsets[i] = off[i];
+    // groups: g < S shared expert g (rows = B); g >= S slot g - S (rows = counts).  Two classes: "thin" groups
+    // (at most kThinRows rows: their items are weight streams) and "fat" ones (tensor-core bound at prefill).
+    // The two item sequences are merged evenly, so that at any moment the CTAs hold a mix of both and the
+    // weight stream of the thin items overlaps the arithmetic of the fat ones.
+    constexpr int kThinRows = 64;
     const int G = P + S;
-    int32_t *nblk = blk + G + 1;       // [G] scratch
+    int32_t *nblk = blk + G + 1;            // [G] token blocks of fat groups (0 for thin ones)
+    int32_t *blk_t = nblk + G;              // [G + 1] scan of the thin groups' token blocks
+    int32_t *nblk_t = blk_t + G + 1;        // [G]
     for (int g = threadIdx.x; g < G; g += 256) {
-        const int rows = g < S ? B : counts[g - S];
-        nblk[g] = (rows + NT - 1) / NT;
+        const int rows = g < S ? B : cnt_s[g - S];
+        const int nb = (rows + NT - 1) / NT;
+        const bool thin = rows <= kThinRows;
+        nblk[g] = thin ? 0 : nb;
+        nblk_t[g] = thin ? nb : 0;
     }
     __syncthreads();
     block_exclusive_scan(nblk, blk, G, warp_sums);
-    const int total_blocks = blk[G];
-    if (threadIdx.x == 0) { n_items[0] = total_blocks * R1; n_items[1] = total_blocks * R2; }
-    for (int g = warp; g < G; g += 8) {
-        const int nb = nblk[g];
+    block_exclusive_scan(nblk_t, blk_t, G, warp_sums);
+    const int fat_blocks = blk[G], thin_blocks = blk_t[G];
+    if (blockIdx.x == 0 && threadIdx.x == 0) { n_items[0] = (fat_blocks + thin_blocks) * R1; n_items[1] = (fat_blocks + thin_blocks) * R2; }
+    for (int g = warp + 8 * blockIdx.x; g < G; g += 8 * kPlanners) {
+        const bool thin = nblk_t[g] > 0;
+        const int nb = thin ? nblk_t[g] : nblk[g];
         if (nb == 0) continue;
         const bool shared = g < S;
-        const int rows = shared ? B : counts[g - S];
+        const int rows = shared ? B : cnt_s[g - S];
         const int slot = shared ? P + g : g - S;
         const int in0 = shared ? 0 : off[g - S];
         const int out0 = shared ? g * B : S * B + off[g - S];
         for (int pass = 0; pass < 2; ++pass) {
             const int R = pass ? R2 : R1;
-            GemmItem *dst = (pass ? items2 : items1) + (size_t)blk[g] * R;
+            const long long n_fat = (long long)fat_blocks * R, n_thin = (long long)thin_blocks * R;
+            const long long first = (long long)(thin ? blk_t[g] : blk[g]) * R;    // index inside the group's own class
+            const bool small = (n_fat + 1) * (n_thin + 1) < (1ll << 31);
+            GemmItem *dst = pass ? items2 : items1;
             for (int i = lane; i < nb * R; i += 32) {
                 const int tile = i / nb, c = i % nb;
                 GemmItem it;
@@ -211,7 +232,21 @@ __global__ void __launch_bounds__(256) permute_kernel(const uint4 *__restrict__ 
                 it.rows = min(NT, rows - c * NT);
                 it.from_x = (!pass && shared) ? 1 : 0;
                 it.pad0 = it.pad1 = 0;
-                dst[i] = it;
+                // merged position: thin item q has floor(q*n_fat/n_thin) fat items before it, and fat item q
+                // the thin items that rule puts before it
+                const long long q = first + i;
+                long long pos;
+                if (small) {                                  // every product fits 32 bits: cheap divisions
+                    const unsigned qu = (unsigned)q, nf = (unsigned)n_fat, nt = (unsigned)n_thin;
+                    if (thin) pos = nf ? qu + qu * nf / nt : qu;
+                    else pos = nt ? qu + min(nt, ((qu + 1) * nt + nf - 1) / nf) : qu;
+                } else {
+                    if (thin) pos = n_fat ? q + q * n_fat / n_thin : q;
+                    else pos = n_thin ? q + min(n_thin, ((q + 1) * n_thin + n_fat - 1) / n_fat) : q;
+                }
+                int4 *d4 = reinterpret_cast<int4 *>(dst + pos);      // one item = two 16-byte stores
+                d4[0] = make_int4(it.slot, it.tile, it.in_row, it.out_row);
+                d4[1] = make_int4(it.rows, it.from_x, 0, 0);
             }
         }
     }
@@ -269,8 +304,8 @@ int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
     const int R1 = (c.inter + 127) / 128, R2 = (c.hidden + 127) / 128;
     const long long pairs = (long long)B * c.top_k;
-    const int grid = (int)((pairs + 7) / 8) + 1;
-    const size_t smem = ((size_t)(p->P + 1) + 2 * (size_t)(p->P + c.num_shared) + 2) * 4;
+    const int grid = (int)((pairs + 7) / 8) + kPlanners;
+    const size_t smem = ((size_t)(p->P + 1) + 4 * (size_t)(p->P + c.num_shared + 1) + p->P) * 4;
     return launch_pdl(permute_kernel, dim3(grid), dim3(256), smem, st, (const uint4 *)x, p->ws.slot_ids, p->ws.rank,
                       p->ws.counts, B, c.top_k, c.hidden, p->P, c.num_shared, p->token_tile, R1, R2, p->ws.offsets, p->ws.inv,
                       (uint4 *)p->ws.xp, p->ws.items1, p->ws.items2, p->ws.n_items);

@@ -52,7 +52,7 @@ struct LayerState {
     std::vector<int32_t> pi_host;  // master copy
     bool base_loaded = false;
     CUtensorMap map_w13, map_w2;   // TMA descriptors over the two virtual tensors
-    CUtensorMap map_router;        // and over the router rows [M, H]
+    CUtensorMap map_router[3];     // and over the router rows [M, H], with boxes of 1, 2 and 4 K-atoms
 };
 
 }  // namespace ew

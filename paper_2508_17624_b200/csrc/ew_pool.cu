@@ -232,7 +232,9 @@ extern "C" ew_status_t ew_pool_create(const ew_config_t *cfg, ew_pool_t **out) {
                 uint32_t box[3] = {64, 128, 1};
                 if (make_tensor_map(p, &L.map_w13, (void *)L.w13.base, 3, d13, box) ||
                     make_tensor_map(p, &L.map_w2, (void *)L.w2.base, 3, d2, box) ||
-                    make_atom_map(p, &L.map_router, L.router_w, c.hidden, c.num_experts, (c.num_experts + 15) / 16 * 16, 4))
+                    make_atom_map(p, &L.map_router[0], L.router_w, c.hidden, c.num_experts, (c.num_experts + 15) / 16 * 16, 1) ||
+                    make_atom_map(p, &L.map_router[1], L.router_w, c.hidden, c.num_experts, (c.num_experts + 15) / 16 * 16, 2) ||
+                    make_atom_map(p, &L.map_router[2], L.router_w, c.hidden, c.num_experts, (c.num_experts + 15) / 16 * 16, 4))
                     return EW_ERR_CUDA;
             }
             ew_status_t s = alloc_workspace(p);

@@ -3,7 +3,7 @@
 //
 // One CTA owns `tok_tile` (32, 64 or 128) tokens.  The logits tile D[128, M] = X[128, H] * Wr[M, H]^T is
 // one tcgen05 accumulator (M <= 256 fp32 columns of TMEM); X and the router rows stream through a TMA
-// ring.  The kernel is latency-bound, so each TMA instruction fetches kAtoms 64-element K-atoms at once
+// ring.  The kernel is latency-bound, so each TMA instruction fetches up to four 64-element K-atoms at once
 // (3-D descriptors ordered element, row, atom: shared memory receives one swizzled tile per atom).  Only the first
 // `tok_tile` rows of the 128-row MMA tile are loaded; the other rows hold whatever shared memory held
 // and feed accumulator lanes nobody reads.  TMEM lane i belongs to token i, so in the epilogue every
@@ -24,7 +24,7 @@ using namespace tc;
 constexpr int kThreads = 192;
 constexpr int kTileRows = 128;
 constexpr int kMaxStages = 16;
-constexpr int kAtoms = 4;            // 64-element K-atoms per TMA box and pipeline stage
+constexpr int kMaxAtoms = 4;         // 64-element K-atoms per TMA box and pipeline stage: 4, 2 or 1
 constexpr int kMaxPiSmem = 16 * 1024;
 
 __device__ __forceinline__ int checked_aid(int a, int N, const int32_t *loaded, int *err) {
@@ -39,7 +39,7 @@ struct RouterArgs {
     const int32_t *aid, *pi, *loaded;
     int B, H, M, k, N, renormalize;
     float scale;
-    int stages, tmem_cols, pi_in_smem, tok_tile;
+    int stages, tmem_cols, pi_in_smem, tok_tile, atoms;
     int32_t *topk_ids;
     float *topk_w;
     int32_t *slot_ids, *rank, *counts;
@@ -80,7 +80,7 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
-    const int M = A.M, stages = A.stages, tok_tile = A.tok_tile;
+    const int M = A.M, stages = A.stages, tok_tile = A.tok_tile, kAtoms = A.atoms;
     const int n_mma = ((M + 15) >> 4) << 4;                          // router rows arrive as one box of n_mma rows
     const int x_atom = tok_tile * kBlockK * 2;                       // bytes of one K-atom of the token tile (multiple of 4 KiB)
     const int r_atom = (n_mma * kBlockK * 2 + 1023) & ~1023;         // and of the router tile
@@ -282,47 +282,74 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                      : "memory");
 }
 
+
+// Launch geometry of the router kernel for a batch of B tokens: tokens per CTA, K-atoms per stage, ring depth.
+struct RouterGeometry {
+    int tok_tile, atoms, stages, pi_in_smem, tmem_cols, grid;
+    bool reg;
+    size_t smem;
+};
+
+static bool router_geometry(const ew_pool *p, int B, RouterGeometry *g) {
+    const ew_config_t &c = p->cfg;
+    const int M = c.num_experts, n_mma = (M + 15) / 16 * 16;
+    // tokens per CTA: small batches are spread over more SMs (each CTA streams the whole router matrix)
+    g->tok_tile = B <= 32 * p->sm_count ? 32 : B <= 64 * p->sm_count ? 64 : 128;
+    const size_t pi_bytes = (size_t)c.max_adapters * M * 4;
+    g->pi_in_smem = pi_bytes <= (size_t)kMaxPiSmem;
+    const size_t tail = 1024 /*alignment*/ + kTileRows * kBlockK * 2 + 8 * (2 * kMaxStages + 1) + 16 +
+                        (g->pi_in_smem ? pi_bytes : 0) + 64;
+    g->reg = M <= 64;
+    const size_t pbuf_bytes = g->reg ? 0 : (size_t)M * kTileRows * 4;
+    for (int atoms = kMaxAtoms; atoms >= 1; atoms >>= 1) {      // as many K-atoms per stage as leave a ring of >= 3 (else 2) stages
+        const int stage_bytes = atoms * (g->tok_tile * kBlockK * 2 + ((n_mma * kBlockK * 2 + 1023) & ~1023));
+        int stages = (int)((227 * 1024 - tail) / stage_bytes);
+        if (stages > kMaxStages) stages = kMaxStages;
+        const bool fits = (size_t)stages * stage_bytes + kTileRows * kBlockK * 2 >= pbuf_bytes;
+        if ((stages >= 3 || (atoms == 1 && stages >= 2)) && fits) {
+            g->atoms = atoms;
+            g->stages = stages;
+            g->smem = (size_t)stages * stage_bytes + tail;
+            g->tmem_cols = n_mma <= 32 ? 32 : n_mma <= 64 ? 64 : n_mma <= 128 ? 128 : 256;
+            g->grid = (B + g->tok_tile - 1) / g->tok_tile;
+            return true;
+        }
+    }
+    return false;
+}
+
+static int router_launch(ew_pool *p, int layer, const void *x, const RouterGeometry &g, RouterArgs &A, bool pdl, cudaStream_t st) {
+    const ew_config_t &c = p->cfg;
+    const LayerState &L = p->layers[layer];
+    CUtensorMap map_x;
+    if (make_atom_map(p, &map_x, x, c.hidden, A.B, g.tok_tile, g.atoms)) return (int)cudaErrorInvalidValue;
+    const CUtensorMap &map_r = L.map_router[g.atoms == 4 ? 2 : g.atoms == 2 ? 1 : 0];
+    A.pi = L.pi_dev; A.loaded = p->ws.loaded;
+    A.H = c.hidden; A.M = c.num_experts; A.k = c.top_k; A.N = c.max_adapters; A.renormalize = c.renormalize;
+    A.scale = c.routed_scale;
+    A.stages = g.stages; A.tmem_cols = g.tmem_cols; A.pi_in_smem = g.pi_in_smem; A.tok_tile = g.tok_tile; A.atoms = g.atoms;
+    cudaError_t e = g.reg ? cudaFuncSetAttribute(router_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
+                          : cudaFuncSetAttribute(router_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return (int)e;
+    if (pdl) {
+        if (g.reg) return launch_pdl(router_kernel<true>, dim3(g.grid), dim3(kThreads), g.smem, st, map_x, map_r, A);
+        return launch_pdl(router_kernel<false>, dim3(g.grid), dim3(kThreads), g.smem, st, map_x, map_r, A);
+    }
+    if (g.reg) router_kernel<true><<<g.grid, kThreads, g.smem, st>>>(map_x, map_r, A);
+    else router_kernel<false><<<g.grid, kThreads, g.smem, st>>>(map_x, map_r, A);
+    return (int)cudaGetLastError();
+}
+
 }  // namespace
 
 int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B, cudaStream_t st) {
-    const ew_config_t &c = p->cfg;
-    const LayerState &L = p->layers[layer];
-    const int M = c.num_experts;
-    const int n_mma = (M + 15) / 16 * 16;
-    // tokens per CTA: small batches are spread over more SMs (each CTA streams the whole router matrix)
-    const int tok_tile = B <= 32 * p->sm_count ? 32 : B <= 64 * p->sm_count ? 64 : 128;
-    const int stage_bytes = kAtoms * (tok_tile * kBlockK * 2 + ((n_mma * kBlockK * 2 + 1023) & ~1023));
-    const size_t pi_bytes = (size_t)c.max_adapters * M * 4;
-    const int pi_in_smem = pi_bytes <= (size_t)kMaxPiSmem;
-    const size_t tail = 1024 /*alignment*/ + kTileRows * kBlockK * 2 + 8 * (2 * kMaxStages + 1) + 16 +
-                        (pi_in_smem ? pi_bytes : 0) + 64;
-    int stages = (int)((227 * 1024 - tail) / stage_bytes);
-    if (stages > kMaxStages) stages = kMaxStages;
-    const bool reg = M <= 64;
-    const size_t pbuf_bytes = reg ? 0 : (size_t)M * kTileRows * 4;
-    if ((size_t)stages * stage_bytes + kTileRows * kBlockK * 2 < pbuf_bytes || stages < 2)
-        return (int)cudaErrorInvalidConfiguration;
-    const size_t smem = (size_t)stages * stage_bytes + tail;
-    CUtensorMap map_x;
-    if (make_atom_map(p, &map_x, x, c.hidden, B, tok_tile, kAtoms)) return (int)cudaErrorInvalidValue;
+    RouterGeometry g;
+    if (!router_geometry(p, B, &g)) return (int)cudaErrorInvalidConfiguration;
     RouterArgs A;
-    A.aid = aid; A.pi = L.pi_dev; A.loaded = p->ws.loaded;
-    A.B = B; A.H = c.hidden; A.M = M; A.k = c.top_k; A.N = c.max_adapters; A.renormalize = c.renormalize;
-    A.scale = c.routed_scale;
-    A.stages = stages; A.tmem_cols = n_mma <= 32 ? 32 : n_mma <= 64 ? 64 : n_mma <= 128 ? 128 : 256;
-    A.pi_in_smem = pi_in_smem; A.tok_tile = tok_tile;
+    A.aid = aid; A.B = B;
     A.topk_ids = p->ws.topk_ids; A.topk_w = p->ws.topk_w; A.slot_ids = p->ws.slot_ids; A.rank = p->ws.rank;
     A.counts = p->ws.counts; A.err = p->ws.err;
-    static size_t attr_set[2] = {0, 0};
-    if (smem > attr_set[reg]) {
-        cudaError_t e = reg ? cudaFuncSetAttribute(router_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                            : cudaFuncSetAttribute(router_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return (int)e;
-        attr_set[reg] = smem;
-    }
-    const int grid = (B + tok_tile - 1) / tok_tile;
-    if (reg) return launch_pdl(router_kernel<true>, dim3(grid), dim3(kThreads), smem, st, map_x, L.map_router, A);
-    return launch_pdl(router_kernel<false>, dim3(grid), dim3(kThreads), smem, st, map_x, L.map_router, A);
+    return router_launch(p, layer, x, g, A, true, st);
 }
 
 }  // namespace ew
@@ -399,39 +426,14 @@ extern "C" ew_status_t ew_route_noalloc(ew_pool_t *p, int32_t layer, const void 
     if (n_tokens == 0) return EW_OK;
     if (!x || !adapter_ids || !topk_ids || !topk_w || !slot_ids || ((uintptr_t)x & 15)) return EW_ERR_INVALID_ARG;
 
-    const LayerState &L = p->layers[layer];
-    const int M = c.num_experts, B = n_tokens;
-    const int n_mma = (M + 15) / 16 * 16;
-    const int tok_tile = B <= 32 * p->sm_count ? 32 : B <= 64 * p->sm_count ? 64 : 128;
-    const int stage_bytes = kAtoms * (tok_tile * kBlockK * 2 + ((n_mma * kBlockK * 2 + 1023) & ~1023));
-    const size_t pi_bytes = (size_t)c.max_adapters * M * 4;
-    const int pi_in_smem = pi_bytes <= (size_t)kMaxPiSmem;
-    const size_t tail = 1024 + kTileRows * kBlockK * 2 + 8 * (2 * kMaxStages + 1) + 16 + (pi_in_smem ? pi_bytes : 0) + 64;
-    int stages = (int)((227 * 1024 - tail) / stage_bytes);
-    if (stages > kMaxStages) stages = kMaxStages;
-    const bool reg = M <= 64;
-    if (stages < 2 || (!reg && (size_t)stages * stage_bytes + kTileRows * kBlockK * 2 < (size_t)M * kTileRows * 4))
-        return EW_ERR_INVALID_ARG;
-    const size_t smem = (size_t)stages * stage_bytes + tail;
-    CUtensorMap map_x;
-    if (make_atom_map(p, &map_x, x, c.hidden, B, tok_tile, kAtoms)) return EW_ERR_CUDA;
+    RouterGeometry g;
+    if (!router_geometry(p, n_tokens, &g)) return EW_ERR_INVALID_ARG;
     RouterArgs A;
-    A.aid = adapter_ids; A.pi = L.pi_dev; A.loaded = p->ws.loaded;
-    A.B = B; A.H = c.hidden; A.M = M; A.k = c.top_k; A.N = c.max_adapters; A.renormalize = c.renormalize;
-    A.scale = c.routed_scale;
-    A.stages = stages; A.tmem_cols = n_mma <= 32 ? 32 : n_mma <= 64 ? 64 : n_mma <= 128 ? 128 : 256;
-    A.pi_in_smem = pi_in_smem; A.tok_tile = tok_tile;
+    A.aid = adapter_ids; A.B = n_tokens;
     A.topk_ids = topk_ids; A.topk_w = topk_w; A.slot_ids = slot_ids; A.counts = counts;
     A.rank = reinterpret_cast<int32_t *>(scratch + kNoAllocHeader);      // scratch: position of each pair in its slot
     A.err = reinterpret_cast<int *>(scratch);                            // scratch: device status word
-    e = reg ? cudaFuncSetAttribute(router_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
-            : cudaFuncSetAttribute(router_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e == cudaSuccess) {
-        const int grid = (B + tok_tile - 1) / tok_tile;
-        if (reg) router_kernel<true><<<grid, kThreads, smem, st>>>(map_x, L.map_router, A);
-        else router_kernel<false><<<grid, kThreads, smem, st>>>(map_x, L.map_router, A);
-        e = cudaGetLastError();
-    }
+    e = (cudaError_t)router_launch(p, layer, x, g, A, false, st);
     if (e == cudaSuccess && device_status)
         e = cudaMemcpyAsync(device_status, scratch, 4, cudaMemcpyDeviceToDevice, st);
     if (e != cudaSuccess) {

@@ -323,3 +323,42 @@ def test_adapter_churn_under_load():
     assert st["pages_mapped"] + st["pages_free"] == st["pages_created_total"]
     assert created[-1] == max(created) and created[-1] <= created[len(created) // 2] + 1   # pages are reused, not re-created
     pool.destroy()
+
+
+@pytest.mark.parametrize("shape", [
+    dict(hidden=64, inter=8, num_experts=4, num_shared=0, top_k=1, max_adapters=1, e_max=1, n_tokens=5),      # smallest legal sizes
+    dict(hidden=128, inter=200, num_experts=40, num_shared=1, top_k=5, max_adapters=3, e_max=4, n_tokens=77),  # I, M off the tile sizes
+    dict(hidden=192, inter=136, num_experts=8, num_shared=2, top_k=8, max_adapters=2, e_max=8, n_tokens=40),   # k = M: dense mixture
+    dict(hidden=256, inter=128, num_experts=80, num_shared=0, top_k=3, max_adapters=2, e_max=2, n_tokens=130), # M > 64: shared-memory softmax path
+    dict(hidden=64, inter=64, num_experts=256, num_shared=1, top_k=4, max_adapters=1, e_max=3, n_tokens=33),   # the largest M
+])
+@pytest.mark.parametrize("renorm", [0, 1])
+def test_odd_shapes(shape, renorm):
+    """Shapes off every tile size, degenerate top-k, no shared experts, renormalised and scaled weights."""
+    import torch
+    cfg = wl.MoEConfig(name="odd", num_layers=1, seed=21, **shape)
+    bank = wl.NoiseBank(cfg.seed)
+    rng = np.random.default_rng(21)
+    scale = 2.5 if renorm else 1.0
+    pool = binding.Pool.from_config(cfg, renormalize=renorm, routed_scale=scale)
+    counts = rng.integers(0, cfg.e_max + 1, size=(cfg.max_adapters, 1))
+    counts[0, 0] = cfg.e_max
+    tuned = wl.tuned_sets(cfg, counts)
+    _, bases = binding.load_model(pool, cfg, bank, tuned=tuned)
+    olayer = oracle_layer(cfg, 0, bank, tuned, base=bases[0])
+    olayer.cfg.renormalize, olayer.cfg.routed_scale = renorm, scale
+    x = wl.gen_tokens(cfg)
+    if cfg.num_experts > 64:      # spread the logits so that the 1e-5 near-tie window stays rare with many experts
+        x = wl.f32_to_bf16_bits(wl.bf16_bits_to_f32(x) * 6.0)
+    aid = wl.gen_adapter_ids(cfg, mode="uniform")
+    r = pool.moe_forward_debug(0, to_dev(x), to_dev(aid))
+    torch.cuda.synchronize()
+    assert pool.last_device_error() == 0
+    ids, w, slots, flips = check_routing(cfg, olayer, x, aid, r)
+    assert flips <= max(2, cfg.n_tokens // 20)
+    ref = oracle.ffn_given_slots(olayer, x, slots, w)
+    got = bf16_to_f32(r["out"])
+    tol = 2e-2 * max(1.0, float(np.abs(ref).max()) / 2.0)      # the absolute bound scales with the output magnitude
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-2
+    assert np.abs(got - ref).max() <= tol
+    pool.destroy()

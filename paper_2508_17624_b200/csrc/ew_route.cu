@@ -13,52 +13,65 @@ namespace {
 
 // ------------------------------------------------------------------------------------------------
 // Batched rerouting alone: slot = aid < 0 ? id : Pi[aid][id] (bad adapter ids behave as -1 and raise
-// bit 0 of the error word).  A CTA moves tiles of 256 tokens (256*k ids, so every tile starts 16-byte
-// aligned) through a three-stage shared-memory ring filled by 16-byte asynchronous copies (two tiles
-// ahead are in flight); a thread rewrites 16-byte vectors of four ids in place (the token of an id is a
-// multiply-shift on its index inside the tile, exact for i < 8192 and k <= 32; adapter ids are staged
-// per tile), and the tile leaves with coalesced 16-byte streaming stores.  Expert map and loaded flags
-// sit in shared memory; the per-CTA shared-memory histogram is flushed with one atomic per non-empty slot.
+// bit 0 of the error word).  A persistent CTA moves tiles of 256 tokens (256*k ids plus their 256
+// adapter ids) through a four-stage shared-memory ring with bulk asynchronous copies in both
+// directions (cp.async.bulk global->shared completing on an mbarrier, shared->global as bulk groups),
+// so the data path costs a handful of instructions per tile and many tiles are in flight per SM; the
+// threads only rewrite the ids in place, four at a time (the token of an id is a multiply-shift on
+// its index inside the tile, exact for i < 8192 and k <= 32).  Expert map and loaded flags sit in
+// shared memory; the per-CTA shared-memory histogram is flushed with one atomic per non-empty slot.
+// Buffers that are not 16-byte aligned take reroute_kernel_unaligned (one thread per pair).
 // ------------------------------------------------------------------------------------------------
 constexpr int kRerouteTok = 256;
-constexpr int kRerouteStages = 3;
+constexpr int kRerouteStages = 4;
 
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
-                 : "memory");
+__device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void *gmem_src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_dst), "l"(gmem_src), "r"(bytes), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_store(void *gmem_dst, uint32_t smem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gmem_dst), "r"(smem_src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 
 __global__ void __launch_bounds__(256) reroute_kernel(const int32_t *__restrict__ ids, const int32_t *__restrict__ aid,
                                                       const int32_t *__restrict__ pi, const int32_t *__restrict__ loaded,
-                                                      int n_tokens, int k, int M, int N, int P, int vec_ok,
+                                                      int n_tokens, int k, int M, int N, int P,
                                                       int32_t *__restrict__ slots, int32_t *__restrict__ counts, int *err) {
-    extern __shared__ int32_t smem_i[];
-    const int tile_ints_max = kRerouteTok * k;         // multiple of 4 ints: every stage stays 16-byte aligned
-    const int stage_ints = tile_ints_max;
-    int32_t *tiles = smem_i;                           // [kRerouteStages][256 * k]
-    int32_t *pi_s = tiles + kRerouteStages * stage_ints, *hist = pi_s + N * M, *loaded_s = hist + P, *aid_s = loaded_s + N;
+    extern __shared__ __align__(128) int32_t smem_i[];
+    const int tile_ints_max = kRerouteTok * k;
+    const int stage_ints = kRerouteTok + tile_ints_max;            // a stage = 256 adapter ids, then 256*k ids (both 16-byte multiples)
+    int32_t *stages = smem_i;
+    int32_t *pi_s = stages + kRerouteStages * stage_ints, *hist = pi_s + N * M, *loaded_s = hist + P;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(((uintptr_t)(loaded_s + N) + 7) & ~(uintptr_t)7);
+    __shared__ int abort_flag;
     for (int i = threadIdx.x; i < N * M; i += blockDim.x) pi_s[i] = pi[i];
     for (int i = threadIdx.x; i < N; i += blockDim.x) loaded_s[i] = loaded[i];
     if (counts)
         for (int i = threadIdx.x; i < P; i += blockDim.x) hist[i] = 0;
-    __syncthreads();                                   // the staged flags are read right away (adapter-id check)
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kRerouteStages; ++s) tc::mbar_init(tc::smem_u32(bars + s), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
     const unsigned div_magic = ((1u << 20) + k - 1) / k;
     const int n_tiles = (n_tokens + kRerouteTok - 1) / kRerouteTok;
     int flags = 0;
-    auto tile_ints = [&](int tl) { return min(kRerouteTok, n_tokens - tl * kRerouteTok) * k; };
-    // asynchronous copy of tile tl into stage st (16-byte pieces; unaligned buffers fall back to plain loads)
-    auto fetch = [&](int tl, int st) {
-        if (tl < n_tiles) {
-            const int32_t *src = ids + (size_t)tl * tile_ints_max;
-            int32_t *dst = tiles + st * stage_ints;
-            const int n_int = tile_ints(tl), n_vec = vec_ok ? n_int >> 2 : 0;
-            for (int i = threadIdx.x; i < n_vec; i += 256) cp_async16(dst + 4 * i, src + 4 * i);
-            for (int i = (n_vec << 2) + threadIdx.x; i < n_int; i += 256) dst[i] = src[i];
-        }
-        cp_async_commit();                             // one group per call, empty or not, keeps the wait count uniform
+    // thread 0 starts the two bulk loads of tile tl into stage s; a tail shorter than 16 bytes is fetched with plain loads
+    auto fetch = [&](int tl, int s) {
+        const int n_tok = min(kRerouteTok, n_tokens - tl * kRerouteTok), n_int = n_tok * k;
+        const uint32_t ab = (uint32_t)(n_tok & ~3) * 4, ib = (uint32_t)(n_int & ~3) * 4;
+        const uint32_t bar = tc::smem_u32(bars + s);
+        int32_t *st = stages + s * stage_ints;
+        const int32_t *asrc = aid + (size_t)tl * kRerouteTok, *isrc = ids + (size_t)tl * tile_ints_max;
+        for (int i = n_tok & ~3; i < n_tok; ++i) st[i] = asrc[i];              // before the arrive, which releases them
+        for (int i = n_int & ~3; i < n_int; ++i) st[kRerouteTok + i] = isrc[i];
+        tc::mbar_expect_tx(bar, ab + ib);
+        if (ab) bulk_load(tc::smem_u32(st), asrc, ab, bar);
+        if (ib) bulk_load(tc::smem_u32(st + kRerouteTok), isrc, ib, bar);
     };
     auto checked = [&](int a) -> int {                 // adapter ids outside [-1,N) or of unloaded adapters act as -1
         if (a < -1 || a >= N || (a >= 0 && !loaded_s[a])) { flags |= 1; a = -1; }
@@ -70,55 +83,74 @@ __global__ void __launch_bounds__(256) reroute_kernel(const int32_t *__restrict_
         if (counts) atomicAdd(hist + sl, 1);
         return sl;
     };
-    for (int s0 = 0; s0 < kRerouteStages - 1; ++s0) fetch(blockIdx.x + s0 * gridDim.x, s0);
-    int st = 0;
-    for (int tl = blockIdx.x; tl < n_tiles; tl += gridDim.x) {
-        const size_t base = (size_t)tl * tile_ints_max;
-        const int n_int = tile_ints(tl), n_vec = n_int >> 2;     // n_int is a multiple of k; tiles but the last of 256*k
-        int32_t *tile = tiles + st * stage_ints;
-        {
-            const int t = tl * kRerouteTok + threadIdx.x;
-            const int a = checked(t < n_tokens ? __ldg(aid + t) : -1);
-            __syncthreads();                           // previous tile fully processed and stored; tables staged
-            aid_s[threadIdx.x] = a;
-        }
-        // the stage freed by the previous tile receives the tile kRerouteStages-1 ahead
-        fetch(tl + (kRerouteStages - 1) * gridDim.x, (st + kRerouteStages - 1) % kRerouteStages);
-        cp_async_wait<kRerouteStages - 1>();           // this tile's group has landed
+    if (threadIdx.x == 0)
+        for (int s = 0; s < kRerouteStages; ++s)
+            if (blockIdx.x + s * (int)gridDim.x < n_tiles) fetch(blockIdx.x + s * gridDim.x, s);
+    int it = 0;
+    for (int tl = blockIdx.x; tl < n_tiles; tl += gridDim.x, ++it) {
+        const int s = it % kRerouteStages;
+        const uint32_t parity = (it / kRerouteStages) & 1;
+        const int n_tok = min(kRerouteTok, n_tokens - tl * kRerouteTok), n_int = n_tok * k, n_vec = n_int >> 2;
+        int32_t *aid_s = stages + s * stage_ints, *tile = aid_s + kRerouteTok;
+        // one warp polls the barrier, the others sleep in the CTA barrier instead of spending issue slots on polling
+        if (threadIdx.x < 32) tc::mbar_wait(tc::smem_u32(bars + s), parity, &abort_flag, err);
         __syncthreads();
+        if (abort_flag) break;
         for (int v = threadIdx.x; v < n_vec; v += 256) {
             int4 r = reinterpret_cast<int4 *>(tile)[v];
             const int i0 = v << 2;
             int tok = (int)(((unsigned)i0 * div_magic) >> 20);
             int rem = i0 - tok * k;                    // position of the vector's first id inside its token's row
-            int a = aid_s[tok];
+            int a = checked(aid_s[tok]);
             int *e = reinterpret_cast<int *>(&r);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                if (rem == k) { rem = 0; a = aid_s[++tok]; }
+                if (rem == k) { rem = 0; a = checked(aid_s[++tok]); }
                 e[j] = map_one(e[j], a);
                 ++rem;
             }
             reinterpret_cast<int4 *>(tile)[v] = r;
         }
         for (int i = (n_vec << 2) + threadIdx.x; i < n_int; i += 256)       // last tile when its length is not a multiple of 4
-            tile[i] = map_one(tile[i], aid_s[((unsigned)i * div_magic) >> 20]);
+            tile[i] = map_one(tile[i], checked(aid_s[((unsigned)i * div_magic) >> 20]));
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");          // generic-proxy writes -> visible to the bulk store
         __syncthreads();
-        if (vec_ok) {
-            for (int i = threadIdx.x; i < n_vec; i += 256)
-                __stcs(reinterpret_cast<int4 *>(slots + base) + i, reinterpret_cast<const int4 *>(tile)[i]);
-            for (int i = (n_vec << 2) + threadIdx.x; i < n_int; i += 256) slots[base + i] = tile[i];
-        } else {
-            for (int i = threadIdx.x; i < n_int; i += 256) slots[base + i] = tile[i];
+        if (threadIdx.x == 0) {
+            int32_t *dst = slots + (size_t)tl * tile_ints_max;
+            const uint32_t ib = (uint32_t)(n_int & ~3) * 4;
+            if (ib) bulk_store(dst, tc::smem_u32(tile), ib);
+            bulk_commit();
+            for (int i = n_int & ~3; i < n_int; ++i) dst[i] = tile[i];
+            // the stage used one tile ago has been read out by its store by now: refill it
+            if (it >= 1) {
+                bulk_wait_read<1>();
+                const int nxt = tl + (kRerouteStages - 1) * (int)gridDim.x;
+                if (nxt < n_tiles) fetch(nxt, (it - 1) % kRerouteStages);
+            }
         }
-        st = (st + 1) % kRerouteStages;
     }
-    cp_async_wait<0>();
+    if (threadIdx.x == 0) bulk_wait_read<0>();
     if (flags) atomicOr(err, flags);
     if (counts) {
         __syncthreads();
         for (int i = threadIdx.x; i < P; i += blockDim.x)
             if (hist[i]) atomicAdd(counts + i, hist[i]);
+    }
+}
+
+// any alignment: one thread per (token, expert) pair
+__global__ void __launch_bounds__(256) reroute_kernel_unaligned(const int32_t *__restrict__ ids, const int32_t *__restrict__ aid,
+                                                                const int32_t *__restrict__ pi, const int32_t *__restrict__ loaded,
+                                                                long long n_pairs, int k, int M, int N,
+                                                                int32_t *__restrict__ slots, int32_t *__restrict__ counts, int *err) {
+    for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n_pairs; q += (long long)gridDim.x * blockDim.x) {
+        int a = aid[q / k];
+        if (a < -1 || a >= N || (a >= 0 && !loaded[a])) { atomicOr(err, 1); a = -1; }
+        const int e = ids[q];
+        if ((unsigned)e >= (unsigned)M) { atomicOr(err, 4); slots[q] = e; continue; }
+        const int sl = a < 0 ? e : pi[a * M + e];
+        slots[q] = sl;
+        if (counts) atomicAdd(counts + sl, 1);
     }
 }
 
@@ -320,10 +352,18 @@ int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st) {
 int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid, int B, int32_t *slots,
                    int32_t *counts, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
+    const int32_t *pi = p->layers[layer].pi_dev;
+    if ((((uintptr_t)ids | (uintptr_t)slots | (uintptr_t)aid) & 15) != 0) {
+        const long long pairs = (long long)B * c.top_k;
+        long long blocks = (pairs + 255) / 256;
+        if (blocks > (long long)p->sm_count * 8) blocks = (long long)p->sm_count * 8;
+        reroute_kernel_unaligned<<<(int)blocks, 256, 0, st>>>(ids, aid, pi, p->ws.loaded, pairs, c.top_k, c.num_experts,
+                                                              c.max_adapters, slots, counts, p->ws.err);
+        return (int)cudaGetLastError();
+    }
     long long blocks = ((long long)B + kRerouteTok - 1) / kRerouteTok;
-    const size_t smem = ((size_t)kRerouteStages * kRerouteTok * c.top_k + (size_t)c.max_adapters * c.num_experts + p->P + c.max_adapters + kRerouteTok) * 4 + 16;
-    // 16-byte accesses need aligned buffers; every tile starts at a multiple of 256*k ints
-    const int vec_ok = (((uintptr_t)ids | (uintptr_t)slots) & 15) == 0;
+    const size_t smem = ((size_t)kRerouteStages * kRerouteTok * (c.top_k + 1) + (size_t)c.max_adapters * c.num_experts + p->P +
+                         c.max_adapters) * 4 + 8 * kRerouteStages + 32;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(reroute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return (int)e;
@@ -333,8 +373,8 @@ int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, reroute_kernel, 256, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
     const long long cap = (long long)p->sm_count * per_sm;
     if (blocks > cap) blocks = cap;
-    reroute_kernel<<<(int)blocks, 256, smem, st>>>(ids, aid, p->layers[layer].pi_dev, p->ws.loaded, B, c.top_k,
-                                                   c.num_experts, c.max_adapters, p->P, vec_ok, slots, counts, p->ws.err);
+    reroute_kernel<<<(int)blocks, 256, smem, st>>>(ids, aid, pi, p->ws.loaded, B, c.top_k, c.num_experts, c.max_adapters,
+                                                   p->P, slots, counts, p->ws.err);
     return (int)cudaGetLastError();
 }
 

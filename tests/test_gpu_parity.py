@@ -148,6 +148,25 @@ def test_reroute_operator_c4_sample():
     assert np.array_equal(slots.cpu().numpy(), want)
     assert np.array_equal(cnt.cpu().numpy(), oracle.counts(want, cfg.num_slots))
     assert pool.last_device_error() == 0
+    # buffers that are not 16-byte aligned (views starting one row in) take the generic kernel
+    big_ids = torch.zeros((ids.shape[0] + 1, cfg.top_k), dtype=torch.int32, device="cuda")
+    big_ids[1:] = to_dev(ids)
+    big_aid = torch.zeros(aid.shape[0] + 1, dtype=torch.int32, device="cuda")
+    big_aid[1:] = to_dev(aid)
+    assert big_ids[1:].data_ptr() % 16 != 0
+    slots2, cnt2 = pool.reroute(0, big_ids[1:], big_aid[1:])
+    torch.cuda.synchronize()
+    assert np.array_equal(slots2.cpu().numpy(), want) and torch.equal(cnt2, cnt)
+    # ids outside [0, M) pass through unchanged and raise the flag; bad adapter ids act as base tokens
+    bad_ids = to_dev(ids).clone()
+    bad_ids[5, 2] = cfg.num_experts + 7
+    bad_aid = to_dev(aid).clone()
+    bad_aid[9] = cfg.max_adapters
+    slots3, _ = pool.reroute(0, bad_ids, bad_aid)
+    torch.cuda.synchronize()
+    assert int(slots3[5, 2]) == cfg.num_experts + 7
+    assert torch.equal(slots3[9], bad_ids[9])
+    assert pool.last_device_error() in (1, 8)
     pool.destroy()
 
 

@@ -381,3 +381,37 @@ def test_odd_shapes(shape, renorm):
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-2
     assert np.abs(got - ref).max() <= tol
     pool.destroy()
+
+
+def test_c3_stack_throughput_report():
+    """Timing of a 4-layer slice of the stacked configuration (1024 tokens per layer, 20 adapters, Zipf ids):
+    layers back to back on one stream.  Reported, with a loose sanity bound (the per-layer weight stream is
+    ~3.8 GB, so a layer cannot take less than 0.5 ms nor, on a healthy B200, more than 3 ms)."""
+    import torch
+    cfg = wl.with_(wl.CONFIGS["c3"], num_layers=4)
+    bank = wl.NoiseBank(cfg.seed)
+    pool = binding.Pool.from_config(cfg)
+    binding.load_model(pool, cfg, bank)
+    aid = to_dev(wl.gen_adapter_ids(cfg))
+    xs = [to_dev(wl.gen_tokens(cfg, l)) for l in range(cfg.num_layers)]
+    outs = [torch.empty_like(x) for x in xs]
+    for _ in range(3):
+        for l in range(cfg.num_layers):
+            pool.moe_forward(l, xs[l], aid, outs[l])
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    reps = 20
+    for _ in range(reps):
+        for l in range(cfg.num_layers):
+            pool.moe_forward(l, xs[l], aid, outs[l])
+    e1.record()
+    torch.cuda.synchronize()
+    ms_layer = e0.elapsed_time(e1) / (reps * cfg.num_layers)
+    d = pool.moe_forward_debug(0, xs[0], aid)
+    live = int((d["counts"] > 0).sum()) + cfg.num_shared
+    gb = live * 3 * cfg.inter * cfg.hidden * 2 / 1e9
+    print(f"c3: {ms_layer:.4f} ms per layer, {live} live experts, {gb:.2f} GB of weights per layer, "
+          f"{gb / ms_layer:.2f} TB/s, {cfg.n_tokens / ms_layer / 26:.1f} k tokens/s through a 26-layer stack")
+    assert 0.5 < ms_layer < 3.0
+    pool.destroy()

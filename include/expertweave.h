@@ -141,6 +141,9 @@ ew_status_t ew_pool_trim(ew_pool_t *pool);
  *   out          device bf16 [n_tokens, H]
  *   cuda_stream  a cudaStream_t (null = the legacy default stream)
  * No host synchronisation; token counts never leave the device.  n_tokens = 0 is a no-op.
+ * The call may be captured into a CUDA graph after one uncaptured warm-up call with the same n_tokens;
+ * ew_unload_adapter and ew_load_base wait for forwards issued directly, not for replays of such a graph:
+ * synchronise those yourself before evicting.
  * Errors: EW_ERR_INVALID_ARG (null, layer out of range, n_tokens > max_tokens), EW_ERR_NOT_LOADED,
  * EW_ERR_NO_DEVICE, EW_ERR_CUDA (launch failure). */
 ew_status_t ew_moe_forward(ew_pool_t *pool, int32_t layer, const void *x, const int32_t *adapter_ids,

@@ -50,8 +50,8 @@ template <int NT, bool GLU>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
                     const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_a_big,
-                    const __grid_constant__ CUtensorMap map_x_big, const GemmItem *__restrict__ items,
-                    const int32_t *__restrict__ n_items_ptr, int K, int out_rows_per_slot, void *__restrict__ out,
+                    const __grid_constant__ CUtensorMap map_x_big, const GemmItem *items,
+                    const int32_t *n_items_ptr, int K, int out_rows_per_slot, void *out,
                     int *err) {
     using C = Cfg<NT, GLU>;
     extern __shared__ uint8_t smem_raw[];
@@ -93,8 +93,11 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
-    pdl_wait();                                         // the item list and the activations come from the previous kernels
-    const int n_items = *n_items_ptr;
+    // The item list and the activations come from the previous kernels: nothing of them may be read before this
+    // wait.  (The pointers are deliberately not __restrict__/const-qualified read-only data: the compiler may
+    // hoist such loads above the wait.)
+    pdl_wait();
+    const int n_items = *reinterpret_cast<const volatile int32_t *>(n_items_ptr);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -230,7 +233,7 @@ int launch_one(ew_pool *p, const CUtensorMap &mw, const CUtensorMap &ma, const C
                const CUtensorMap &mxb, const GemmItem *items, const int32_t *n_items, int K, int out_rows, void *out,
                cudaStream_t st) {
     using C = Cfg<NT, GLU>;
-    return launch_pdl(grouped_gemm_kernel<NT, GLU>, dim3(p->sm_count), dim3(kThreads), C::kSmemBytes, st, mw, ma, mx, mab,
+    return launch_pdl(GLU ? 2 : 3, grouped_gemm_kernel<NT, GLU>, dim3(p->sm_count), dim3(kThreads), C::kSmemBytes, st, mw, ma, mx, mab,
                       mxb, items, n_items, K, out_rows, out, p->ws.err);
 }
 

@@ -87,10 +87,13 @@ namespace ew {
 
 void set_last_error(const std::string &s);
 
+// EW_DISABLE_PDL=1 in the environment turns the launch overlap off (plain stream order), for debugging.
+bool pdl_enabled(int kind = -1);
+
 // Launch with programmatic stream serialization (the kernel calls pdl_wait() before it reads its
 // predecessor's output).
 template <class... KArgs, class... Args>
-int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+int launch_pdl(int kind, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -100,7 +103,7 @@ int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cud
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = pdl_enabled(kind) ? 1 : 0;
     return (int)cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 

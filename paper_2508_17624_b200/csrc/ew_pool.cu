@@ -1,6 +1,7 @@
 // Host side of the C ABI: pool creation, base / adapter loading and eviction, the forward call.
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -9,6 +10,11 @@
 namespace ew {
 static thread_local std::string g_last_error;
 void set_last_error(const std::string &s) { g_last_error = s; }
+bool pdl_enabled(int kind) {
+    static const bool on = [] { const char *e = getenv("EW_DISABLE_PDL"); return !(e && e[0] == '1'); }();
+    static const int mask = [] { const char *e = getenv("EW_PDL_MASK"); return e ? atoi(e) : 31; }();
+    return on && (kind < 0 || ((mask >> kind) & 1));
+}
 }  // namespace ew
 
 using namespace ew;
@@ -478,6 +484,10 @@ extern "C" ew_status_t ew_last_device_error(ew_pool_t *p, int32_t *code) {
 }
 
 static ew_status_t note_forward(ew_pool *p, cudaStream_t st) {
+    // A forward that is being captured into a CUDA graph is not running yet: there is nothing to record.  The
+    // caller who replays such a graph orders its replays against ew_unload_adapter / ew_load_base itself.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap != cudaStreamCaptureStatusNone) return EW_OK;
     for (auto &e : p->fwd_events)
         if (e.first == st) {
             CU_TRY(cudaEventRecord(e.second, st));

@@ -162,7 +162,7 @@ __global__ void __launch_bounds__(256) reroute_kernel_unaligned(const int32_t *_
 //   per group the items are ordered (weight tile, token block) so that CTAs working at the same time
 //   share a weight tile through L2; thin and fat groups are merged evenly (see below).
 // ------------------------------------------------------------------------------------------------
-__device__ void block_exclusive_scan(const int32_t *__restrict__ in, int32_t *out, int n, int32_t *warp_sums) {
+__device__ void block_exclusive_scan(const int32_t *in, int32_t *out, int n, int32_t *warp_sums) {
     // out[0..n] = exclusive scan of in[0..n-1] (out[n] = total); blockDim.x = 256
     const int per = (n + 255) / 256;
     const int lo = min(threadIdx.x * per, n), hi = min(lo + per, n);
@@ -187,18 +187,20 @@ __device__ void block_exclusive_scan(const int32_t *__restrict__ in, int32_t *ou
 
 constexpr int kPlanners = 8;
 
-__global__ void __launch_bounds__(256) permute_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ slot_ids,
-                                                      const int32_t *__restrict__ rank, const int32_t *__restrict__ counts,
+__global__ void __launch_bounds__(256) permute_kernel(const uint4 *x, const int32_t *slot_ids,
+                                                      const int32_t *rank, const int32_t *counts,
                                                       int B, int k, int H, int P, int S, int NT, int R1, int R2,
-                                                      int32_t *__restrict__ offsets, int32_t *__restrict__ inv,
-                                                      uint4 *__restrict__ xp, GemmItem *__restrict__ items1,
-                                                      GemmItem *__restrict__ items2, int32_t *__restrict__ n_items) {
+                                                      int32_t *offsets, int32_t *inv,
+                                                      uint4 *xp, GemmItem *items1,
+                                                      GemmItem *items2, int32_t *n_items) {
     extern __shared__ int32_t sm[];
     int32_t *off = sm;                 // [P + 1]
     int32_t *blk = sm + P + 1;         // [P + S + 1] token blocks per group, scanned
     __shared__ int32_t warp_sums[8];
     tc::pdl_launch_dependents();
-    tc::pdl_wait();                                     // counts, slot ids and ranks come from the router kernel
+    // counts, slot ids and ranks come from the router kernel, x from the caller's earlier work: none of the kernel's
+    // pointer parameters is __restrict__, so that no load can be hoisted above this wait
+    tc::pdl_wait();
     int32_t *cnt_s = sm + (P + 1) + 4 * (P + S + 1);    // [P] the counts, staged once
     for (int i = threadIdx.x; i < P; i += 256) cnt_s[i] = counts[i];
     __syncthreads();
@@ -287,9 +289,9 @@ __global__ void __launch_bounds__(256) permute_kernel(const uint4 *__restrict__ 
 // ------------------------------------------------------------------------------------------------
 // out[t] = sum_j w[t,j] * Y[S*B + inv[t,j]] + sum_q Y[q*B + t], fp32, j in router order, one rounding
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) combine_kernel(const float4 *__restrict__ y, const int32_t *__restrict__ inv,
-                                                      const float *__restrict__ w, int B, int k, int H, int S,
-                                                      uint2 *__restrict__ out, int32_t *__restrict__ counts, int P) {
+__global__ void __launch_bounds__(256) combine_kernel(const float4 *y, const int32_t *inv,
+                                                      const float *w, int B, int k, int H, int S,
+                                                      uint2 *out, int32_t *counts, int P) {
     __shared__ int32_t rows[32];
     __shared__ float wts[32];
     const int t = blockIdx.x;
@@ -306,13 +308,13 @@ __global__ void __launch_bounds__(256) combine_kernel(const float4 *__restrict__
     for (int v = threadIdx.x; v < hv; v += blockDim.x) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int j = 0; j < k; ++j) {
-            const float4 a = __ldg(y + (size_t)rows[j] * hv + v);
+            const float4 a = y[(size_t)rows[j] * hv + v];
             const float wj = wts[j];
             acc.x = fmaf(wj, a.x, acc.x); acc.y = fmaf(wj, a.y, acc.y);
             acc.z = fmaf(wj, a.z, acc.z); acc.w = fmaf(wj, a.w, acc.w);
         }
         for (int q = 0; q < S; ++q) {
-            const float4 a = __ldg(y + ((size_t)q * B + t) * hv + v);
+            const float4 a = y[((size_t)q * B + t) * hv + v];
             acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
         }
         const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
@@ -338,14 +340,14 @@ int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st) {
     const long long pairs = (long long)B * c.top_k;
     const int grid = (int)((pairs + 7) / 8) + kPlanners;
     const size_t smem = ((size_t)(p->P + 1) + 4 * (size_t)(p->P + c.num_shared + 1) + p->P) * 4;
-    return launch_pdl(permute_kernel, dim3(grid), dim3(256), smem, st, (const uint4 *)x, p->ws.slot_ids, p->ws.rank,
+    return launch_pdl(1, permute_kernel, dim3(grid), dim3(256), smem, st, (const uint4 *)x, p->ws.slot_ids, p->ws.rank,
                       p->ws.counts, B, c.top_k, c.hidden, p->P, c.num_shared, p->token_tile, R1, R2, p->ws.offsets, p->ws.inv,
                       (uint4 *)p->ws.xp, p->ws.items1, p->ws.items2, p->ws.n_items);
 }
 
 int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
-    return launch_pdl(combine_kernel, dim3(B), dim3(256), 0, st, (const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B, c.top_k,
+    return launch_pdl(4, combine_kernel, dim3(B), dim3(256), 0, st, (const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B, c.top_k,
                       c.hidden, c.num_shared, (uint2 *)out, p->ws.counts, p->P);
 }
 

@@ -332,8 +332,8 @@ static int router_launch(ew_pool *p, int layer, const void *x, const RouterGeome
                           : cudaFuncSetAttribute(router_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return (int)e;
     if (pdl) {
-        if (g.reg) return launch_pdl(router_kernel<true>, dim3(g.grid), dim3(kThreads), g.smem, st, map_x, map_r, A);
-        return launch_pdl(router_kernel<false>, dim3(g.grid), dim3(kThreads), g.smem, st, map_x, map_r, A);
+        if (g.reg) return launch_pdl(0, router_kernel<true>, dim3(g.grid), dim3(kThreads), g.smem, st, map_x, map_r, A);
+        return launch_pdl(0, router_kernel<false>, dim3(g.grid), dim3(kThreads), g.smem, st, map_x, map_r, A);
     }
     if (g.reg) router_kernel<true><<<g.grid, kThreads, g.smem, st>>>(map_x, map_r, A);
     else router_kernel<false><<<g.grid, kThreads, g.smem, st>>>(map_x, map_r, A);

@@ -350,6 +350,7 @@ def test_adapter_churn_under_load():
     dict(hidden=192, inter=136, num_experts=8, num_shared=2, top_k=8, max_adapters=2, e_max=8, n_tokens=40),   # k = M: dense mixture
     dict(hidden=256, inter=128, num_experts=80, num_shared=0, top_k=3, max_adapters=2, e_max=2, n_tokens=130), # M > 64: shared-memory softmax path
     dict(hidden=64, inter=64, num_experts=256, num_shared=1, top_k=4, max_adapters=1, e_max=3, n_tokens=33),   # the largest M
+    dict(hidden=64, inter=64, num_experts=256, num_shared=0, top_k=2, max_adapters=20, e_max=1, n_tokens=70),  # expert map too large for shared memory
 ])
 @pytest.mark.parametrize("renorm", [0, 1])
 def test_odd_shapes(shape, renorm):
@@ -414,4 +415,86 @@ def test_c3_stack_throughput_report():
     print(f"c3: {ms_layer:.4f} ms per layer, {live} live experts, {gb:.2f} GB of weights per layer, "
           f"{gb / ms_layer:.2f} TB/s, {cfg.n_tokens / ms_layer / 26:.1f} k tokens/s through a 26-layer stack")
     assert 0.5 < ms_layer < 3.0
+    pool.destroy()
+
+
+def test_side_stream_and_cuda_graph():
+    """The forward is asynchronous on the caller's stream: it runs on a side stream, and it can be captured
+    into a CUDA graph (after a warm-up call) and replayed with the same bits as a direct call."""
+    import torch
+    cfg = wl.CONFIGS["c0"]
+    pool = binding.Pool.from_config(cfg)
+    binding.load_model(pool, cfg)
+    x, aid = to_dev(wl.gen_tokens(cfg)), to_dev(wl.gen_adapter_ids(cfg))
+    ref = pool.moe_forward(0, x, aid).clone()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    out = torch.empty_like(x)
+    with torch.cuda.stream(side):
+        pool.moe_forward(0, x, aid, out)
+    side.synchronize()
+    assert torch.equal(out, ref)
+    g = torch.cuda.CUDAGraph()
+    out2 = torch.zeros_like(x)
+    with torch.cuda.graph(g):
+        pool.moe_forward(0, x, aid, out2)
+    for _ in range(3):
+        out2.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out2, ref)
+    assert pool.last_device_error() == 0
+    # a direct call after the replays still works (the slot counters were left clean by the graph's last kernel)
+    assert torch.equal(pool.moe_forward(0, x, aid), ref)
+    pool.destroy()
+
+
+def test_two_pools_on_one_device():
+    import torch
+    c0, c1 = wl.CONFIGS["c0"], wl.with_(wl.CONFIGS["c0"], seed=5, max_adapters=1)
+    pa, pb = binding.Pool.from_config(c0), binding.Pool.from_config(c1)
+    binding.load_model(pa, c0)
+    binding.load_model(pb, c1)
+    xa, xb = to_dev(wl.gen_tokens(c0)), to_dev(wl.gen_tokens(c1))
+    aa, ab = to_dev(wl.gen_adapter_ids(c0)), to_dev(wl.gen_adapter_ids(c1))
+    ra, rb = pa.moe_forward(0, xa, aa).clone(), pb.moe_forward(0, xb, ab).clone()
+    for _ in range(5):                               # interleaved calls do not disturb each other's workspaces
+        oa, ob = pa.moe_forward(0, xa, aa), pb.moe_forward(0, xb, ab)
+    torch.cuda.synchronize()
+    assert torch.equal(oa, ra) and torch.equal(ob, rb) and not torch.equal(ra, rb)
+    pa.destroy()
+    pb.destroy()
+
+
+@pytest.mark.parametrize("name", ["c0", "c1"])
+def test_back_to_back_forwards_with_changing_inputs(name):
+    """The kernels of consecutive forwards overlap their launches; with a different batch in every call any
+    read that slipped ahead of its producer would pick up the previous batch's intermediate results."""
+    import torch
+    cfg = wl.CONFIGS[name]
+    pool = binding.Pool.from_config(cfg)
+    binding.load_model(pool, cfg)
+    rng = np.random.default_rng(0)
+    batches = []
+    for i in range(6):
+        n = cfg.n_tokens if i % 2 == 0 else max(1, cfg.n_tokens - 17 * i)
+        x = wl.f32_to_bf16_bits(rng.standard_normal((n, cfg.hidden)).astype(np.float32))
+        aid = rng.integers(-1, cfg.max_adapters, size=n).astype(np.int32)
+        batches.append((to_dev(x), to_dev(aid)))
+    ref = []
+    for x, aid in batches:                      # one at a time, fully synchronised
+        ref.append(pool.moe_forward(0, x, aid).clone())
+        torch.cuda.synchronize()
+    outs = [torch.empty_like(b[0]) for b in batches]
+    busy = torch.empty(1 << 28, dtype=torch.uint8, device="cuda")
+    for rep in range(6):
+        busy.zero_()                            # keeps the GPU busy so that the following launches queue up densely
+        order = rng.permutation(len(batches))
+        for i in order:
+            pool.moe_forward(0, batches[i][0], batches[i][1], outs[i])
+        torch.cuda.synchronize()
+        for i in range(len(batches)):
+            assert torch.equal(outs[i], ref[i]), (rep, i)
+            outs[i].zero_()
+    assert pool.last_device_error() == 0
     pool.destroy()

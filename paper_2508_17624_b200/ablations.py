@@ -9,6 +9,8 @@ Prints one JSON object:
                      (Section 5.3 "virtual weight tensor vs padding", Section 5.4 memory)
   churn              evicting and re-loading one adapter (8 experts, 132 MiB) while forwards are in flight:
                      host-side latency of ew_unload_adapter / ew_load_adapter and page reuse (Section 4.2)
+  batch_sweep        the c1 layer (4 adapters) from 1 to 8192 tokens per call: ms, tokens/s, live experts, weight
+                     stream TB/s and TFLOP/s (where the layer turns from weight-bound to tensor-bound)
   reroute            the batched rerouting step three ways: fused into the router kernel (its share of the
                      layer), the stand-alone operator, and the unfused formulation from stock tensor ops
                      (broadcast the adapter ids, compute offsets into the map, gather: the paper's
@@ -148,6 +150,26 @@ def main():
                     "adapter_bytes": int(ew3.w_gate.nbytes * 3), "forwards_in_flight": 20,
                     "pages_created_during_churn": pool.stats()["pages_created_total"] - created0,
                     "device_error": pool.last_device_error()}
+
+    # ---- batch-size sweep on a pool sized for 8192 tokens
+    big = binding.Pool.from_config(cfg, max_tokens=8192)
+    binding.load_model(big, cfg, bank)
+    rng = np.random.default_rng(0)
+    sweep = []
+    for B in (1, 4, 16, 64, 128, 256, 512, 1024, 2048, 4096, 8192):
+        xb = torch.from_numpy(wl.f32_to_bf16_bits(rng.standard_normal((B, cfg.hidden)).astype(np.float32)).view(np.int16)).cuda().view(torch.bfloat16)
+        ab = torch.from_numpy(rng.integers(-1, cfg.max_adapters, size=B).astype(np.int32)).cuda()
+        ob = torch.empty_like(xb)
+        dd = big.moe_forward_debug(0, xb, ab)
+        torch.cuda.synchronize()
+        live_b = int((dd["counts"] > 0).sum()) + cfg.num_shared
+        ms = _time(lambda: big.moe_forward(0, xb, ab, ob), min(args.steps, 200 if B <= 1024 else 50), torch)
+        gb = live_b * 3 * cfg.inter * cfg.hidden * 2 / 1e9
+        fl = (B * cfg.top_k + cfg.num_shared * B) * 6 * cfg.inter * cfg.hidden / 1e12
+        sweep.append({"tokens": B, "ms": ms, "tokens_per_s": B / ms * 1e3, "live_experts": live_b,
+                      "weight_stream_TBps": gb / ms, "TFLOPps": fl / ms * 1e3})
+    big.destroy()
+    res["batch_sweep"] = sweep
 
     # ---- stand-alone operator vs unfused tensor ops, at the decode batch and at 65536 tokens
     pi_dev = torch.from_numpy(pool.get_expert_map(0)).cuda()

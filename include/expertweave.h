@@ -161,11 +161,14 @@ ew_status_t ew_moe_forward_debug(ew_pool_t *pool, int32_t layer, const void *x, 
                                  float *topk_w, int32_t *slot_ids, int32_t *counts, int32_t *inv,
                                  int32_t *offsets);
 
-/* Same forward with HOST buffers: copies x and adapter_ids to device staging owned by the pool, runs
- * ew_moe_forward on them and copies the result back, all asynchronous on `cuda_stream` when the host
- * buffers are page-locked (pageable buffers make the copies synchronous).  The caller synchronises
- * the stream before reading out_host.  x_host, out_host: host bf16 [n_tokens, H]; adapter_ids_host:
- * host int32 [n_tokens]. */
+/* Same forward with HOST buffers, pipelined across calls: x and adapter_ids are uploaded to device staging
+ * owned by the pool, the forward runs on them and the result is downloaded to out_host.  Upload, kernels and
+ * download run on three streams of the pool with double-buffered staging, so that, with page-locked host
+ * buffers, the upload of the next call and the download of the previous one overlap the kernels of the current
+ * one (pageable buffers make the copies synchronous).  `cuda_stream` is made to wait for the download: the
+ * caller synchronises that stream (or an event recorded on it) before reading out_host or reusing x_host.
+ * The host buffers must be ready when the call is made (work queued earlier on `cuda_stream` is not waited for).
+ * x_host, out_host: host bf16 [n_tokens, H]; adapter_ids_host: host int32 [n_tokens]. */
 ew_status_t ew_moe_forward_host(ew_pool_t *pool, int32_t layer, const void *x_host,
                                 const int32_t *adapter_ids_host, int32_t n_tokens, void *out_host,
                                 void *cuda_stream);

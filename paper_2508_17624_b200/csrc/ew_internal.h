@@ -75,8 +75,13 @@ struct ew_pool {
     bool profiling = false;
     std::vector<cudaEvent_t> prof_events;   // 6 per recorded forward
     size_t prof_used = 0;                   // events in use
-    void *stage_x = nullptr, *stage_out = nullptr;   // device staging of ew_moe_forward_host
-    int32_t *stage_aid = nullptr;
+    // ew_moe_forward_host: double-buffered device staging and three internal streams, so that the upload of call
+    // n+1 and the download of call n-1 overlap the kernels of call n
+    void *stage_x[2] = {nullptr, nullptr}, *stage_out[2] = {nullptr, nullptr};
+    int32_t *stage_aid[2] = {nullptr, nullptr};
+    cudaStream_t host_h2d = nullptr, host_comp = nullptr, host_d2h = nullptr;
+    cudaEvent_t host_h2d_done[2] = {nullptr, nullptr}, host_comp_done[2] = {nullptr, nullptr}, host_d2h_done[2] = {nullptr, nullptr};
+    uint64_t host_calls = 0;
     uint64_t live_expert_bytes = 0, live_experts = 0;
     CUresult (*encode_tiled)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                              const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,

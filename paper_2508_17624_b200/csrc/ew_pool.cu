@@ -107,7 +107,8 @@ static ew_status_t alloc_workspace(ew_pool *p) {
         {(void **)&w.items2, rb * r2 * sizeof(GemmItem)}, {(void **)&w.xp, (Bm * k + 32) * H * 2},
         {(void **)&w.act, rows * I * 2}, {(void **)&w.y, rows * H * 4}, {(void **)&w.err, 256},
         {(void **)&w.loaded, (size_t)c.max_adapters * 4 + 16},
-        {&p->stage_x, Bm * H * 2}, {&p->stage_out, Bm * H * 2}, {(void **)&p->stage_aid, Bm * 4},
+        {&p->stage_x[0], Bm * H * 2}, {&p->stage_out[0], Bm * H * 2}, {(void **)&p->stage_aid[0], Bm * 4},
+        {&p->stage_x[1], Bm * H * 2}, {&p->stage_out[1], Bm * H * 2}, {(void **)&p->stage_aid[1], Bm * 4},
     };
     size_t total = 0;
     for (auto &s : segs) total += align_up(s.bytes, 1024);
@@ -151,6 +152,14 @@ static void destroy_pool(ew_pool *p) {
         if (p->ws.topk_ids) cudaFree(p->ws.topk_ids);   // the workspace is one allocation; topk_ids is its base
         for (auto &e : p->fwd_events) cudaEventDestroy(e.second);
         for (auto &e : p->prof_events) cudaEventDestroy(e);
+        for (int i = 0; i < 2; ++i) {
+            if (p->host_h2d_done[i]) cudaEventDestroy(p->host_h2d_done[i]);
+            if (p->host_comp_done[i]) cudaEventDestroy(p->host_comp_done[i]);
+            if (p->host_d2h_done[i]) cudaEventDestroy(p->host_d2h_done[i]);
+        }
+        if (p->host_h2d) cudaStreamDestroy(p->host_h2d);
+        if (p->host_comp) cudaStreamDestroy(p->host_comp);
+        if (p->host_d2h) cudaStreamDestroy(p->host_d2h);
         if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
     }
     delete p->be;
@@ -597,16 +606,43 @@ extern "C" ew_status_t ew_moe_forward_host(ew_pool_t *p, int32_t layer, const vo
     if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
     if (B == 0) return EW_OK;
     if (!x_host || !aid_host || !out_host) return EW_ERR_INVALID_ARG;
-    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaStream_t user = (cudaStream_t)cuda_stream;
     int dev = -1;
     CU_TRY(cudaGetDevice(&dev));
     if (dev != p->cfg.device) CU_TRY(cudaSetDevice(p->cfg.device));
-    size_t xb = (size_t)B * p->cfg.hidden * 2;
-    CU_TRY(cudaMemcpyAsync(p->stage_x, x_host, xb, cudaMemcpyHostToDevice, st));
-    CU_TRY(cudaMemcpyAsync(p->stage_aid, aid_host, (size_t)B * 4, cudaMemcpyHostToDevice, st));
-    ew_status_t s = ew_moe_forward(p, layer, p->stage_x, p->stage_aid, B, p->stage_out, cuda_stream);
+    if (!p->host_h2d) {                                   // first use: the pipeline's streams and events
+        CU_TRY(cudaStreamCreateWithFlags(&p->host_h2d, cudaStreamNonBlocking));
+        CU_TRY(cudaStreamCreateWithFlags(&p->host_comp, cudaStreamNonBlocking));
+        CU_TRY(cudaStreamCreateWithFlags(&p->host_d2h, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+            CU_TRY(cudaEventCreateWithFlags(&p->host_h2d_done[i], cudaEventDisableTiming));
+            CU_TRY(cudaEventCreateWithFlags(&p->host_comp_done[i], cudaEventDisableTiming));
+            CU_TRY(cudaEventCreateWithFlags(&p->host_d2h_done[i], cudaEventDisableTiming));
+        }
+    }
+    const int slot = (int)(p->host_calls & 1);
+    const bool reuse = p->host_calls >= 2;                // the slot was used two calls ago
+    const size_t xb = (size_t)B * p->cfg.hidden * 2;
+    // upload: may start as soon as the kernels of the call that last used this slot have read it
+    if (reuse) CU_TRY(cudaStreamWaitEvent(p->host_h2d, p->host_comp_done[slot], 0));
+    CU_TRY(cudaMemcpyAsync(p->stage_x[slot], x_host, xb, cudaMemcpyHostToDevice, p->host_h2d));
+    CU_TRY(cudaMemcpyAsync(p->stage_aid[slot], aid_host, (size_t)B * 4, cudaMemcpyHostToDevice, p->host_h2d));
+    CU_TRY(cudaEventRecord(p->host_h2d_done[slot], p->host_h2d));
+    // kernels: after the upload, after the download that last read this slot's output, and after forwards the
+    // caller issued directly on other streams (they share the workspace)
+    CU_TRY(cudaStreamWaitEvent(p->host_comp, p->host_h2d_done[slot], 0));
+    if (reuse) CU_TRY(cudaStreamWaitEvent(p->host_comp, p->host_d2h_done[slot], 0));
+    for (auto &e : p->fwd_events)
+        if (e.first != p->host_comp) CU_TRY(cudaStreamWaitEvent(p->host_comp, e.second, 0));
+    ew_status_t s = ew_moe_forward(p, layer, p->stage_x[slot], p->stage_aid[slot], B, p->stage_out[slot], p->host_comp);
     if (s != EW_OK) return s;
-    CU_TRY(cudaMemcpyAsync(out_host, p->stage_out, xb, cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaEventRecord(p->host_comp_done[slot], p->host_comp));
+    // download, then join the caller's stream: synchronising it covers the whole call
+    CU_TRY(cudaStreamWaitEvent(p->host_d2h, p->host_comp_done[slot], 0));
+    CU_TRY(cudaMemcpyAsync(out_host, p->stage_out[slot], xb, cudaMemcpyDeviceToHost, p->host_d2h));
+    CU_TRY(cudaEventRecord(p->host_d2h_done[slot], p->host_d2h));
+    CU_TRY(cudaStreamWaitEvent(user, p->host_d2h_done[slot], 0));
+    ++p->host_calls;
     return EW_OK;
 }
 

@@ -498,3 +498,39 @@ def test_back_to_back_forwards_with_changing_inputs(name):
             outs[i].zero_()
     assert pool.last_device_error() == 0
     pool.destroy()
+
+
+def test_host_buffer_pipeline():
+    """ew_moe_forward_host overlaps upload, kernels and download across calls with double-buffered staging:
+    different batches issued back to back (and mixed with direct device-side calls) give the direct results."""
+    import torch
+    cfg = wl.CONFIGS["c0"]
+    pool = binding.Pool.from_config(cfg)
+    binding.load_model(pool, cfg)
+    rng = np.random.default_rng(3)
+    host, ref = [], []
+    for i in range(7):
+        n = cfg.n_tokens - 5 * i
+        xb = wl.f32_to_bf16_bits(rng.standard_normal((n, cfg.hidden)).astype(np.float32))
+        ab = rng.integers(-1, cfg.max_adapters, size=n).astype(np.int32)
+        xh = torch.from_numpy(xb.view(np.int16).copy()).pin_memory()
+        ah = torch.from_numpy(ab.copy()).pin_memory()
+        oh = torch.zeros((n, cfg.hidden), dtype=torch.int16).pin_memory()
+        host.append((xh, ah, oh))
+        ref.append(pool.moe_forward(0, to_dev(xb), to_dev(ab)).clone())
+        torch.cuda.synchronize()
+    xd, ad = to_dev(wl.gen_tokens(cfg)), to_dev(wl.gen_adapter_ids(cfg))
+    direct_ref = pool.moe_forward(0, xd, ad).clone()
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for i, (xh, ah, oh) in enumerate(host):
+            pool.moe_forward_host(0, xh, ah, oh)
+            if i == 3:
+                direct = pool.moe_forward(0, xd, ad)          # a device-side call in the middle of the pipeline
+        torch.cuda.synchronize()
+        assert torch.equal(direct, direct_ref)
+        for (xh, ah, oh), r in zip(host, ref):
+            assert torch.equal(oh.cuda().view(torch.bfloat16), r), rep
+            oh.zero_()
+    assert pool.last_device_error() == 0
+    pool.destroy()

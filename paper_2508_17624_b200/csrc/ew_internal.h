@@ -61,6 +61,7 @@ struct ew_pool {
     ew_config_t cfg;
     int P = 0;                      // M + N * E_max
     int token_tile = 32;            // NT: token rows per GEMM work item
+    bool use_pairs = false;         // NT = 256: GEMM-2's work items are processed by CTA pairs (cta_group::2)
     ew::PageBackend *be = nullptr;
     ew::PagePool pages;
     std::vector<ew::LayerState> layers;
@@ -94,6 +95,8 @@ void set_last_error(const std::string &s);
 
 // EW_DISABLE_PDL=1 in the environment turns the launch overlap off (plain stream order), for debugging.
 bool pdl_enabled(int kind = -1);
+// EW_DISABLE_PAIRS=1 keeps prefill-sized token tiles on the one-CTA kernel.
+bool pairs_enabled();
 
 // Launch with programmatic stream serialization (the kernel calls pdl_wait() before it reads its
 // predecessor's output).

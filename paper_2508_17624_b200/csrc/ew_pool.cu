@@ -10,6 +10,10 @@
 namespace ew {
 static thread_local std::string g_last_error;
 void set_last_error(const std::string &s) { g_last_error = s; }
+bool pairs_enabled() {
+    static const bool on = [] { const char *e = getenv("EW_DISABLE_PAIRS"); return !(e && e[0] == '1'); }();
+    return on;
+}
 bool pdl_enabled(int kind) {
     static const bool on = [] { const char *e = getenv("EW_DISABLE_PDL"); return !(e && e[0] == '1'); }();
     static const int mask = [] { const char *e = getenv("EW_PDL_MASK"); return e ? atoi(e) : 31; }();
@@ -539,6 +543,7 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     if (make_tensor_map(p, &map_x, x, 2, dx, box)) return EW_ERR_CUDA;
     CUtensorMap map_x_big = map_x;
     p->token_tile = pick_token_tile(p, B);
+    p->use_pairs = p->token_tile == 256 && pairs_enabled();
     if (p->token_tile >= 128) {
         uint32_t bbox[2] = {64, (uint32_t)p->token_tile};
         if (make_tensor_map(p, &map_x_big, x, 2, dx, bbox)) return EW_ERR_CUDA;

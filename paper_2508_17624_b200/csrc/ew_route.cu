@@ -214,7 +214,17 @@ __global__ void __launch_bounds__(256) permute_kernel(const uint4 *x, const int3
             const int hv = H >> 3;
             const uint4 *src = x + (size_t)(q / k) * hv;
             uint4 *dst = xp + (size_t)dest * hv;
-            for (int v = lane; v < hv; v += 32) dst[v] = src[v];
+            // eight 16-byte loads in flight per lane, then the stores (the pointers are not __restrict__, so the
+            // compiler would otherwise serialise every load behind the previous store)
+            for (int v0 = 0; v0 < hv; v0 += 256) {
+                uint4 r[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (v0 + u * 32 + lane < hv) r[u] = src[v0 + u * 32 + lane];
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (v0 + u * 32 + lane < hv) dst[v0 + u * 32 + lane] = r[u];
+            }
         }
         return;
     }
@@ -336,7 +346,10 @@ int pick_token_tile(const ew_pool *p, int B) {
 
 int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
-    const int R1 = (c.inter + 127) / 128, R2 = (c.hidden + 127) / 128;
+    // weight tiles per group: 128-row tiles, or 256-row tile pairs where the CTA-pair kernel runs the items
+    const int R1 = (c.inter + 127) / 128;                        // GEMM-1 always runs on the one-CTA kernel
+    const int tile_rows2 = p->use_pairs ? 256 : 128;
+    const int R2 = (c.hidden + tile_rows2 - 1) / tile_rows2;
     const long long pairs = (long long)B * c.top_k;
     const int grid = (int)((pairs + 7) / 8) + kPlanners;
     const size_t smem = ((size_t)(p->P + 1) + 4 * (size_t)(p->P + c.num_shared + 1) + p->P) * 4;

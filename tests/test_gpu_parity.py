@@ -534,3 +534,14 @@ def test_host_buffer_pipeline():
             oh.zero_()
     assert pool.last_device_error() == 0
     pool.destroy()
+
+
+def test_token_tile_of_128_rows():
+    """640 tokens on the decode-shaped layer give ~60 rows per expert: the 128-row token tile (the one size the
+    five workloads do not reach) with its double-buffered accumulators and 128-row activation boxes."""
+    cfg = wl.CONFIGS["c1"]
+    sample = np.sort(np.random.default_rng(6).choice(640, size=96, replace=False))
+    res = run_layer(cfg, n_tokens=640, sample=sample)
+    counts = np.bincount(res["slots"].reshape(-1), minlength=cfg.num_slots)
+    assert 64 < counts[:cfg.num_experts].max() <= 128
+    assert res["flips"] <= 6

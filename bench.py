@@ -269,7 +269,7 @@ def run_cuda(args):
             "ms_per_step_with_kernel_events": ms_plain / args.steps,
         }
         if not args.no_cpu_baseline and not args.minimal and world == 1:
-            result["cpu_baseline"] = cpu_baseline(cfg, budget_s=12.0)
+            result["cpu_baseline"] = cpu_baseline(cfg, budget_s=24.0)
     pool.destroy()
     if world > 1:
         dist.barrier()

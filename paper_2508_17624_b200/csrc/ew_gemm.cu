@@ -486,7 +486,7 @@ int launch_gemm2(ew_pool *p, int layer, int, cudaStream_t st) {
     const int K = p->cfg.inter, H = p->cfg.hidden;
     const Workspace &w = p->ws;
     const CUtensorMap &a = p->map_act;
-    switch (p->token_tile) {
+    switch (p->token_tile2) {
         case 32: return launch_one<32, false>(p, L.map_w2, a, a, a, a, w.items2, w.n_items + 1, K, H, w.y, st);
         case 64: return launch_one<64, false>(p, L.map_w2, a, a, a, a, w.items2, w.n_items + 1, K, H, w.y, st);
         case 128: return launch_one<128, false>(p, L.map_w2, a, a, p->map_act_big[0], a, w.items2, w.n_items + 1, K, H, w.y, st);

@@ -60,7 +60,8 @@ struct LayerState {
 struct ew_pool {
     ew_config_t cfg;
     int P = 0;                      // M + N * E_max
-    int token_tile = 32;            // NT: token rows per GEMM work item
+    int token_tile = 32;            // NT: token rows per GEMM-1 work item
+    int token_tile2 = 32;           // and per GEMM-2 work item
     bool use_pairs = false;         // NT = 256: GEMM-2's work items are processed by CTA pairs (cta_group::2)
     ew::PageBackend *be = nullptr;
     ew::PagePool pages;

@@ -5,6 +5,8 @@
 //   combine_kernel   weighted un-permute and sum, one rounding to bf16 (Section 2.1)
 #include <cuda_bf16.h>
 
+#include <cstdlib>
+
 #include "ew_internal.h"
 #include "ew_tc.cuh"
 
@@ -189,7 +191,7 @@ constexpr int kPlanners = 8;
 
 __global__ void __launch_bounds__(256) permute_kernel(const uint4 *x, const int32_t *slot_ids,
                                                       const int32_t *rank, const int32_t *counts,
-                                                      int B, int k, int H, int P, int S, int NT, int R1, int R2,
+                                                      int B, int k, int H, int P, int S, int NT1, int NT2, int R1, int R2,
                                                       int32_t *offsets, int32_t *inv,
                                                       uint4 *xp, GemmItem *items1,
                                                       GemmItem *items2, int32_t *n_items) {
@@ -240,33 +242,38 @@ __global__ void __launch_bounds__(256) permute_kernel(const uint4 *x, const int3
     int32_t *nblk = blk + G + 1;            // [G] token blocks of fat groups (0 for thin ones)
     int32_t *blk_t = nblk + G;              // [G + 1] scan of the thin groups' token blocks
     int32_t *nblk_t = blk_t + G + 1;        // [G]
-    for (int g = threadIdx.x; g < G; g += 256) {
-        const int rows = g < S ? B : cnt_s[g - S];
-        const int nb = (rows + NT - 1) / NT;
-        const bool thin = rows <= kThinRows;
-        nblk[g] = thin ? 0 : nb;
-        nblk_t[g] = thin ? nb : 0;
-    }
-    __syncthreads();
-    block_exclusive_scan(nblk, blk, G, warp_sums);
-    block_exclusive_scan(nblk_t, blk_t, G, warp_sums);
-    const int fat_blocks = blk[G], thin_blocks = blk_t[G];
-    if (blockIdx.x == 0 && threadIdx.x == 0) { n_items[0] = (fat_blocks + thin_blocks) * R1; n_items[1] = (fat_blocks + thin_blocks) * R2; }
-    for (int g = warp + 8 * blockIdx.x; g < G; g += 8 * kPlanners) {
-        const bool thin = nblk_t[g] > 0;
-        const int nb = thin ? nblk_t[g] : nblk[g];
-        if (nb == 0) continue;
-        const bool shared = g < S;
-        const int rows = shared ? B : cnt_s[g - S];
-        const int slot = shared ? P + g : g - S;
-        const int in0 = shared ? 0 : off[g - S];
-        const int out0 = shared ? g * B : S * B + off[g - S];
-        for (int pass = 0; pass < 2; ++pass) {
-            const int R = pass ? R2 : R1;
-            const long long n_fat = (long long)fat_blocks * R, n_thin = (long long)thin_blocks * R;
+    // GEMM-1 and GEMM-2 may use different token tiles (NT1, NT2): each pass has its own block counts and scans
+    for (int pass = 0; pass < 2; ++pass) {
+        const int NT = pass ? NT2 : NT1;
+        const int R = pass ? R2 : R1;
+        if (pass == 0 || NT2 != NT1) {                    // same tile in both GEMMs (decode): one set of scans serves both
+            __syncthreads();                              // the previous pass has finished reading the scan arrays
+            for (int g = threadIdx.x; g < G; g += 256) {
+                const int rows = g < S ? B : cnt_s[g - S];
+                const int nb = (rows + NT - 1) / NT;
+                const bool thin = rows <= kThinRows;
+                nblk[g] = thin ? 0 : nb;
+                nblk_t[g] = thin ? nb : 0;
+            }
+            __syncthreads();
+            block_exclusive_scan(nblk, blk, G, warp_sums);
+            block_exclusive_scan(nblk_t, blk_t, G, warp_sums);
+        }
+        const int fat_blocks = blk[G], thin_blocks = blk_t[G];
+        if (blockIdx.x == 0 && threadIdx.x == 0) n_items[pass] = (fat_blocks + thin_blocks) * R;
+        const long long n_fat = (long long)fat_blocks * R, n_thin = (long long)thin_blocks * R;
+        const bool small = (n_fat + 1) * (n_thin + 1) < (1ll << 31);
+        GemmItem *dst = pass ? items2 : items1;
+        for (int g = warp + 8 * blockIdx.x; g < G; g += 8 * kPlanners) {
+            const bool thin = nblk_t[g] > 0;
+            const int nb = thin ? nblk_t[g] : nblk[g];
+            if (nb == 0) continue;
+            const bool shared = g < S;
+            const int rows = shared ? B : cnt_s[g - S];
+            const int slot = shared ? P + g : g - S;
+            const int in0 = shared ? 0 : off[g - S];
+            const int out0 = shared ? g * B : S * B + off[g - S];
             const long long first = (long long)(thin ? blk_t[g] : blk[g]) * R;    // index inside the group's own class
-            const bool small = (n_fat + 1) * (n_thin + 1) < (1ll << 31);
-            GemmItem *dst = pass ? items2 : items1;
             for (int i = lane; i < nb * R; i += 32) {
                 const int tile = i / nb, c = i % nb;
                 GemmItem it;
@@ -339,6 +346,8 @@ __global__ void __launch_bounds__(256) combine_kernel(const float4 *y, const int
 
 // Token rows per GEMM work item: the smallest tile that holds ~1.5x the mean rows per routed expert.
 int pick_token_tile(const ew_pool *p, int B) {
+    static const int forced = [] { const char *e = getenv("EW_FORCE_NT"); return e ? atoi(e) : 0; }();
+    if (forced == 32 || forced == 64 || forced == 128 || forced == 256) return forced;   // debugging / tuning aid
     const double mean = (double)B * p->cfg.top_k / p->cfg.num_experts;
     const double want = mean * 1.5;
     return want <= 32 ? 32 : want <= 64 ? 64 : want <= 128 ? 128 : 256;
@@ -354,7 +363,7 @@ int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st) {
     const int grid = (int)((pairs + 7) / 8) + kPlanners;
     const size_t smem = ((size_t)(p->P + 1) + 4 * (size_t)(p->P + c.num_shared + 1) + p->P) * 4;
     return launch_pdl(1, permute_kernel, dim3(grid), dim3(256), smem, st, (const uint4 *)x, p->ws.slot_ids, p->ws.rank,
-                      p->ws.counts, B, c.top_k, c.hidden, p->P, c.num_shared, p->token_tile, R1, R2, p->ws.offsets, p->ws.inv,
+                      p->ws.counts, B, c.top_k, c.hidden, p->P, c.num_shared, p->token_tile, p->token_tile2, R1, R2, p->ws.offsets, p->ws.inv,
                       (uint4 *)p->ws.xp, p->ws.items1, p->ws.items2, p->ws.n_items);
 }
 

@@ -37,13 +37,14 @@ WORKLOAD = WORKLOADS["c1"]
 
 
 def load_peaks():
-    """-> (HBM GB/s, bf16 TFLOP/s burst, kind)"""
+    """-> (HBM GB/s, bf16 TFLOP/s burst, bf16 TFLOP/s sustained under the power cap, kind)"""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), "measured"
-    return 6650.0, 1590.0, "fallback"
+        return (float(d["hbm_gbs"]), float(d["bf16_tflops"]),
+                float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "measured")
+    return 6650.0, 1590.0, 1400.0, "fallback"
 
 
 class ClockSampler(threading.Thread):
@@ -228,7 +229,7 @@ def run_cuda(args):
 
     result = None
     if rank == 0:
-        peak, peak_tf, peak_kind = load_peaks()
+        peak, peak_tf, peak_tf_sustained, peak_kind = load_peaks()
         g1_ms = kern_ms["gemm1"] / max(n_prof, 1)
         achieved = bytes_gemm1 / (g1_ms * 1e-3) / 1e9
         flops_gemm1 = 2.0 * rows_act * 2 * cfg.inter * H
@@ -239,7 +240,10 @@ def run_cuda(args):
                     "achieved": flops_gemm1 / (g1_ms * 1e-3) / 1e12, "peak": peak_tf, "unit": "TFLOP/s",
                     "frac": flops_gemm1 / (g1_ms * 1e-3) / 1e12 / peak_tf, "of": peak_kind + " (bf16 burst)",
                     "traffic": None, "algorithmic_flops": flops_gemm1, "avg_launch_ms": g1_ms,
-                    "hbm_gbs": achieved}
+                    "hbm_gbs": achieved,
+                    # the timed loop runs for seconds under the power cap: the sustained cuBLAS figure beside it
+                    "peak_sustained": peak_tf_sustained,
+                    "frac_of_sustained": flops_gemm1 / (g1_ms * 1e-3) / 1e12 / peak_tf_sustained}
         else:
             roof = {"bound": "hbm", "kernel": "grouped_gemm_kernel<GLU> (GEMM-1 + SwiGLU)",
                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -295,7 +299,7 @@ def run_reroute(args):
                         max_tokens=8)
     z = np.zeros((M, 64, 64), np.uint16)
     pool.load_base(0, np.zeros((M, 64), np.uint16), z, z, z)
-    peak, _, peak_kind = load_peaks()
+    peak, _, _, peak_kind = load_peaks()
     lines = []
 
     def measure(B, iters):

@@ -15,7 +15,11 @@
 //   GEMM-2 (GLU = false): y[row, o]   = Wdown[slot][o,:] . act_row                                  -> fp32
 //
 // One persistent CTA per SM walks the device-built item list.  Warp 0 lane 0 issues TMA loads into a
-// ring of shared-memory stages, warp 1 lane 0 issues tcgen05.mma, warps 2..5 drain TMEM.  Every
+// ring of shared-memory stages, warp 1 lane 0 issues tcgen05.mma, warps 2..5 drain TMEM.  In gather
+// mode (GEMM-1 at prefill) four more warps fetch the token operand: each thread copies its row of x,
+// found through the row -> token table of the permute step, into the 128-byte-swizzled stage with
+// 16-byte cp.async, so no permuted copy of x exists in memory (Section 2.1's "permute" folded into
+// the GEMM's operand load).  Every
 // barrier wait is bounded in time: on expiry the CTA raises bit 1 of the device error word, stops
 // issuing work, lets its copies in flight land, frees its TMEM and returns.
 #include <cuda_bf16.h>
@@ -28,6 +32,7 @@ namespace {
 using namespace tc;
 
 constexpr int kThreads = 192;
+constexpr int kGatherThreads = 128;  // gather mode: one more warpgroup, one thread per token row of the block
 constexpr int kTileRows = 128;      // weight rows per tile = MMA M
 constexpr int kATileBytes = kTileRows * kBlockK * 2;   // 16 KiB
 constexpr int kSmemBudget = 227 * 1024 - 2048;
@@ -46,13 +51,27 @@ struct Cfg {
 };
 
 // ------------------------------------------------------------------------------------------- kernel
-template <int NT, bool GLU>
-__global__ void __launch_bounds__(kThreads, 1)
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+// arrives on the barrier (whose expected count already includes this arrival) once all cp.async copies issued by
+// this thread so far have landed
+__device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+// orders shared-memory writes made through the generic proxy (observed through a barrier) before the tensor
+// core's reads of shared memory
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+template <int NT, bool GLU, bool GATHER = false>
+__global__ void __launch_bounds__(GATHER ? kThreads + kGatherThreads : kThreads, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
                     const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_a_big,
                     const __grid_constant__ CUtensorMap map_x_big, const GemmItem *items,
                     const int32_t *n_items_ptr, int K, int out_rows_per_slot, void *out,
-                    int *err) {
+                    int *err, const uint8_t *x_rows, const int32_t *src_tok) {
+    static_assert(!GATHER || (GLU && NT == kGatherThreads), "gather mode: GEMM-1, one gather thread per token row");
     using C = Cfg<NT, GLU>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -69,7 +88,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::kStages; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_full + 8 * s, GATHER ? 1 + kGatherThreads : 1);        // the TMA thread, and each gather thread
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -79,7 +98,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_map(&map_w);
-        prefetch_map(&map_a);
+        if (!GATHER) prefetch_map(&map_a);
         if (GLU) prefetch_map(&map_x);
     }
     if (warp == 1) {   // TMEM allocation is a whole-warp operation
@@ -110,7 +129,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
                 // thin items fetch their rows in 32-row boxes; fat ones (prefill) with one NT-row box per stage
                 const bool big = NT >= 128 && it.rows > 2 * kChunkRows;
                 const CUtensorMap *amap = (GLU && it.from_x) ? (big ? &map_x_big : &map_x) : (big ? &map_a_big : &map_a);
-                const uint32_t b_bytes = big ? NT * kBlockK * 2 : nchunk * kChunkBytes;
+                // gather mode: only the shared experts' rows (contiguous in x) still come by TMA
+                const bool tma_tokens = !GATHER || it.from_x;
+                const uint32_t b_bytes = !tma_tokens ? 0 : big ? NT * kBlockK * 2 : nchunk * kChunkBytes;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1, abort_flag, err))) break;
                     const uint32_t sa = smem_base + stage * C::kStageBytes;
@@ -123,7 +144,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
                         tma_load_3d(sa, &map_w, kb * kBlockK, it.tile * kTileRows, it.slot, full);
                     }
                     const uint32_t sb = sa + (GLU ? 2 : 1) * kATileBytes;
-                    if (big) {
+                    if (!tma_tokens) {
+                        // the token operand of this stage is written by the gather warps
+                    } else if (big) {
                         tma_load_2d(sb, amap, kb * kBlockK, it.in_row, full);
                     } else {
                         for (int c = 0; c < nchunk; ++c)
@@ -147,6 +170,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
                 const uint32_t d0 = tmem_base + acc * C::kAccCols;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!(ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, err))) break;
+                    if (GATHER) fence_proxy_async_smem();           // the token rows were written by cp.async, not by TMA
                     tc_fence_after();
                     const uint32_t sa = smem_base + stage * C::kStageBytes;
                     const uint64_t a0 = smem_desc_sw128(sa);
@@ -166,6 +190,48 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
                 if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1; }
             }
         }
+    } else if (GATHER && warp >= kThreads / 32) {
+        // ------------------------------------------------------------------ token gather (warps 6..9)
+        // Eight consecutive threads copy one 128-byte row segment (one k-block of one token row of x) as eight
+        // 16-byte chunks, so a warp instruction reads four whole 128-byte lines; thread t serves chunk t mod 8 of
+        // rows t/8 + 16 i (i = 0..7).  Chunk c of row r lands where the 128-byte swizzle puts it: at chunk position
+        // c ^ (r mod 8) inside the row.  Each thread's arrival on the stage's barrier fires when its copies have landed
+        // (cp.async.mbarrier.arrive.noinc), so the threads never block on their own copies; the MMA thread fences
+        // the generic-proxy writes against the tensor core's reads after its wait.
+        const int t = (int)threadIdx.x - kThreads;
+        const int chunk = t & 7, r0 = t >> 3;
+        constexpr int kRowsPerThread = NT / (kGatherThreads / 8);
+        uint32_t dst_off[kRowsPerThread];
+#pragma unroll
+        for (int i = 0; i < kRowsPerThread; ++i) {
+            const int r = r0 + i * (kGatherThreads / 8);
+            dst_off[i] = (uint32_t)((GLU ? 2 : 1) * kATileBytes + r * 128 + ((chunk ^ (r & 7)) << 4));
+        }
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
+            const GemmItem it = items[w];
+            const int n = ((it.rows + 15) >> 4) << 4;
+            const uint8_t *src[kRowsPerThread];                  // rows beyond n are not read by the MMA: not fetched
+#pragma unroll
+            for (int i = 0; i < kRowsPerThread; ++i) {
+                const int r = r0 + i * (kGatherThreads / 8);
+                const int rr = min(r, it.rows - 1);               // rows it.rows..n-1 repeat the last row; never stored
+                const int tok = it.from_x ? 0 : src_tok[it.in_row + rr];   // shared experts: the TMA thread loads x rows
+                src[i] = x_rows + (size_t)tok * K * 2 + chunk * 16;
+            }
+            for (int kb = 0; kb < num_kb; ++kb) {
+                if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1, abort_flag, err))) break;
+                const uint32_t d = smem_base + stage * C::kStageBytes;
+#pragma unroll
+                for (int i = 0; i < kRowsPerThread; ++i)
+                    if (!it.from_x && r0 + i * (kGatherThreads / 8) < n)
+                        cp_async16(d + dst_off[i], src[i] + (size_t)kb * (kBlockK * 2));
+                cp_async_arrive_noinc(bar_full + 8 * stage);      // fires when this thread's copies have landed
+                if (++stage == C::kStages) { stage = 0; phase ^= 1; }
+            }
+        }
+        cp_async_wait_all();                                      // nothing of this thread stays in flight at exit
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int lg = warp & 3;                        // TMEM lane group this warp may read
@@ -441,18 +507,19 @@ int launch_pair(ew_pool *p, const CUtensorMap &mw, const CUtensorMap &ma, const 
     return (int)cudaLaunchKernelEx(&cfg, grouped_gemm_pair_kernel<GLU>, mw, ma, mx, items, n_items, K, out_rows, out, p->ws.err);
 }
 
-template <int NT, bool GLU>
+template <int NT, bool GLU, bool GATHER = false>
 int launch_one(ew_pool *p, const CUtensorMap &mw, const CUtensorMap &ma, const CUtensorMap &mx, const CUtensorMap &mab,
                const CUtensorMap &mxb, const GemmItem *items, const int32_t *n_items, int K, int out_rows, void *out,
-               cudaStream_t st) {
+               cudaStream_t st, const void *x_rows = nullptr) {
     using C = Cfg<NT, GLU>;
-    return launch_pdl(GLU ? 2 : 3, grouped_gemm_kernel<NT, GLU>, dim3(p->sm_count), dim3(kThreads), C::kSmemBytes, st, mw, ma, mx, mab,
-                      mxb, items, n_items, K, out_rows, out, p->ws.err);
+    return launch_pdl(GLU ? 2 : 3, grouped_gemm_kernel<NT, GLU, GATHER>, dim3(p->sm_count),
+                      dim3(GATHER ? kThreads + kGatherThreads : kThreads), C::kSmemBytes, st, mw, ma, mx, mab, mxb, items, n_items,
+                      K, out_rows, out, p->ws.err, (const uint8_t *)x_rows, (const int32_t *)p->ws.src_tok);
 }
 
-template <int NT, bool GLU>
+template <int NT, bool GLU, bool GATHER = false>
 int setup_one() {
-    return (int)cudaFuncSetAttribute(grouped_gemm_kernel<NT, GLU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return (int)cudaFuncSetAttribute(grouped_gemm_kernel<NT, GLU, GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      Cfg<NT, GLU>::kSmemBytes);
 }
 
@@ -461,6 +528,7 @@ int setup_one() {
 int gemm_setup(ew_pool *) {
     int rc = 0;
     rc |= setup_one<32, true>() | setup_one<64, true>() | setup_one<128, true>() | setup_one<256, true>();
+    rc |= setup_one<128, true, true>();
     rc |= setup_one<32, false>() | setup_one<64, false>() | setup_one<128, false>() | setup_one<256, false>();
     rc |= (int)cudaFuncSetAttribute(grouped_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<true>::kSmemBytes);
     rc |= (int)cudaFuncSetAttribute(grouped_gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<false>::kSmemBytes);
@@ -468,10 +536,14 @@ int gemm_setup(ew_pool *) {
     return rc;
 }
 
-int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, const CUtensorMap &map_x_big, int, cudaStream_t st) {
+int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, const CUtensorMap &map_x_big, const void *x, int,
+                 cudaStream_t st) {
     const LayerState &L = p->layers[layer];
     const int K = p->cfg.hidden, I = p->cfg.inter;
     const Workspace &w = p->ws;
+    if (p->gather)
+        return launch_one<128, true, true>(p, L.map_w13, p->map_xp, map_x, p->map_xp_big[0], map_x_big, w.items1, w.n_items, K, I,
+                                           w.act, st, x);
     switch (p->token_tile) {
         case 32: return launch_one<32, true>(p, L.map_w13, p->map_xp, map_x, p->map_xp, map_x, w.items1, w.n_items, K, I, w.act, st);
         case 64: return launch_one<64, true>(p, L.map_w13, p->map_xp, map_x, p->map_xp, map_x, w.items1, w.n_items, K, I, w.act, st);

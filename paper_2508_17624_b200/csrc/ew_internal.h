@@ -37,6 +37,7 @@ struct Workspace {
     GemmItem *items2 = nullptr;
     int32_t max_items1 = 0, max_items2 = 0;
     void *xp = nullptr;            // [Bmax*k, H] bf16 permuted activations
+    int32_t *src_tok = nullptr;    // [Bmax*k] token of each slot-contiguous row (gather mode: GEMM-1 fetches x rows itself)
     void *act = nullptr;           // [S*Bmax + Bmax*k, I] bf16 SwiGLU output
     float *y = nullptr;            // [S*Bmax + Bmax*k, H] fp32 expert outputs
     int32_t *err = nullptr;        // device error word
@@ -63,6 +64,7 @@ struct ew_pool {
     int token_tile = 32;            // NT: token rows per GEMM-1 work item
     int token_tile2 = 32;           // and per GEMM-2 work item
     bool use_pairs = false;         // NT = 256: GEMM-2's work items are processed by CTA pairs (cta_group::2)
+    bool gather = false;            // GEMM-1 gathers its token rows from x; no permuted copy of x is written
     ew::PageBackend *be = nullptr;
     ew::PagePool pages;
     std::vector<ew::LayerState> layers;
@@ -98,6 +100,8 @@ void set_last_error(const std::string &s);
 bool pdl_enabled(int kind = -1);
 // EW_DISABLE_PAIRS=1 keeps prefill-sized token tiles on the one-CTA kernel.
 bool pairs_enabled();
+// EW_DISABLE_GATHER=1 keeps the permuted copy of x at prefill (GEMM-1 then reads it by TMA), for debugging.
+bool gather_enabled();
 
 // Launch with programmatic stream serialization (the kernel calls pdl_wait() before it reads its
 // predecessor's output).
@@ -127,7 +131,8 @@ int make_atom_map(ew_pool *p, CUtensorMap *out, const void *base, int H, int row
 // Kernel launchers (all asynchronous on `st`; return cudaError_t as int).
 int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B, cudaStream_t st);
 int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st);
-int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, const CUtensorMap &map_x_big, int B, cudaStream_t st);
+int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, const CUtensorMap &map_x_big, const void *x, int B,
+                 cudaStream_t st);
 int pick_token_tile(const ew_pool *p, int B);
 int launch_gemm2(ew_pool *p, int layer, int B, cudaStream_t st);
 int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st);

@@ -14,6 +14,10 @@ bool pairs_enabled() {
     static const bool on = [] { const char *e = getenv("EW_DISABLE_PAIRS"); return !(e && e[0] == '1'); }();
     return on;
 }
+bool gather_enabled() {
+    static const bool on = [] { const char *e = getenv("EW_DISABLE_GATHER"); return !(e && e[0] == '1'); }();
+    return on;
+}
 bool pdl_enabled(int kind) {
     static const bool on = [] { const char *e = getenv("EW_DISABLE_PDL"); return !(e && e[0] == '1'); }();
     static const int mask = [] { const char *e = getenv("EW_PDL_MASK"); return e ? atoi(e) : 31; }();
@@ -109,6 +113,7 @@ static ew_status_t alloc_workspace(ew_pool *p) {
         {(void **)&w.rank, Bm * k * 4}, {(void **)&w.inv, Bm * k * 4}, {(void **)&w.counts, P * 4},
         {(void **)&w.offsets, (P + 1) * 4}, {(void **)&w.n_items, 16}, {(void **)&w.items1, rb * r1 * sizeof(GemmItem)},
         {(void **)&w.items2, rb * r2 * sizeof(GemmItem)}, {(void **)&w.xp, (Bm * k + 32) * H * 2},
+        {(void **)&w.src_tok, (Bm * k + 32) * 4},
         {(void **)&w.act, rows * I * 2}, {(void **)&w.y, rows * H * 4}, {(void **)&w.err, 256},
         {(void **)&w.loaded, (size_t)c.max_adapters * 4 + 16},
         {&p->stage_x[0], Bm * H * 2}, {&p->stage_out[0], Bm * H * 2}, {(void **)&p->stage_aid[0], Bm * 4},
@@ -548,6 +553,9 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     p->token_tile2 = pick_token_tile(p, B);
     p->token_tile = p->token_tile2 == 256 ? 128 : p->token_tile2;
     p->use_pairs = p->token_tile2 == 256 && pairs_enabled();
+    // At prefill the permuted copy of x (k rows per token) is not written: the permute kernel only records which token
+    // each slot-contiguous row is, and GEMM-1 gathers those rows of x (which stay in L2) into its token operand.
+    p->gather = p->token_tile == 128 && gather_enabled();
     if (p->token_tile >= 128) {
         uint32_t bbox[2] = {64, (uint32_t)p->token_tile};
         if (make_tensor_map(p, &map_x_big, x, 2, dx, bbox)) return EW_ERR_CUDA;
@@ -577,7 +585,7 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     if (counts) CU_TRY(cudaMemcpyAsync(counts, p->ws.counts, (size_t)p->P * 4, cudaMemcpyDeviceToDevice, st));
     if (inv) CU_TRY(cudaMemcpyAsync(inv, p->ws.inv, nk * 4, cudaMemcpyDeviceToDevice, st));
     if (offsets) CU_TRY(cudaMemcpyAsync(offsets, p->ws.offsets, ((size_t)p->P + 1) * 4, cudaMemcpyDeviceToDevice, st));
-    LAUNCH_TRY(launch_gemm1(p, layer, map_x, map_x_big, B, st));
+    LAUNCH_TRY(launch_gemm1(p, layer, map_x, map_x_big, x, B, st));
     PROF_MARK(3);
     LAUNCH_TRY(launch_gemm2(p, layer, B, st));
     PROF_MARK(4);

@@ -193,7 +193,7 @@ __global__ void __launch_bounds__(256) permute_kernel(const uint4 *x, const int3
                                                       const int32_t *rank, const int32_t *counts,
                                                       int B, int k, int H, int P, int S, int NT1, int NT2, int R1, int R2,
                                                       int32_t *offsets, int32_t *inv,
-                                                      uint4 *xp, GemmItem *items1,
+                                                      uint4 *xp, int32_t *src_tok, GemmItem *items1,
                                                       GemmItem *items2, int32_t *n_items) {
     extern __shared__ int32_t sm[];
     int32_t *off = sm;                 // [P + 1]
@@ -208,6 +208,16 @@ __global__ void __launch_bounds__(256) permute_kernel(const uint4 *x, const int3
     __syncthreads();
     block_exclusive_scan(cnt_s, off, P, warp_sums);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (blockIdx.x >= kPlanners && src_tok) {
+        // gather mode: no copy of x; one thread per (token, j) pair records the pair's row and the row's token
+        const long long q = (long long)(blockIdx.x - kPlanners) * 256 + threadIdx.x;
+        if (q < (long long)B * k) {
+            const int dest = off[slot_ids[q]] + rank[q];
+            inv[q] = dest;
+            src_tok[dest] = (int32_t)(q / k);
+        }
+        return;
+    }
     if (blockIdx.x >= kPlanners) {                       // the first CTAs (dispatched first) are the planners
         const long long q = (long long)(blockIdx.x - kPlanners) * 8 + warp;
         if (q < (long long)B * k) {
@@ -360,11 +370,12 @@ int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st) {
     const int tile_rows2 = p->use_pairs ? 256 : 128;
     const int R2 = (c.hidden + tile_rows2 - 1) / tile_rows2;
     const long long pairs = (long long)B * c.top_k;
-    const int grid = (int)((pairs + 7) / 8) + kPlanners;
+    const int grid = (int)(p->gather ? (pairs + 255) / 256 : (pairs + 7) / 8) + kPlanners;
     const size_t smem = ((size_t)(p->P + 1) + 4 * (size_t)(p->P + c.num_shared + 1) + p->P) * 4;
     return launch_pdl(1, permute_kernel, dim3(grid), dim3(256), smem, st, (const uint4 *)x, p->ws.slot_ids, p->ws.rank,
                       p->ws.counts, B, c.top_k, c.hidden, p->P, c.num_shared, p->token_tile, p->token_tile2, R1, R2, p->ws.offsets, p->ws.inv,
-                      (uint4 *)p->ws.xp, p->ws.items1, p->ws.items2, p->ws.n_items);
+                      (uint4 *)p->ws.xp, p->gather ? p->ws.src_tok : (int32_t *)nullptr, p->ws.items1, p->ws.items2,
+                      p->ws.n_items);
 }
 
 int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st) {

@@ -52,10 +52,12 @@ def table1_shaped_counts(max_e: int, avg_e: float, layers: int, seed: int) -> np
     return e.astype(np.int32)
 
 
-def memory_table1_shapes():
+def memory_table1_shapes(page_bytes: int = 0):
     """Adapter memory, pages on demand vs padding, for Table-1-shaped adapters of the DeepSeek-V2-Lite shape
     (26 layers, 64 experts, 16.5 MiB per expert), on the accounting-only backend (no GPU needed).  The paper's
-    Section 5.4 loads gate-math, then gate-intent, then token-math and reports 40.4 %, 28.9 % and 37.3 % less."""
+    Section 5.4 loads gate-math, then gate-intent, then token-math and reports 40.4 %, 28.9 % and 37.3 % less.
+    `page_bytes` = 0 takes the driver's minimum granularity (2 MiB); larger pages cost rounding at every adapter's
+    two ends (Section 4.2's sub-page sharing removes it between neighbours only)."""
     from . import binding, workloads as wl
     shapes = [("gate-math", 12, 7.04), ("gate-intent", 12, 9.50), ("token-math", 9, 6.12)]
     L, M, e_max = 26, 64, 12
@@ -63,7 +65,8 @@ def memory_table1_shapes():
     pools = {}
     for mode in (0, 1):
         pools[mode] = binding.Pool(device=-1, num_layers=L, hidden=2048, inter=1408, num_experts=M, num_shared=2,
-                                   top_k=6, max_adapters=3, e_max=e_max, max_tokens=16, pool_mode=mode)
+                                   top_k=6, max_adapters=3, e_max=e_max, max_tokens=16, pool_mode=mode,
+                                   page_bytes=page_bytes)
         for l in range(L):
             pools[mode].load_base(l, None, None, None, None, None, None, None)
     base = {m: pools[m].stats()["physical_bytes"] for m in pools}
@@ -82,6 +85,43 @@ def memory_table1_shapes():
     for m in pools:
         pools[m].destroy()
     return out
+
+
+def page_size_sweep(gpu: bool):
+    """Page size of the physical pool (Section 4.2): larger pages mean fewer map/unmap driver calls per adapter
+    (the load latency is mostly those calls) and more rounding at the adapters' ends.  Memory side on the
+    accounting backend (Table-1-shaped adapters), latency side (if `gpu`) on one c1-shaped adapter of 8 experts
+    with its weights in page-locked host memory and no forward in flight."""
+    from . import binding, workloads as wl
+    rows = []
+    for mib in (2, 4, 8, 32):
+        row = {"page_MiB": mib, "table1_saving": [r["saving"] for r in memory_table1_shapes(mib << 20)]}
+        if gpu:
+            import time
+            import torch
+            cfg = wl.CONFIGS["c1"]
+            bank = wl.NoiseBank(cfg.seed)
+            pool = binding.Pool.from_config(cfg, page_bytes=mib << 20)
+            binding.load_model(pool, cfg, bank)
+            tuned = wl.tuned_sets(cfg)
+            ew3 = wl.gen_adapter_layer(cfg, 3, 0, tuned[3][0], bank)
+            src = [torch.from_numpy(a.view(np.int16)).pin_memory().numpy().view(np.uint16)
+                   for a in (ew3.w_gate, ew3.w_up, ew3.w_down)]
+            t_un, t_ld = [], []
+            for _ in range(6):
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                pool.unload_adapter(3)
+                t1 = time.perf_counter()
+                pool.load_adapter(3, np.array([len(tuned[3][0])], np.int32), tuned[3][0], *src)
+                t2 = time.perf_counter()
+                t_un.append((t1 - t0) * 1e3)
+                t_ld.append((t2 - t1) * 1e3)
+            row.update(unload_ms=float(np.median(t_un)), load_ms=float(np.median(t_ld)),
+                       pages_per_adapter=int(-(-ew3.w_gate.nbytes * 3 // (mib << 20))))
+            pool.destroy()
+        rows.append(row)
+    return rows
 
 
 def main():
@@ -131,8 +171,12 @@ def main():
     ew3 = wl.gen_adapter_layer(cfg, 3, 0, tuned[3][0], bank)
     aid_wo3 = torch.where(aid == 3, torch.full_like(aid, -1), aid)
     created0 = pool.stats()["pages_created_total"]
-    t_un, t_ld = [], []
-    for _ in range(5):
+    # the same weights in page-locked host memory: the copy then runs at the host link's speed, and what is left
+    # of the load latency is the page mapping
+    pinned = [torch.from_numpy(a.view(np.int16)).pin_memory().numpy().view(np.uint16) for a in (ew3.w_gate, ew3.w_up, ew3.w_down)]
+    t_un, t_ld, t_ld_pinned = [], [], []
+    for it in range(10):
+        src = pinned if it >= 5 else (ew3.w_gate, ew3.w_up, ew3.w_down)
         for _ in range(20):
             pool.moe_forward(0, x, aid, out)
         t0 = time.perf_counter()
@@ -141,15 +185,18 @@ def main():
         for _ in range(20):
             pool.moe_forward(0, x, aid_wo3, out)
         t2 = time.perf_counter()
-        pool.load_adapter(3, np.array([len(tuned[3][0])], np.int32), tuned[3][0], ew3.w_gate, ew3.w_up, ew3.w_down)
+        pool.load_adapter(3, np.array([len(tuned[3][0])], np.int32), tuned[3][0], *src)
         t3 = time.perf_counter()
         t_un.append((t1 - t0) * 1e3)
-        t_ld.append((t3 - t2) * 1e3)
+        (t_ld_pinned if it >= 5 else t_ld).append((t3 - t2) * 1e3)
     torch.cuda.synchronize()
     res["churn"] = {"unload_ms_median": float(np.median(t_un)), "load_ms_median": float(np.median(t_ld)),
+                    "load_ms_median_pinned_source": float(np.median(t_ld_pinned)),
                     "adapter_bytes": int(ew3.w_gate.nbytes * 3), "forwards_in_flight": 20,
                     "pages_created_during_churn": pool.stats()["pages_created_total"] - created0,
                     "device_error": pool.last_device_error()}
+
+    res["page_size_sweep"] = page_size_sweep(gpu=True)
 
     # ---- batch-size sweep on a pool sized for 8192 tokens
     big = binding.Pool.from_config(cfg, max_tokens=8192)

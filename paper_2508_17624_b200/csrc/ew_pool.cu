@@ -291,15 +291,24 @@ extern "C" ew_status_t ew_pool_trim(ew_pool_t *p) {
 
 // Copy e experts' gate and up blocks into slots [first, first+e) of the fused tensor, and the down
 // blocks into the down tensor.  Source layout: [e, I, H], [e, I, H], [e, H, I].
-static ew_status_t copy_experts(ew_pool *p, LayerState &L, size_t first, size_t e, const void *g, const void *u,
-                                const void *d) {
+static ew_status_t copy_gate_up(ew_pool *p, LayerState &L, size_t first, size_t e, const void *g, const void *u) {
     if (e == 0 || p->cfg.device < 0) return EW_OK;
     size_t blk = (size_t)p->cfg.inter * p->cfg.hidden * 2;
     char *dst13 = (char *)L.w13.slot_addr(first);
     CU_TRY(cudaMemcpy2DAsync(dst13, 2 * blk, g, blk, blk, e, cudaMemcpyHostToDevice, p->copy_stream));
     CU_TRY(cudaMemcpy2DAsync(dst13 + blk, 2 * blk, u, blk, blk, e, cudaMemcpyHostToDevice, p->copy_stream));
+    return EW_OK;
+}
+static ew_status_t copy_down(ew_pool *p, LayerState &L, size_t first, size_t e, const void *d) {
+    if (e == 0 || p->cfg.device < 0) return EW_OK;
+    size_t blk = (size_t)p->cfg.inter * p->cfg.hidden * 2;
     CU_TRY(cudaMemcpyAsync((void *)L.w2.slot_addr(first), d, blk * e, cudaMemcpyHostToDevice, p->copy_stream));
     return EW_OK;
+}
+static ew_status_t copy_experts(ew_pool *p, LayerState &L, size_t first, size_t e, const void *g, const void *u,
+                                const void *d) {
+    ew_status_t st = copy_gate_up(p, L, first, e, g, u);
+    return st == EW_OK ? copy_down(p, L, first, e, d) : st;
 }
 
 extern "C" ew_status_t ew_load_base(ew_pool_t *p, int32_t layer, const void *router_w, const void *w_gate,
@@ -365,35 +374,28 @@ extern "C" ew_status_t ew_load_adapter(ew_pool_t *p, int32_t a, const int32_t *c
     if (gpu) CU_TRY(cudaSetDevice(c.device));
     size_t delta = (size_t)M + (size_t)a * c.e_max;     // Delta_i = M + i * E_max
     ew_status_t st = EW_OK;
-    int done = 0;                                       // layers fully mapped so far (for rollback)
-    if (c.pool_mode == 0)
-        for (; done < L; ++done) {
-            LayerState &Ls = p->layers[done];
-            if ((st = be_status(p, Ls.w13.map_slots(delta, counts[done]))) != EW_OK) break;
-            if ((st = be_status(p, Ls.w2.map_slots(delta, counts[done]))) != EW_OK) {
-                Ls.w13.unmap_slots(delta, counts[done]);
-                break;
-            }
-        }
+    // Layer by layer, tensor by tensor: map the slots' pages (driver calls on this thread, ~0.1 ms per page), then
+    // queue the copy into them, so that the copies run while the next pages are being mapped.
+    int done13 = 0, done2 = 0;                          // layers whose gate/up and down slots are mapped (for rollback)
+    const bool vmm = c.pool_mode == 0;
     size_t blk = (size_t)c.inter * c.hidden * 2;
-    if (st == EW_OK && gpu) {
-        size_t q = 0;
-        for (int l = 0; l < L && st == EW_OK; ++l) {
-            st = copy_experts(p, p->layers[l], delta, counts[l], (const char *)w_gate + q * blk,
-                              (const char *)w_up + q * blk, (const char *)w_down + q * blk);
-            q += counts[l];
-        }
-        if (st == EW_OK && cudaStreamSynchronize(p->copy_stream) != cudaSuccess) {
-            set_last_error("ew_load_adapter: weight copy failed");
-            st = EW_ERR_CUDA;
-        }
+    size_t q = 0;
+    for (int l = 0; l < L && st == EW_OK; ++l) {
+        LayerState &Ls = p->layers[l];
+        if (vmm && (st = be_status(p, Ls.w13.map_slots(delta, counts[l]))) == EW_OK) ++done13;
+        if (st == EW_OK && gpu)
+            st = copy_gate_up(p, Ls, delta, counts[l], (const char *)w_gate + q * blk, (const char *)w_up + q * blk);
+        if (st == EW_OK && vmm && (st = be_status(p, Ls.w2.map_slots(delta, counts[l]))) == EW_OK) ++done2;
+        if (st == EW_OK && gpu) st = copy_down(p, Ls, delta, counts[l], (const char *)w_down + q * blk);
+        q += counts[l];
+    }
+    if (gpu && cudaStreamSynchronize(p->copy_stream) != cudaSuccess && st == EW_OK) {   // also before any rollback
+        set_last_error("ew_load_adapter: weight copy failed");
+        st = EW_ERR_CUDA;
     }
     if (st != EW_OK) {
-        if (c.pool_mode == 0)
-            for (int l = 0; l < done; ++l) {
-                p->layers[l].w13.unmap_slots(delta, counts[l]);
-                p->layers[l].w2.unmap_slots(delta, counts[l]);
-            }
+        for (int l = 0; l < done13; ++l) p->layers[l].w13.unmap_slots(delta, counts[l]);
+        for (int l = 0; l < done2; ++l) p->layers[l].w2.unmap_slots(delta, counts[l]);
         return st;
     }
     // publish: Pi[l][a][j] = Delta + rank of j, only after the weights are in place

@@ -85,17 +85,15 @@ struct CudaBackend : PageBackend {
     }
     int map(uint64_t va, size_t bytes, uint64_t handle) override {
         CUresult r = pMap((CUdeviceptr)va, bytes, 0, (CUmemGenericAllocationHandle)handle, 0);
-        if (r != CUDA_SUCCESS) return fail("cuMemMap", r);
+        return r == CUDA_SUCCESS ? 0 : fail("cuMemMap", r);
+    }
+    int set_access(uint64_t va, size_t bytes) override {
         CUmemAccessDesc a = {};
         a.location.type = CU_MEM_LOCATION_TYPE_DEVICE;
         a.location.id = device;
         a.flags = CU_MEM_ACCESS_FLAGS_PROT_READWRITE;
-        r = pSetAccess((CUdeviceptr)va, bytes, &a, 1);
-        if (r != CUDA_SUCCESS) {
-            pUnmap((CUdeviceptr)va, bytes);
-            return fail("cuMemSetAccess", r);
-        }
-        return 0;
+        CUresult r = pSetAccess((CUdeviceptr)va, bytes, &a, 1);
+        return r == CUDA_SUCCESS ? 0 : fail("cuMemSetAccess", r);
     }
     int unmap(uint64_t va, size_t bytes) override {
         CUresult r = pUnmap((CUdeviceptr)va, bytes);
@@ -126,15 +124,28 @@ struct MockBackend : PageBackend {
         mapped.push_back({va, bytes});
         return 0;
     }
-    int unmap(uint64_t va, size_t bytes) override {
-        for (size_t i = 0; i < mapped.size(); ++i)
-            if (mapped[i].first == va && mapped[i].second == bytes) {
+    int set_access(uint64_t va, size_t bytes) override {   // the range must be covered by mapped pages, without a hole
+        size_t covered = 0;
+        for (auto &m : mapped)
+            if (m.first >= va && m.first + m.second <= va + bytes) covered += m.second;
+            else if (va < m.first + m.second && m.first < va + bytes) { last_error = "mock: set_access cuts a mapping"; return 6; }
+        if (covered != bytes) { last_error = "mock: set_access over an unmapped hole"; return 6; }
+        return 0;
+    }
+    int unmap(uint64_t va, size_t bytes) override {        // whole mappings only, and no hole in the range
+        size_t covered = 0;
+        for (auto &m : mapped)
+            if (m.first >= va && m.first + m.second <= va + bytes) covered += m.second;
+            else if (va < m.first + m.second && m.first < va + bytes) { last_error = "mock: unmap cuts a mapping"; return 6; }
+        if (covered != bytes) { last_error = "mock: unmap of an unmapped range"; return 6; }
+        for (size_t i = 0; i < mapped.size();)
+            if (mapped[i].first >= va && mapped[i].first + mapped[i].second <= va + bytes) {
                 mapped[i] = mapped.back();
                 mapped.pop_back();
-                return 0;
+            } else {
+                ++i;
             }
-        last_error = "mock: unmap of an unmapped range";
-        return 6;
+        return 0;
     }
 };
 
@@ -242,8 +253,22 @@ bool VirtualTensor::slot_mapped(size_t slot) const {
     return true;
 }
 
+// Calls f(first_page, n_pages) for every maximal run of consecutive page indices in the ascending list `pages`.
+template <class F>
+static int for_each_run(const std::vector<size_t> &pages, F f) {
+    for (size_t i = 0; i < pages.size();) {
+        size_t j = i + 1;
+        while (j < pages.size() && pages[j] == pages[j - 1] + 1) ++j;
+        int rc = f(pages[i], j - i);
+        if (rc) return rc;
+        i = j;
+    }
+    return 0;
+}
+
 int VirtualTensor::map_slots(size_t first, size_t n) {
     size_t page = pool->page_bytes;
+    std::vector<size_t> fresh;                 // pages mapped by this call, ascending
     for (size_t s = first; s < first + n; ++s) {
         size_t p0 = s * expert_bytes / page, p1 = ((s + 1) * expert_bytes - 1) / page;
         for (size_t p = p0; p <= p1; ++p) {
@@ -262,25 +287,34 @@ int VirtualTensor::map_slots(size_t first, size_t n) {
                 }
                 handle[p] = h;
                 ++pages_mapped;
+                fresh.push_back(p);
             }
             ++refcnt[p];
         }
     }
-    return 0;
+    // access rights once per run of new pages (an adapter's pages are one run, or two around a shared boundary page)
+    int rc = for_each_run(fresh, [&](size_t p, size_t len) { return be->set_access(base + p * page, len * page); });
+    if (rc) unmap_slots(first, n);
+    return rc;
 }
 
 void VirtualTensor::unmap_slots(size_t first, size_t n) {
     size_t page = pool->page_bytes;
+    std::vector<size_t> dead;                  // pages no live expert touches any more, ascending
     for (size_t s = first; s < first + n; ++s) {
         size_t p0 = s * expert_bytes / page, p1 = ((s + 1) * expert_bytes - 1) / page;
         for (size_t p = p0; p <= p1; ++p) {
             if (refcnt[p] == 0) continue;
-            if (--refcnt[p] == 0) {
-                be->unmap(base + p * page, page);
-                pool->give_back(handle[p]);
-                --pages_mapped;
-            }
+            if (--refcnt[p] == 0) dead.push_back(p);
         }
+    }
+    for_each_run(dead, [&](size_t p, size_t len) {
+        be->unmap(base + p * page, len * page);
+        return 0;
+    });
+    for (size_t p : dead) {
+        pool->give_back(handle[p]);
+        --pages_mapped;
     }
 }
 

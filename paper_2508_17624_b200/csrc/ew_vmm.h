@@ -23,8 +23,11 @@ struct PageBackend {
     virtual int free_va(uint64_t va, size_t bytes) = 0;
     virtual int create(size_t bytes, uint64_t *handle) = 0;
     virtual int release(uint64_t handle) = 0;
-    virtual int map(uint64_t va, size_t bytes, uint64_t handle) = 0;   // map + make it read/write
-    virtual int unmap(uint64_t va, size_t bytes) = 0;
+    virtual int map(uint64_t va, size_t bytes, uint64_t handle) = 0;   // map one page; not accessible yet
+    // make a fully mapped range (any number of neighbouring pages) readable and writable: one driver call per run of
+    // pages, because the call's cost hardly depends on the size of the range
+    virtual int set_access(uint64_t va, size_t bytes) = 0;
+    virtual int unmap(uint64_t va, size_t bytes) = 0;                  // a range made of whole mapped pages
     std::string last_error;
 };
 

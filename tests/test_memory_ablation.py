@@ -19,3 +19,15 @@ def test_table1_shaped_counts_have_the_printed_statistics():
     for mx, avg in ((12, 7.04), (13, 4.69), (6, 3.85)):
         e = ablations.table1_shaped_counts(mx, avg, 26, seed=1)
         assert e.max() == mx and e.min() >= 1 and abs(e.mean() - avg) < 0.02
+
+
+def test_larger_pages_save_less():
+    """Rounding happens at the two ends of every adapter's slot range in every layer and tensor (neighbours share
+    their boundary page, Section 4.2), so the saving can only shrink as the page grows, and at the driver's minimum
+    page the rounding is a small part of the adapter's bytes."""
+    build.build()
+    sweep = ablations.page_size_sweep(gpu=False)
+    assert [r["page_MiB"] for r in sweep] == [2, 4, 8, 32]
+    for a, b in zip(sweep, sweep[1:]):
+        assert all(x >= y for x, y in zip(a["table1_saving"], b["table1_saving"])), (a, b)
+    assert sweep[0]["table1_saving"][0] - sweep[1]["table1_saving"][0] < 0.02

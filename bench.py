@@ -25,7 +25,7 @@ sys.path.insert(0, ROOT)
 
 # DRAM bytes (read + write) per launch of the dominant kernel from the committed ncu captures
 # (profiles/c1_decode_grouped_gemm_full.md); reported beside the algorithmic bytes, not used in any ratio.
-NCU_TRAFFIC_BYTES = {"c1": 1.1480e9}
+NCU_TRAFFIC_BYTES = {"c1": 1.1529e9}
 
 METRIC = "adapter-aware MoE layer tokens/s"
 UNIT = "tokens/s"

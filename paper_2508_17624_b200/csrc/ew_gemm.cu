@@ -16,11 +16,10 @@
 //
 // One persistent CTA per SM walks the device-built item list.  Warp 0 lane 0 issues TMA loads into a
 // ring of shared-memory stages, warp 1 lane 0 issues tcgen05.mma, warps 2..5 drain TMEM.  In gather
-// mode (GEMM-1 at prefill) four more warps fetch the token operand: each thread copies its row of x,
-// found through the row -> token table of the permute step, into the 128-byte-swizzled stage with
-// 16-byte cp.async, so no permuted copy of x exists in memory (Section 2.1's "permute" folded into
-// the GEMM's operand load).  Every
-// barrier wait is bounded in time: on expiry the CTA raises bit 1 of the device error word, stops
+// mode (GEMM-1) four more warps fetch the token operand: eight threads copy one 128-byte piece of a
+// row of x, found through the row -> token table of the permute step, into the 128-byte-swizzled
+// stage with 16-byte cp.async, so no permuted copy of x exists in memory (Section 2.1's "permute"
+// folded into the GEMM's operand load).  Every barrier wait is bounded in time: on expiry the CTA raises bit 1 of the device error word, stops
 // issuing work, lets its copies in flight land, frees its TMEM and returns.
 #include <cuda_bf16.h>
 
@@ -71,7 +70,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
                     const __grid_constant__ CUtensorMap map_x_big, const GemmItem *items,
                     const int32_t *n_items_ptr, int K, int out_rows_per_slot, void *out,
                     int *err, const uint8_t *x_rows, const int32_t *src_tok) {
-    static_assert(!GATHER || (GLU && NT == kGatherThreads), "gather mode: GEMM-1, one gather thread per token row");
+    static_assert(!GATHER || (GLU && NT <= kGatherThreads), "gather mode: GEMM-1, eight gather threads per token row");
     using C = Cfg<NT, GLU>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -528,7 +527,7 @@ int setup_one() {
 int gemm_setup(ew_pool *) {
     int rc = 0;
     rc |= setup_one<32, true>() | setup_one<64, true>() | setup_one<128, true>() | setup_one<256, true>();
-    rc |= setup_one<128, true, true>();
+    rc |= setup_one<128, true, true>() | setup_one<64, true, true>() | setup_one<32, true, true>();
     rc |= setup_one<32, false>() | setup_one<64, false>() | setup_one<128, false>() | setup_one<256, false>();
     rc |= (int)cudaFuncSetAttribute(grouped_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<true>::kSmemBytes);
     rc |= (int)cudaFuncSetAttribute(grouped_gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<false>::kSmemBytes);
@@ -541,9 +540,13 @@ int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, const CUtensor
     const LayerState &L = p->layers[layer];
     const int K = p->cfg.hidden, I = p->cfg.inter;
     const Workspace &w = p->ws;
-    if (p->gather)
+    if (p->gather && p->token_tile == 128)
         return launch_one<128, true, true>(p, L.map_w13, p->map_xp, map_x, p->map_xp_big[0], map_x_big, w.items1, w.n_items, K, I,
                                            w.act, st, x);
+    if (p->gather && p->token_tile == 64)
+        return launch_one<64, true, true>(p, L.map_w13, p->map_xp, map_x, p->map_xp, map_x, w.items1, w.n_items, K, I, w.act, st, x);
+    if (p->gather && p->token_tile == 32)
+        return launch_one<32, true, true>(p, L.map_w13, p->map_xp, map_x, p->map_xp, map_x, w.items1, w.n_items, K, I, w.act, st, x);
     switch (p->token_tile) {
         case 32: return launch_one<32, true>(p, L.map_w13, p->map_xp, map_x, p->map_xp, map_x, w.items1, w.n_items, K, I, w.act, st);
         case 64: return launch_one<64, true>(p, L.map_w13, p->map_xp, map_x, p->map_xp, map_x, w.items1, w.n_items, K, I, w.act, st);

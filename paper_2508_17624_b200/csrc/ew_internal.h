@@ -36,8 +36,8 @@ struct Workspace {
     GemmItem *items1 = nullptr;
     GemmItem *items2 = nullptr;
     int32_t max_items1 = 0, max_items2 = 0;
-    void *xp = nullptr;            // [Bmax*k, H] bf16 permuted activations
-    int32_t *src_tok = nullptr;    // [Bmax*k] token of each slot-contiguous row (gather mode: GEMM-1 fetches x rows itself)
+    void *xp = nullptr;            // [Bmax*k, H] bf16 permuted activations (written only with EW_DISABLE_GATHER=1)
+    int32_t *src_tok = nullptr;    // [Bmax*k] token of each slot-contiguous row: GEMM-1 fetches those rows of x itself
     void *act = nullptr;           // [S*Bmax + Bmax*k, I] bf16 SwiGLU output
     float *y = nullptr;            // [S*Bmax + Bmax*k, H] fp32 expert outputs
     int32_t *err = nullptr;        // device error word
@@ -100,7 +100,7 @@ void set_last_error(const std::string &s);
 bool pdl_enabled(int kind = -1);
 // EW_DISABLE_PAIRS=1 keeps prefill-sized token tiles on the one-CTA kernel.
 bool pairs_enabled();
-// EW_DISABLE_GATHER=1 keeps the permuted copy of x at prefill (GEMM-1 then reads it by TMA), for debugging.
+// EW_DISABLE_GATHER=1 brings back the permuted copy of x (GEMM-1 then reads it by TMA), for debugging and A/B runs.
 bool gather_enabled();
 
 // Launch with programmatic stream serialization (the kernel calls pdl_wait() before it reads its

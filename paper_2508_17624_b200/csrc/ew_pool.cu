@@ -555,9 +555,9 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     p->token_tile2 = pick_token_tile(p, B);
     p->token_tile = p->token_tile2 == 256 ? 128 : p->token_tile2;
     p->use_pairs = p->token_tile2 == 256 && pairs_enabled();
-    // At prefill the permuted copy of x (k rows per token) is not written: the permute kernel only records which token
-    // each slot-contiguous row is, and GEMM-1 gathers those rows of x (which stay in L2) into its token operand.
-    p->gather = p->token_tile == 128 && gather_enabled();
+    // The permuted copy of x (k rows per token) is not written: the permute kernel only records which token each
+    // slot-contiguous row is, and GEMM-1 gathers those rows of x (which stay in L2) into its token operand.
+    p->gather = gather_enabled();
     if (p->token_tile >= 128) {
         uint32_t bbox[2] = {64, (uint32_t)p->token_tile};
         if (make_tensor_map(p, &map_x_big, x, 2, dx, bbox)) return EW_ERR_CUDA;

@@ -30,8 +30,9 @@
  * Parity pins (tests, "not gpu"): Figure 4's parameters for the map; merged-model equivalence,
  * base-only equivalence, identical-copy equivalence, batch and permutation invariance; fp64 brute
  * force over all C(M,k) subsets on tiny inputs; M=1,k=1 and k=M special cases against library
- * matmuls in fp64.  Nothing in the paper prints numerical layer outputs, so value-level parity of
- * ewo_ffn_given_slots rests on those invariants and library special cases.
+ * matmuls in fp64.  The paper prints no numerical layer outputs, so ewo_ffn_given_slots has no
+ * golden-value fixture: its values are pinned by those library special cases, the brute force and
+ * the bit-for-bit equality with the merged-model path.
  */
 #include <math.h>
 #include <stdint.h>

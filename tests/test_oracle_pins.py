@@ -317,3 +317,31 @@ def test_staged_path_equals_whole_path_on_c0():
     assert np.array_equal(out, out2)
     assert np.array_equal(out, oracle.layer_forward_merged(layer, x, aid))
     assert set(np.unique(aid)) == {-1, 0, 1}
+
+
+def test_counts_is_a_histogram():
+    """Tokens per slot (Section 2.1 dispatch) is a plain histogram of the slot ids: numpy's bincount."""
+    rng = np.random.default_rng(11)
+    P = 37
+    slots = rng.integers(0, P, size=(500, 3)).astype(np.int32)
+    slots[slots == 5] = 6                                     # an empty slot in the middle
+    assert np.array_equal(oracle.counts(slots, P), np.bincount(slots.reshape(-1), minlength=P))
+    assert np.array_equal(oracle.counts(np.zeros((0, 3), np.int32), P), np.zeros(P, np.int64))
+
+
+def test_topk_from_logits_against_library_topk():
+    """Given logits (the stand-alone operator's input recipe), ids and weights are the library's softmax + top-k
+    in fp64 wherever the k-th and (k+1)-th probabilities are not within rounding of each other."""
+    rng = np.random.default_rng(12)
+    B, M, k = 300, 64, 6
+    logits = rng.standard_normal((B, M)).astype(np.float32)
+    cfg = oracle.OracleConfig(16, 4, M, 0, k, 1, 1)
+    ids, w, gap = oracle.topk_from_logits(cfg, logits)
+    p = torch.softmax(torch.from_numpy(logits).double(), dim=1)
+    tw, ti = torch.topk(p, k, dim=1)                          # sorted descending
+    clear = gap > 1e-6
+    assert clear.mean() > 0.9
+    assert np.array_equal(ids[clear], ti.numpy()[clear].astype(np.int32))
+    assert np.abs(w[clear] - tw.numpy()[clear]).max() < 1e-6
+    full = np.sort(p.numpy(), axis=1)[:, ::-1]
+    assert np.abs(gap - (full[:, k - 1] - full[:, k])).max() < 1e-6

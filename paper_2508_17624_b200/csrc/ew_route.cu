@@ -1,7 +1,8 @@
 // Routing-side kernels of the adapter-aware MoE layer:
 //   reroute_kernel   the batched rerouting operator alone (Section 4.3) + histogram
-//   permute_kernel   exclusive scan of the counts, scatter of token rows into slot-contiguous order,
-//                    and (one extra CTA) the work-item lists of the grouped GEMMs
+//   permute_kernel   exclusive scan of the counts, the slot-contiguous order of the (token, expert) pairs as a
+//                    row -> token table (GEMM-1 gathers the rows of x itself), and the work-item lists of the
+//                    grouped GEMMs
 //   combine_kernel   weighted un-permute and sum, one rounding to bf16 (Section 2.1)
 #include <cuda_bf16.h>
 
@@ -159,8 +160,10 @@ __global__ void __launch_bounds__(256) reroute_kernel_unaligned(const int32_t *_
 // ------------------------------------------------------------------------------------------------
 // Scan + permute + plan.  Every CTA recomputes the exclusive scan of the (small) count array in
 // shared memory; the first kPlanners CTAs publish the offsets and write the GEMM work items (the item
-// loop is a chain of dependent integer arithmetic, so it is spread over several CTAs), the other CTAs copy
-// one token row per warp to its slot-contiguous position.  Item order:
+// loop is a chain of dependent integer arithmetic, so it is spread over several CTAs), the other CTAs record for
+// each (token, expert) pair its slot-contiguous row (inv) and for each row its token (src_tok), one thread per
+// pair.  (Without a src_tok table they copy the token rows instead, one row per warp: the debugging path that keeps
+// a permuted copy of x.)  Item order:
 //   per group the items are ordered (weight tile, token block) so that CTAs working at the same time
 //   share a weight tile through L2; thin and fat groups are merged evenly (see below).
 // ------------------------------------------------------------------------------------------------

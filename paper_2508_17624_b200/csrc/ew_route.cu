@@ -9,6 +9,7 @@
 #include <cstdlib>
 
 #include "ew_internal.h"
+#include "ew_plan.cuh"
 #include "ew_tc.cuh"
 
 namespace ew {
@@ -167,29 +168,6 @@ __global__ void __launch_bounds__(256) reroute_kernel_unaligned(const int32_t *_
 //   per group the items are ordered (weight tile, token block) so that CTAs working at the same time
 //   share a weight tile through L2; thin and fat groups are merged evenly (see below).
 // ------------------------------------------------------------------------------------------------
-__device__ void block_exclusive_scan(const int32_t *in, int32_t *out, int n, int32_t *warp_sums) {
-    // out[0..n] = exclusive scan of in[0..n-1] (out[n] = total); blockDim.x = 256
-    const int per = (n + 255) / 256;
-    const int lo = min(threadIdx.x * per, n), hi = min(lo + per, n);
-    int32_t s = 0;
-    for (int i = lo; i < hi; ++i) s += in[i];
-    int32_t incl = s;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (lane == 31) warp_sums[warp] = incl;
-    __syncthreads();
-    int32_t base = 0;
-    for (int w = 0; w < warp; ++w) base += warp_sums[w];
-    int32_t run = base + incl - s;
-    for (int i = lo; i < hi; ++i) { out[i] = run; run += in[i]; }
-    if (threadIdx.x == 255) out[n] = run;     // thread 255's range ends at n
-    __syncthreads();
-}
-
 constexpr int kPlanners = 8;
 
 __global__ void __launch_bounds__(256) permute_kernel(const uint4 *x, const int32_t *slot_ids,
@@ -199,32 +177,32 @@ __global__ void __launch_bounds__(256) permute_kernel(const uint4 *x, const int3
                                                       uint4 *xp, int32_t *src_tok, GemmItem *items1,
                                                       GemmItem *items2, int32_t *n_items) {
     extern __shared__ int32_t sm[];
-    int32_t *off = sm;                 // [P + 1]
-    int32_t *blk = sm + P + 1;         // [P + S + 1] token blocks per group, scanned
     __shared__ int32_t warp_sums[8];
     tc::pdl_launch_dependents();
     // counts, slot ids and ranks come from the router kernel, x from the caller's earlier work: none of the kernel's
     // pointer parameters is __restrict__, so that no load can be hoisted above this wait
     tc::pdl_wait();
-    int32_t *cnt_s = sm + (P + 1) + 4 * (P + S + 1);    // [P] the counts, staged once
-    for (int i = threadIdx.x; i < P; i += 256) cnt_s[i] = counts[i];
-    __syncthreads();
-    block_exclusive_scan(cnt_s, off, P, warp_sums);
+    const int32_t *cnt_s = plan::stage_and_scan(sm, counts, P, S, warp_sums, 256);
+    const int32_t *off = sm;                 // [P + 1]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long n_pairs = (long long)B * k;
     if (blockIdx.x >= kPlanners && src_tok) {
         // gather mode: no copy of x; one thread per (token, j) pair records the pair's row and the row's token
         const long long q = (long long)(blockIdx.x - kPlanners) * 256 + threadIdx.x;
-        if (q < (long long)B * k) {
+        if (q < n_pairs) {
             const int dest = off[slot_ids[q]] + rank[q];
-            inv[q] = dest;
-            src_tok[dest] = (int32_t)(q / k);
+            if (dest < n_pairs) {            // always, unless the routing kernel gave up midway (error word set)
+                inv[q] = dest;
+                src_tok[dest] = (int32_t)(q / k);
+            }
         }
         return;
     }
     if (blockIdx.x >= kPlanners) {                       // the first CTAs (dispatched first) are the planners
         const long long q = (long long)(blockIdx.x - kPlanners) * 8 + warp;
-        if (q < (long long)B * k) {
+        if (q < n_pairs) {
             const int dest = off[slot_ids[q]] + rank[q];
+            if (dest >= n_pairs) return;
             if (lane == 0) inv[q] = dest;
             const int hv = H >> 3;
             const uint4 *src = x + (size_t)(q / k) * hv;
@@ -243,77 +221,11 @@ __global__ void __launch_bounds__(256) permute_kernel(const uint4 *x, const int3
         }
         return;
     }
-    // ---- planner CTAs: each repeats the (cheap) scans and writes the items of every kPlanners-th group
-    if (blockIdx.x == 0)
-        for (int i = threadIdx.x; i <= P; i += 256) offsets[i] = off[i];
-    // groups: g < S shared expert g (rows = B); g >= S slot g - S (rows = counts).  Two classes: "thin" groups
-    // (at most kThinRows rows: their items are weight streams) and "fat" ones (tensor-core bound at prefill).
-    // The two item sequences are merged evenly, so that at any moment the CTAs hold a mix of both and the
-    // weight stream of the thin items overlaps the arithmetic of the fat ones.
-    constexpr int kThinRows = 64;
-    const int G = P + S;
-    int32_t *nblk = blk + G + 1;            // [G] token blocks of fat groups (0 for thin ones)
-    int32_t *blk_t = nblk + G;              // [G + 1] scan of the thin groups' token blocks
-    int32_t *nblk_t = blk_t + G + 1;        // [G]
-    // GEMM-1 and GEMM-2 may use different token tiles (NT1, NT2): each pass has its own block counts and scans
-    for (int pass = 0; pass < 2; ++pass) {
-        const int NT = pass ? NT2 : NT1;
-        const int R = pass ? R2 : R1;
-        if (pass == 0 || NT2 != NT1) {                    // same tile in both GEMMs (decode): one set of scans serves both
-            __syncthreads();                              // the previous pass has finished reading the scan arrays
-            for (int g = threadIdx.x; g < G; g += 256) {
-                const int rows = g < S ? B : cnt_s[g - S];
-                const int nb = (rows + NT - 1) / NT;
-                const bool thin = rows <= kThinRows;
-                nblk[g] = thin ? 0 : nb;
-                nblk_t[g] = thin ? nb : 0;
-            }
-            __syncthreads();
-            block_exclusive_scan(nblk, blk, G, warp_sums);
-            block_exclusive_scan(nblk_t, blk_t, G, warp_sums);
-        }
-        const int fat_blocks = blk[G], thin_blocks = blk_t[G];
-        if (blockIdx.x == 0 && threadIdx.x == 0) n_items[pass] = (fat_blocks + thin_blocks) * R;
-        const long long n_fat = (long long)fat_blocks * R, n_thin = (long long)thin_blocks * R;
-        const bool small = (n_fat + 1) * (n_thin + 1) < (1ll << 31);
-        GemmItem *dst = pass ? items2 : items1;
-        for (int g = warp + 8 * blockIdx.x; g < G; g += 8 * kPlanners) {
-            const bool thin = nblk_t[g] > 0;
-            const int nb = thin ? nblk_t[g] : nblk[g];
-            if (nb == 0) continue;
-            const bool shared = g < S;
-            const int rows = shared ? B : cnt_s[g - S];
-            const int slot = shared ? P + g : g - S;
-            const int in0 = shared ? 0 : off[g - S];
-            const int out0 = shared ? g * B : S * B + off[g - S];
-            const long long first = (long long)(thin ? blk_t[g] : blk[g]) * R;    // index inside the group's own class
-            for (int i = lane; i < nb * R; i += 32) {
-                const int tile = i / nb, c = i % nb;
-                GemmItem it;
-                it.slot = slot; it.tile = tile;
-                it.in_row = (pass ? out0 : in0) + c * NT;     // GEMM-2 reads what GEMM-1 wrote
-                it.out_row = out0 + c * NT;
-                it.rows = min(NT, rows - c * NT);
-                it.from_x = (!pass && shared) ? 1 : 0;
-                it.pad0 = it.pad1 = 0;
-                // merged position: thin item q has floor(q*n_fat/n_thin) fat items before it, and fat item q
-                // the thin items that rule puts before it
-                const long long q = first + i;
-                long long pos;
-                if (small) {                                  // every product fits 32 bits: cheap divisions
-                    const unsigned qu = (unsigned)q, nf = (unsigned)n_fat, nt = (unsigned)n_thin;
-                    if (thin) pos = nf ? qu + qu * nf / nt : qu;
-                    else pos = nt ? qu + min(nt, ((qu + 1) * nt + nf - 1) / nf) : qu;
-                } else {
-                    if (thin) pos = n_fat ? q + q * n_fat / n_thin : q;
-                    else pos = n_thin ? q + min(n_thin, ((q + 1) * n_thin + n_fat - 1) / n_fat) : q;
-                }
-                int4 *d4 = reinterpret_cast<int4 *>(dst + pos);      // one item = two 16-byte stores
-                d4[0] = make_int4(it.slot, it.tile, it.in_row, it.out_row);
-                d4[1] = make_int4(it.rows, it.from_x, 0, 0);
-            }
-        }
-    }
+    // ---- planner CTAs: each has repeated the (cheap) scan and writes the items of every kPlanners-th group
+    plan::Params A;
+    A.B = B; A.k = k; A.P = P; A.S = S; A.NT1 = NT1; A.NT2 = NT2; A.R1 = R1; A.R2 = R2;
+    A.offsets = offsets; A.items1 = items1; A.items2 = items2; A.n_items = n_items;
+    plan::write_items(sm, cnt_s, A, warp_sums, 256, warp + 8 * blockIdx.x, 8 * kPlanners, blockIdx.x == 0);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -366,15 +278,21 @@ int pick_token_tile(const ew_pool *p, int B) {
     return want <= 32 ? 32 : want <= 64 ? 64 : want <= 128 ? 128 : 256;
 }
 
+// weight tiles per group: 128-row tiles, or 256-row tile pairs where the CTA-pair kernel runs the items
+void plan_tiles(const ew_pool *p, int *R1, int *R2) {
+    const ew_config_t &c = p->cfg;
+    *R1 = (c.inter + 127) / 128;                                 // GEMM-1 always runs on the one-CTA kernel
+    const int tile_rows2 = p->use_pairs ? 256 : 128;
+    *R2 = (c.hidden + tile_rows2 - 1) / tile_rows2;
+}
+
 int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
-    // weight tiles per group: 128-row tiles, or 256-row tile pairs where the CTA-pair kernel runs the items
-    const int R1 = (c.inter + 127) / 128;                        // GEMM-1 always runs on the one-CTA kernel
-    const int tile_rows2 = p->use_pairs ? 256 : 128;
-    const int R2 = (c.hidden + tile_rows2 - 1) / tile_rows2;
+    int R1, R2;
+    plan_tiles(p, &R1, &R2);
     const long long pairs = (long long)B * c.top_k;
     const int grid = (int)(p->gather ? (pairs + 255) / 256 : (pairs + 7) / 8) + kPlanners;
-    const size_t smem = ((size_t)(p->P + 1) + 4 * (size_t)(p->P + c.num_shared + 1) + p->P) * 4;
+    const size_t smem = plan::smem_words(p->P, c.num_shared) * 4;
     return launch_pdl(1, permute_kernel, dim3(grid), dim3(256), smem, st, (const uint4 *)x, p->ws.slot_ids, p->ws.rank,
                       p->ws.counts, B, c.top_k, c.hidden, p->P, c.num_shared, p->token_tile, p->token_tile2, R1, R2, p->ws.offsets, p->ws.inv,
                       (uint4 *)p->ws.xp, p->gather ? p->ws.src_tok : (int32_t *)nullptr, p->ws.items1, p->ws.items2,

@@ -256,7 +256,7 @@ def run_cuda(args):
             "config": {"workload": workload, "tokens_per_step_per_gpu": B, "hidden": H, "inter": cfg.inter,
                        "experts": cfg.num_experts, "shared": cfg.num_shared, "top_k": k,
                        "adapters": cfg.max_adapters, "e_max": cfg.e_max, "live_slots": live,
-                       "token_tile": None, "parallelism": f"replicas x{world}",
+                       "parallelism": f"replicas x{world}",
                        "l2": "no flush: each step streams %.2f GB of live expert weights, far above the 126 MB L2"
                              % (bytes_layer / 1e9)},
             "e2e": {"value": whole_job_tokens_per_s(world, B, max(side_steps, 1), ms_e2e), "unit": UNIT,

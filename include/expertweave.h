@@ -141,6 +141,9 @@ ew_status_t ew_pool_trim(ew_pool_t *pool);
  *   out          device bf16 [n_tokens, H]
  *   cuda_stream  a cudaStream_t (null = the legacy default stream)
  * No host synchronisation; token counts never leave the device.  n_tokens = 0 is a no-op.
+ * A pool owns one workspace, so its forwards run one after another: a call on another stream than the
+ * previous one first makes its stream wait for that forward (device-side; the host does not block).
+ * Host calls on one pool are not thread-safe: serialise them, or give each thread its own pool.
  * The call may be captured into a CUDA graph after one uncaptured warm-up call with the same n_tokens;
  * ew_unload_adapter and ew_load_base wait for forwards issued directly, not for replays of such a graph:
  * synchronise those yourself before evicting.

@@ -503,6 +503,16 @@ extern "C" ew_status_t ew_last_device_error(ew_pool_t *p, int32_t *code) {
     return EW_OK;
 }
 
+// The pool has one workspace: a forward issued on one stream must not overlap a forward that was issued earlier on
+// another.  Makes `st` wait for the last forward of every other stream (a no-op when those have finished).
+static ew_status_t order_after_other_streams(ew_pool *p, cudaStream_t st) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap != cudaStreamCaptureStatusNone) return EW_OK;
+    for (auto &e : p->fwd_events)
+        if (e.first != st) CU_TRY(cudaStreamWaitEvent(st, e.second, 0));
+    return EW_OK;
+}
+
 static ew_status_t note_forward(ew_pool *p, cudaStream_t st) {
     // A forward that is being captured into a CUDA graph is not running yet: there is nothing to record.  The
     // caller who replays such a graph orders its replays against ew_unload_adapter / ew_load_base itself.
@@ -574,6 +584,10 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
         p->prof_used += 6;
     }
 #define PROF_MARK(i) do { if (pe) CU_TRY(cudaEventRecord(pe[i], st)); } while (0)
+    {
+        ew_status_t ordered = order_after_other_streams(p, st);
+        if (ordered != EW_OK) return ordered;
+    }
     PROF_MARK(0);
     if (!p->counts_clean) CU_TRY(cudaMemsetAsync(p->ws.counts, 0, (size_t)p->P * 4, st));   // an earlier forward failed midway
     p->counts_clean = false;

@@ -500,6 +500,43 @@ def test_back_to_back_forwards_with_changing_inputs(name):
     pool.destroy()
 
 
+def test_forwards_on_two_streams_share_the_workspace_in_order():
+    """One pool, two streams, no host synchronisation between the calls: the pool makes a forward wait for the one
+    issued before it on the other stream, so the single workspace is never used by two forwards at once."""
+    import torch
+    cfg = wl.CONFIGS["c1"]
+    pool = binding.Pool.from_config(cfg)
+    binding.load_model(pool, cfg)
+    rng = np.random.default_rng(5)
+    batches = []
+    for i in range(6):
+        n = cfg.n_tokens - 13 * i
+        x = wl.f32_to_bf16_bits(rng.standard_normal((n, cfg.hidden)).astype(np.float32))
+        aid = rng.integers(-1, cfg.max_adapters, size=n).astype(np.int32)
+        batches.append((to_dev(x), to_dev(aid)))
+    ref = []
+    for x, aid in batches:
+        ref.append(pool.moe_forward(0, x, aid).clone())
+        torch.cuda.synchronize()
+    outs = [torch.empty_like(b[0]) for b in batches]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    busy = torch.empty(1 << 28, dtype=torch.uint8, device="cuda")
+    for rep in range(4):
+        torch.cuda.synchronize()
+        for s in streams:
+            with torch.cuda.stream(s):
+                busy.zero_()                    # both streams start behind a long kernel: the launches queue up
+        for i in range(len(batches)):
+            with torch.cuda.stream(streams[i % 2]):
+                pool.moe_forward(0, batches[i][0], batches[i][1], outs[i])
+        torch.cuda.synchronize()
+        for i in range(len(batches)):
+            assert torch.equal(outs[i], ref[i]), (rep, i)
+            outs[i].zero_()
+    assert pool.last_device_error() == 0
+    pool.destroy()
+
+
 def test_host_buffer_pipeline():
     """ew_moe_forward_host overlaps upload, kernels and download across calls with double-buffered staging:
     different batches issued back to back (and mixed with direct device-side calls) give the direct results."""

@@ -6,7 +6,9 @@
 // ring.  The kernel is latency-bound, so each TMA instruction fetches up to four 64-element K-atoms at once
 // (3-D descriptors ordered element, row, atom: shared memory receives one swizzled tile per atom).  Only the first
 // `tok_tile` rows of the 128-row MMA tile are loaded; the other rows hold whatever shared memory held
-// and feed accumulator lanes nobody reads.  TMEM lane i belongs to token i, so in the epilogue every
+// and feed accumulator lanes nobody reads.  TMEM lane i belongs to token i.  With 32-token tiles (small
+// batches) one warp spills the logits to shared memory and four threads share each token's softmax and
+// top-k (see the epilogue); with larger tiles every epilogue
 // thread owns one token: it reads its M logits from TMEM, forms the softmax probabilities in fp32, takes
 // k arg-max rounds (probability descending, lower index on ties), looks each chosen expert up in the
 // layer's expert map Pi (staged in shared memory) under the token's adapter id, and bumps the slot's
@@ -157,6 +159,120 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                 if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1; }
             }
             if (ok) tc_commit(bar_done);
+        }
+    } else if (REG && tok_tile == 32) {
+        // epilogue for 32-token tiles (small batches, where this kernel's latency is exposed): the logits sit in
+        // TMEM lanes 0..31 only, which one warp can read; that warp spills them to shared memory and then all four
+        // epilogue warps work on them, four threads per token, each owning a quarter of the experts: partial max
+        // and partial sum for the softmax, then k rounds of "publish my best remaining candidate, everybody picks
+        // the best of the token's four" (value descending, lower expert index on ties).
+        const int g = warp & 3;                                      // expert group of this thread
+        const int E = n_mma >> 2;                                    // experts per group (4, 8, 12 or 16)
+        const int t = tok0 + lane;
+        const int k = A.k;
+        auto quad_sync = [] { asm volatile("bar.sync 1, 128;" ::: "memory"); };   // the four epilogue warps
+        mbar_wait(bar_done, 0, abort_flag, A.err);
+        quad_sync();                                                 // every epilogue thread is past its (bounded) wait
+        if (!*abort_flag) {
+            tc_fence_after();
+            float *lg_s = reinterpret_cast<float *>(smem_al);        // [n_mma][32] logits, expert-major (the ring has drained)
+            float *red_s = lg_s + 64 * 32;                           // [2][4][32] partial max, partial sum
+            float *cv_s = red_s + 2 * 4 * 32;                        // [2][4][32] candidate values, double-buffered by round
+            int *ci_s = reinterpret_cast<int *>(cv_s + 2 * 4 * 32);  // [2][4][32] candidate expert ids
+            if (g == 0) {
+                uint32_t v0[32], v1[32];
+                if (n_mma >= 32) tc_ld32(tmem_base, v0); else tc_ld16(tmem_base, v0);
+                if (n_mma > 32) { if (n_mma - 32 >= 32) tc_ld32(tmem_base + 32, v1); else tc_ld16(tmem_base + 32, v1); }
+                tc_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    if (j < n_mma) lg_s[j * 32 + lane] = __uint_as_float(v0[j]);
+                    if (32 + j < n_mma) lg_s[(32 + j) * 32 + lane] = __uint_as_float(v1[j]);
+                }
+            }
+            quad_sync();
+            float p[16];
+            float mx = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int j = g * E + i;
+                p[i] = (i < E && j < M) ? lg_s[j * 32 + lane] : -INFINITY;
+                mx = fmaxf(mx, p[i]);
+            }
+            red_s[g * 32 + lane] = mx;
+            quad_sync();
+            mx = fmaxf(fmaxf(red_s[lane], red_s[32 + lane]), fmaxf(red_s[64 + lane], red_s[96 + lane]));
+            float sum = 0.f;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {                           // exp(-inf) = 0 for the absent experts
+                p[i] = expf(p[i] - mx);
+                sum += p[i];
+            }
+            red_s[128 + g * 32 + lane] = sum;
+            quad_sync();
+            sum = ((red_s[128 + lane] + red_s[160 + lane]) + red_s[192 + lane]) + red_s[224 + lane];
+            const float inv_sum = 1.f / sum;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) p[i] = (i < E && g * E + i < M) ? p[i] * inv_sum : -1.f;
+            const int a = t < A.B ? checked_aid(A.aid[t], A.N, A.loaded, A.err) : -1;
+            float wsum = 0.f;
+            float my_w[8];                                           // weights and slots of the pairs this thread writes (r = g, g+4, ...)
+            int my_slot[8];
+            for (int r = 0; r < k; ++r) {
+                float bv = -1.f;
+                int bi = 0;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {                       // branch-free selects; strict >: the lower index keeps a tie
+                    const bool gt = p[i] > bv;
+                    bv = gt ? p[i] : bv;
+                    bi = gt ? i : bi;
+                }
+                const int buf = (r & 1) * 128;
+                cv_s[buf + g * 32 + lane] = bv;
+                ci_s[buf + g * 32 + lane] = g * E + bi;
+                quad_sync();
+                float wv = cv_s[buf + lane];
+                int wg = 0;
+#pragma unroll
+                for (int q = 1; q < 4; ++q) {                        // groups in ascending expert order: strict > keeps the lower index
+                    const float c = cv_s[buf + q * 32 + lane];
+                    const bool gt = c > wv;
+                    wv = gt ? c : wv;
+                    wg = gt ? q : wg;
+                }
+                const int wi = ci_s[buf + wg * 32 + lane];
+                if (wg == g) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) p[i] = (i == bi) ? -1.f : p[i];   // taken (probabilities are >= 0)
+                }
+                wsum += wv;
+                if ((r & 3) == g && t < A.B) {                       // the token's four threads share the output work
+                    const int slot = a < 0 ? wi : (A.pi_in_smem ? pi_s[a * M + wi] : __ldg(A.pi + a * M + wi));
+                    const size_t o = (size_t)t * k + r;
+                    A.topk_ids[o] = wi;
+                    A.slot_ids[o] = slot;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        if (u == (r >> 2)) { my_w[u] = wv; my_slot[u] = slot; }
+                }
+            }
+            if (t < A.B) {
+                // per-slot histogram: one atomic per pair, all of this thread's in flight together; the value
+                // returned is the pair's position inside its slot's chunk
+                int got[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (g + 4 * u < k) got[u] = atomicAdd(A.counts + my_slot[u], 1);
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (g + 4 * u < k) {
+                        const size_t o = (size_t)t * k + g + 4 * u;
+                        float w = my_w[u];
+                        if (A.renormalize) w = w / wsum;
+                        A.topk_w[o] = (A.renormalize || A.scale != 1.f) ? w * A.scale : w;
+                        A.rank[o] = got[u];
+                    }
+            }
         }
     } else {
         // epilogue: thread <-> token

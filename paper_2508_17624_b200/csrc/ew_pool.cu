@@ -523,6 +523,17 @@ static ew_status_t note_forward(ew_pool *p, cudaStream_t st) {
             CU_TRY(cudaEventRecord(e.second, st));
             return EW_OK;
         }
+    // a caller that keeps creating streams would grow the list without bound: entries whose forward has completed
+    // carry no ordering information any more
+    if (p->fwd_events.size() >= 32) {
+        size_t kept = 0;
+        for (auto &e : p->fwd_events) {
+            if (cudaEventQuery(e.second) == cudaSuccess) cudaEventDestroy(e.second);
+            else p->fwd_events[kept++] = e;
+        }
+        p->fwd_events.resize(kept);
+        (void)cudaGetLastError();                       // cudaErrorNotReady from the queries is not an error
+    }
     cudaEvent_t ev;
     CU_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
     CU_TRY(cudaEventRecord(ev, st));

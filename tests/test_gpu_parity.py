@@ -537,6 +537,28 @@ def test_forwards_on_two_streams_share_the_workspace_in_order():
     pool.destroy()
 
 
+def test_many_short_lived_streams():
+    """A caller that uses a fresh stream for every call: the pool's per-stream bookkeeping must stay bounded and the
+    results must not change."""
+    import torch
+    cfg = wl.CONFIGS["c0"]
+    pool = binding.Pool.from_config(cfg)
+    binding.load_model(pool, cfg)
+    x, aid = to_dev(wl.gen_tokens(cfg)), to_dev(wl.gen_adapter_ids(cfg))
+    ref = pool.moe_forward(0, x, aid).clone()
+    torch.cuda.synchronize()
+    for i in range(100):
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            out = pool.moe_forward(0, x, aid)
+        s.synchronize()
+        assert torch.equal(out, ref), i
+        del s
+    pool.unload_adapter(0)                      # walks the bookkeeping of every stream still listed
+    assert pool.last_device_error() == 0
+    pool.destroy()
+
+
 def test_host_buffer_pipeline():
     """ew_moe_forward_host overlaps upload, kernels and download across calls with double-buffered staging:
     different batches issued back to back (and mixed with direct device-side calls) give the direct results."""

@@ -1,4 +1,4 @@
-// Dispatch planning shared by the permute kernel and by the router kernel's tail: the exclusive scan of the
+// Dispatch planning (device functions used by the permute kernel): the exclusive scan of the
 // per-slot token counts (Section 2.1 dispatch), the slot-contiguous order of the (token, expert) pairs as two
 // tables (inv: pair -> row, src_tok: row -> token), and the work-item lists of the two grouped GEMMs.
 //

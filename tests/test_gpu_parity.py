@@ -351,6 +351,8 @@ def test_adapter_churn_under_load():
     dict(hidden=256, inter=128, num_experts=80, num_shared=0, top_k=3, max_adapters=2, e_max=2, n_tokens=130), # M > 64: shared-memory softmax path
     dict(hidden=64, inter=64, num_experts=256, num_shared=1, top_k=4, max_adapters=1, e_max=3, n_tokens=33),   # the largest M
     dict(hidden=64, inter=64, num_experts=256, num_shared=0, top_k=2, max_adapters=20, e_max=1, n_tokens=70),  # expert map too large for shared memory
+    dict(hidden=64, inter=64, num_experts=64, num_shared=1, top_k=32, max_adapters=2, e_max=4, n_tokens=50),    # the largest k
+    dict(hidden=64, inter=64, num_experts=64, num_shared=1, top_k=32, max_adapters=2, e_max=4, n_tokens=600),   # and with prefill tiles
     # prefill-sized batches (128-row gather tiles in GEMM-1, 256-row CTA-pair tiles in GEMM-2) on shapes off the tile sizes
     dict(hidden=128, inter=200, num_experts=8, num_shared=1, top_k=2, max_adapters=3, e_max=3, n_tokens=3001),  # H = one weight tile: half-empty tile pair
     dict(hidden=192, inter=72, num_experts=4, num_shared=0, top_k=4, max_adapters=2, e_max=4, n_tokens=1500),   # k = M, I < one tile

@@ -283,7 +283,8 @@ def run_cuda(args):
 
 
 def run_reroute(args):
-    """--workload c4: the batched rerouting operator alone (ids in, slot ids + per-slot counts out).
+    """--workload c4: the batched rerouting operator alone (ids in, slot ids + per-slot counts out), and the same
+    step fused with the gate function before it (fp32 logits in).
 
     One JSON line per coverage (10 / 25 / 50 % of the experts re-tuned) at 65536 tokens, plus a size sweep
     up to 2^24 tokens.  Cold L2: consecutive launches work on different buffer sets whose total exceeds the
@@ -344,6 +345,43 @@ def run_reroute(args):
         if e != 32:
             for i in range(N):
                 pool.unload_adapter(i)
+    # ---- the same step fused with the gate function before it: fp32 logits in; ids, weights, slot ids and counts out
+    def measure_logits(B, iters):
+        nbytes = B * M * 4 + B * 4 + 3 * B * k * 4 + N * M * 4
+        n_sets = min(24, max(2, int((256 << 20) // nbytes) + 1))
+        g = torch.Generator(device="cuda").manual_seed(5)
+        sets = [(torch.randn((B, M), device="cuda", generator=g),
+                 torch.randint(-1, N, (B,), device="cuda", generator=g, dtype=torch.int32)) for _ in range(n_sets)]
+        for i in range(3):
+            pool.route_logits(0, *sets[i % n_sets])
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        outs = pool.route_logits(0, *sets[0])                      # output tensors reused below: no allocation in the loop
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(iters):
+            lg_, aid_ = sets[i % n_sets]
+            binding._check(binding.lib().ew_route_logits(pool._h, 0, binding._dp(lg_), binding._dp(aid_), B, binding._dp(outs[0]),
+                                                         binding._dp(outs[1]), binding._dp(outs[2]), binding._dp(outs[3]),
+                                                         binding._stream()), "ew_route_logits")
+        e1.record()
+        torch.cuda.synchronize()
+        return nbytes, e0.elapsed_time(e1) / iters, n_sets
+
+    Bt = args.tokens or cfg.n_tokens
+    nbytes, ms, n_sets = measure_logits(Bt, args.steps)
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    lines.append({"metric": "gate + reroute from logits GB/s", "value": gbs, "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
+                  "ms_per_launch": ms, "tokens": Bt, "tokens_per_s": Bt / (ms * 1e-3), "dtype": "f32", "data": "synthetic",
+                  "config": {"workload": f"c4: softmax + top-k + reroute + counts from fp32 logits, {Bt} tokens, 20 adapters x 32 of 64 experts",
+                             "l2": f"cold: {n_sets} rotating buffer sets", "includes": "zeroing of counts + kernel"},
+                  "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                               "of": peak_kind, "algorithmic_bytes": nbytes, "traffic": None}})
+    sweep = []
+    for lg in (() if args.tokens else (16, 18, 20, 22)):
+        nb_, ms_, _ = measure_logits(1 << lg, max(20, args.steps >> max(0, lg - 16)))
+        sweep.append({"tokens": 1 << lg, "ms_per_launch": ms_, "GB/s": nb_ / (ms_ * 1e-3) / 1e9,
+                      "frac": nb_ / (ms_ * 1e-3) / 1e9 / peak})
+    lines.append({"metric": "gate + reroute from logits GB/s, size sweep", "sweep": sweep, "peak": peak, "of": peak_kind})
     sweep = []
     for lg in (() if args.tokens else (16, 18, 20, 22, 24)):
         nbytes, ms, n_sets = measure(1 << lg, max(20, args.steps >> max(0, lg - 18)))

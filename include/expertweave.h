@@ -193,6 +193,19 @@ ew_status_t ew_profile_read(ew_pool_t *pool, double *ms, int32_t *n_forwards);
 ew_status_t ew_reroute(ew_pool_t *pool, int32_t layer, const int32_t *topk_ids, const int32_t *adapter_ids,
                        int32_t n_tokens, int32_t *slot_ids, int32_t *counts, void *cuda_stream);
 
+/* Gate function and rerouting from given logits, in one kernel (Sections 2.1 and 4.3; the operator of
+ * ew_reroute fused with the softmax + top-k that precedes it): for every token softmax over its M logits, the
+ * top_k largest probabilities (ties to the lower index) as topk_ids / topk_w (renormalised and scaled as the
+ * pool's config says), slot_ids[t,j] = adapter_ids[t] < 0 ? id : Pi[layer][adapter_ids[t]][id], and the
+ * number of pairs per slot in counts (overwritten).  All pointers DEVICE: logits fp32 [n_tokens, M],
+ * row-major, 16-byte aligned; adapter_ids [n_tokens]; topk_ids, slot_ids [n_tokens, top_k] int32; topk_w
+ * [n_tokens, top_k] fp32; counts [M + N*E_max] int32.  n_tokens is not limited by max_tokens; M must be a
+ * multiple of 4.  Bad adapter ids behave as -1 and raise the device error word.  Asynchronous on cuda_stream.
+ * Errors: EW_ERR_INVALID_ARG, EW_ERR_NOT_LOADED, EW_ERR_NO_DEVICE, EW_ERR_CUDA. */
+ew_status_t ew_route_logits(ew_pool_t *pool, int32_t layer, const float *logits, const int32_t *adapter_ids,
+                            int32_t n_tokens, int32_t *topk_ids, float *topk_w, int32_t *slot_ids, int32_t *counts,
+                            void *cuda_stream);
+
 /* Routing without any allocation (the paper has no counterpart: this entry point exists for callers
  * of this library that cannot allocate device memory when they need a routing decision - an engine
  * whose KV cache has taken all free HBM, code running where the CUDA allocator must not be entered,

@@ -22,7 +22,7 @@ STATUS_NAMES = ["EW_OK", "EW_ERR_INVALID_ARG", "EW_ERR_OOM", "EW_ERR_SLOT_IN_USE
                 "EW_ERR_NO_DEVICE"]
 EXPORTS = ["ew_pool_create", "ew_pool_destroy", "ew_load_base", "ew_load_adapter", "ew_unload_adapter",
            "ew_pool_trim", "ew_moe_forward", "ew_moe_forward_debug", "ew_moe_forward_host", "ew_profile_enable",
-           "ew_profile_read", "ew_reroute", "ew_route_noalloc", "ew_selftest_bounded_wait", "ew_get_expert_map",
+           "ew_profile_read", "ew_reroute", "ew_route_logits", "ew_route_noalloc", "ew_selftest_bounded_wait", "ew_get_expert_map",
            "ew_pool_stats", "ew_last_device_error", "ew_slot_address", "ew_status_str", "ew_last_error_string"]
 
 
@@ -201,6 +201,18 @@ class Pool:
         _check(lib().ew_reroute(self._h, layer, _dp(topk_ids), _dp(adapter_ids), topk_ids.shape[0], _dp(slot_ids),
                                 _dp(counts), _stream()), "ew_reroute")
         return slot_ids, counts
+
+    def route_logits(self, layer, logits, adapter_ids):
+        """Softmax + top-k + rerouting + per-slot counts from fp32 logits [n, M] (device tensors)."""
+        import torch
+        n, k, dev = logits.shape[0], self.cfg.top_k, logits.device
+        ids = torch.empty((n, k), dtype=torch.int32, device=dev)
+        w = torch.empty((n, k), dtype=torch.float32, device=dev)
+        slots = torch.empty((n, k), dtype=torch.int32, device=dev)
+        counts = torch.empty((self.num_slots,), dtype=torch.int32, device=dev)
+        _check(lib().ew_route_logits(self._h, layer, _dp(logits), _dp(adapter_ids), n, _dp(ids), _dp(w), _dp(slots),
+                                     _dp(counts), _stream()), "ew_route_logits")
+        return ids, w, slots, counts
 
     def route_noalloc(self, layer, x, adapter_ids, topk_ids, topk_w, slot_ids, counts, device_status=None):
         """Routing into caller-provided device tensors; the library allocates nothing (see the header)."""

@@ -138,6 +138,8 @@ int launch_gemm2(ew_pool *p, int layer, int B, cudaStream_t st);
 int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st);
 int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid, int B, int32_t *slots,
                    int32_t *counts, cudaStream_t st);
+int launch_route_logits(ew_pool *p, int layer, const float *logits, const int32_t *aid, int B, int32_t *topk_ids,
+                        float *topk_w, int32_t *slot_ids, int32_t *counts, cudaStream_t st);
 int gemm_setup(ew_pool *p);   // once per pool: opt in to the shared memory the GEMM kernels need
 
 }  // namespace ew

@@ -644,6 +644,26 @@ extern "C" ew_status_t ew_reroute(ew_pool_t *p, int32_t layer, const int32_t *to
     return note_forward(p, st);
 }
 
+extern "C" ew_status_t ew_route_logits(ew_pool_t *p, int32_t layer, const float *logits, const int32_t *aid, int32_t B,
+                                       int32_t *topk_ids, float *topk_w, int32_t *slot_ids, int32_t *counts,
+                                       void *cuda_stream) {
+    if (!p || layer < 0 || layer >= p->cfg.num_layers || B < 0 || !counts) return EW_ERR_INVALID_ARG;
+    if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
+    if (!p->layers[layer].base_loaded) return EW_ERR_NOT_LOADED;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int dev = -1;
+    CU_TRY(cudaGetDevice(&dev));
+    if (dev != p->cfg.device) CU_TRY(cudaSetDevice(p->cfg.device));
+    CU_TRY(cudaMemsetAsync(counts, 0, (size_t)p->P * 4, st));
+    if (B == 0) return EW_OK;
+    if (!logits || !aid || !topk_ids || !topk_w || !slot_ids || ((uintptr_t)logits & 15) || (p->cfg.num_experts & 3)) {
+        set_last_error("ew_route_logits: null argument, logits not 16-byte aligned, or M not a multiple of 4");
+        return EW_ERR_INVALID_ARG;
+    }
+    LAUNCH_TRY(launch_route_logits(p, layer, logits, aid, B, topk_ids, topk_w, slot_ids, counts, st));
+    return note_forward(p, st);
+}
+
 extern "C" ew_status_t ew_moe_forward_host(ew_pool_t *p, int32_t layer, const void *x_host, const int32_t *aid_host,
                                            int32_t B, void *out_host, void *cuda_stream) {
     if (!p || layer < 0 || layer >= p->cfg.num_layers || B < 0 || B > p->cfg.max_tokens) return EW_ERR_INVALID_ARG;

@@ -159,6 +159,141 @@ __global__ void __launch_bounds__(256) reroute_kernel_unaligned(const int32_t *_
 }
 
 // ------------------------------------------------------------------------------------------------
+// Gate + rerouting from given logits (the stand-alone operator fused with the gate function it follows,
+// Sections 2.1 and 4.3): softmax over the M logits of each token, k largest probabilities (lower index on ties),
+// slot = Pi[aid][id], per-slot counts.  A CTA owns 128 tokens; the threads copy their logits [128, M] fp32 into
+// shared memory with coalesced 16-byte loads, rows M + 1 words apart so that the per-token reads that follow spread
+// over the banks.  Four neighbouring lanes of a warp share a token, lane g of the four owning the experts
+// [EPT*g, EPT*g + EPT) in registers (EPT = 16 for M <= 64, else 64).  Softmax by partial max and partial sum,
+// exchanged with two butterfly shuffles; then k rounds in which every lane offers its best remaining candidate and
+// the four settle the token's best the same way - no block-wide barrier after the tile has landed.  Counts go
+// through a shared-memory histogram, one atomic per non-empty slot and CTA.
+// ------------------------------------------------------------------------------------------------
+constexpr int kLogitTok = 128;
+
+template <int EPT>
+__global__ void __launch_bounds__(4 * kLogitTok) route_logits_kernel(const float4 *__restrict__ logits, const int32_t *__restrict__ aid,
+                                                                     const int32_t *__restrict__ pi, const int32_t *__restrict__ loaded,
+                                                                     int B, int M, int k, int N, int P, int renormalize, float scale,
+                                                                     int32_t *topk_ids, float *topk_w, int32_t *slot_ids,
+                                                                     int32_t *counts, int *err) {
+    extern __shared__ __align__(16) uint8_t rl_smem[];
+    const int ld = M + 1;                                                   // row stride of the tile, in words
+    float *tile = reinterpret_cast<float *>(rl_smem);                       // [128][M + 1]
+    int32_t *hist_s = reinterpret_cast<int32_t *>(tile + (size_t)kLogitTok * ld);   // [P]
+    int32_t *pi_s = hist_s + P;                                             // [N][M]
+
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int tl = (tid >> 5) * 8 + (lane >> 2), g = lane & 3;              // token inside the tile, expert group
+    const int tok0 = blockIdx.x * kLogitTok;
+    const int rows = min(kLogitTok, B - tok0);
+    const int t = tok0 + tl;
+    {
+        const int mv = M >> 2;                                               // float4 per row
+        const float4 *src = logits + (size_t)tok0 * mv;
+        for (int v0 = tid; v0 < rows * mv; v0 += 4 * (int)blockDim.x) {      // four loads in flight per thread
+            float4 r[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (v0 + u * (int)blockDim.x < rows * mv) r[u] = src[v0 + u * blockDim.x];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int v = v0 + u * blockDim.x;
+                if (v < rows * mv) {
+                    float *d = tile + (size_t)(v / mv) * ld + 4 * (v % mv);
+                    d[0] = r[u].x; d[1] = r[u].y; d[2] = r[u].z; d[3] = r[u].w;
+                }
+            }
+        }
+    }
+    for (int i = tid; i < P; i += blockDim.x) hist_s[i] = 0;
+    for (int i = tid; i < N * M; i += blockDim.x) pi_s[i] = pi[i];
+    __syncthreads();
+
+    constexpr unsigned kFull = 0xffffffffu;
+    const bool live = tl < rows;
+    float p[EPT];                                                            // register i: expert EPT*g + i
+    float mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < EPT; ++i) {
+        const int j = EPT * g + i;
+        p[i] = (live && j < M) ? tile[(size_t)tl * ld + j] : -INFINITY;
+        mx = fmaxf(mx, p[i]);
+    }
+    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 2));
+    if (!live) mx = 0.f;
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < EPT; ++i) {                                          // exp(-inf) = 0 for the absent experts
+        p[i] = expf(p[i] - mx);
+        sum += p[i];
+    }
+    sum += __shfl_xor_sync(kFull, sum, 1);                                   // (s0 + s1) + (s2 + s3) on all four lanes
+    sum += __shfl_xor_sync(kFull, sum, 2);
+    const float inv_sum = live ? 1.f / sum : 0.f;
+#pragma unroll
+    for (int i = 0; i < EPT; ++i) p[i] = EPT * g + i < M ? p[i] * inv_sum : -1.f;
+    int a = -1;
+    if (live) {
+        a = aid[t];
+        if (a < -1 || a >= N || (a >= 0 && !loaded[a])) {
+            atomicOr(err, 1);
+            a = -1;
+        }
+    }
+    float wsum = 0.f;
+    float my_w[8];                                                           // weights of the pairs this lane writes (r = g, g+4, ...)
+    for (int r = 0; r < k; ++r) {
+        float bv = -1.f;
+        int bi = 0;
+#pragma unroll
+        for (int i = 0; i < EPT; ++i) {                                      // strict >: the lower index keeps a tie
+            const bool gt = p[i] > bv;
+            bv = gt ? p[i] : bv;
+            bi = gt ? i : bi;
+        }
+        float wv = bv;
+        int wi = EPT * g + bi;
+#pragma unroll
+        for (int o = 1; o <= 2; o <<= 1) {                                   // the four lanes agree on the token's best
+            const float ov = __shfl_xor_sync(kFull, wv, o);
+            const int oi = __shfl_xor_sync(kFull, wi, o);
+            const bool better = ov > wv || (ov == wv && oi < wi);
+            wv = better ? ov : wv;
+            wi = better ? oi : wi;
+        }
+        if (wi == EPT * g + bi) {                                            // mine: taken (probabilities are >= 0)
+#pragma unroll
+            for (int i = 0; i < EPT; ++i) p[i] = (i == bi) ? -1.f : p[i];
+        }
+        wsum += wv;
+        if ((r & 3) == g && live) {                                          // the four lanes share the output work
+            const int slot = a < 0 ? wi : pi_s[a * M + wi];
+            const size_t o = (size_t)t * k + r;
+            topk_ids[o] = wi;
+            slot_ids[o] = slot;
+            atomicAdd(hist_s + slot, 1);
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (u == (r >> 2)) my_w[u] = wv;
+        }
+    }
+    if (live) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (g + 4 * u < k) {
+                float w = my_w[u];
+                if (renormalize) w = w / wsum;
+                topk_w[(size_t)t * k + g + 4 * u] = (renormalize || scale != 1.f) ? w * scale : w;
+            }
+    }
+    __syncthreads();
+    for (int i = tid; i < P; i += blockDim.x)
+        if (hist_s[i]) atomicAdd(counts + i, hist_s[i]);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Scan + permute + plan.  Every CTA recomputes the exclusive scan of the (small) count array in
 // shared memory; the first kPlanners CTAs publish the offsets and write the GEMM work items (the item
 // loop is a chain of dependent integer arithmetic, so it is spread over several CTAs), the other CTAs record for
@@ -303,6 +438,29 @@ int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
     return launch_pdl(4, combine_kernel, dim3(B), dim3(256), 0, st, (const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B, c.top_k,
                       c.hidden, c.num_shared, (uint2 *)out, p->ws.counts, p->P);
+}
+
+int launch_route_logits(ew_pool *p, int layer, const float *logits, const int32_t *aid, int B, int32_t *topk_ids,
+                        float *topk_w, int32_t *slot_ids, int32_t *counts, cudaStream_t st) {
+    const ew_config_t &c = p->cfg;
+    const int M = c.num_experts, N = c.max_adapters;
+    const size_t smem = ((size_t)kLogitTok * (M + 1) + p->P + (size_t)N * M) * 4;
+    if (smem > 227 * 1024) return (int)cudaErrorInvalidConfiguration;
+    const int grid = (B + kLogitTok - 1) / kLogitTok;
+    const int32_t *pi = p->layers[layer].pi_dev;
+    cudaError_t e;
+    if (M <= 64) {
+        e = cudaFuncSetAttribute(route_logits_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+        route_logits_kernel<16><<<grid, 4 * kLogitTok, smem, st>>>((const float4 *)logits, aid, pi, p->ws.loaded, B, M, c.top_k, N, p->P, c.renormalize,
+                                                                   c.routed_scale, topk_ids, topk_w, slot_ids, counts, p->ws.err);
+    } else {
+        e = cudaFuncSetAttribute(route_logits_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+        route_logits_kernel<64><<<grid, 4 * kLogitTok, smem, st>>>((const float4 *)logits, aid, pi, p->ws.loaded, B, M, c.top_k, N, p->P, c.renormalize,
+                                                                   c.routed_scale, topk_ids, topk_w, slot_ids, counts, p->ws.err);
+    }
+    return (int)cudaGetLastError();
 }
 
 int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid, int B, int32_t *slots,

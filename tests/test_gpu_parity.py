@@ -170,6 +170,62 @@ def test_reroute_operator_c4_sample():
     pool.destroy()
 
 
+@pytest.mark.parametrize("M,k,n,renorm", [(64, 6, 65536, 0), (64, 6, 4099, 1), (16, 2, 130, 0), (80, 3, 1000, 0),
+                                          (256, 8, 777, 1), (4, 4, 33, 0)])
+def test_route_from_logits(M, k, n, renorm):
+    """Softmax + top-k + rerouting + counts from given fp32 logits (the c4 recipe: N(0,1) logits, adapter ids per
+    token): ids equal the oracle's except where the k-th and (k+1)-th probabilities are within rounding of each other,
+    weights to 2e-6 relative (same logits, different summation order), slots and counts bit-exact given the ids."""
+    import torch
+    N, e_max = 5, 3
+    rng = np.random.default_rng(100 + M + k)
+    logits = rng.standard_normal((n, M)).astype(np.float32)
+    aid = rng.integers(-1, N, size=n).astype(np.int32)
+    scale = 1.5 if renorm else 1.0
+    pool = binding.Pool(hidden=64, inter=64, num_experts=M, num_shared=0, top_k=k, max_adapters=N, e_max=e_max,
+                        max_tokens=8, renormalize=renorm, routed_scale=scale)
+    z = np.zeros((M, 64, 64), np.uint16)
+    pool.load_base(0, np.zeros((M, 64), np.uint16), z, z, z)
+    tuned = [np.sort(rng.choice(M, size=min(e_max, M), replace=False)).astype(np.int32) for _ in range(N - 1)]
+    for i, ts in enumerate(tuned):                       # the last adapter stays unloaded
+        za = np.zeros((len(ts), 64, 64), np.uint16)
+        pool.load_adapter(i, np.array([len(ts)], np.int32), ts, za, za, za)
+    aid_loaded = np.where(aid == N - 1, -1, aid).astype(np.int32)
+    oc = oracle.OracleConfig(64, 64, M, 0, k, N, e_max)
+    oc.renormalize, oc.routed_scale = renorm, scale
+    ids_o, w_o, gap = oracle.topk_from_logits(oc, logits)
+    Pi = oracle.build_map(M, N, e_max, tuned + [np.zeros(0, np.int32)])
+    ids, w, slots, cnt = pool.route_logits(0, to_dev(logits), to_dev(aid_loaded))
+    torch.cuda.synchronize()
+    assert pool.last_device_error() == 0
+    ids, w, slots, cnt = ids.cpu().numpy(), w.cpu().numpy(), slots.cpu().numpy(), cnt.cpu().numpy()
+    same = (ids == ids_o).all(axis=1)
+    assert np.all(gap[~same] < 1e-6), "a routing decision differs where the probabilities are not tied"
+    assert (~same).sum() <= max(1, n // 1000)
+    assert np.allclose(w[same], w_o[same], rtol=2e-6, atol=1e-9)
+    assert np.array_equal(slots, oracle.reroute(ids, aid_loaded, Pi))
+    assert np.array_equal(cnt, oracle.counts(slots, M + N * e_max))
+    # an unloaded adapter's id behaves as -1 and raises the error word; so does an id out of range
+    aid_bad = aid.copy()
+    aid_bad[0] = N + 3
+    ids2, w2, slots2, cnt2 = pool.route_logits(0, to_dev(logits), to_dev(aid_bad))
+    torch.cuda.synchronize()
+    assert pool.last_device_error() in (1, 8)
+    assert np.array_equal(ids2.cpu().numpy(), ids)
+    bad_rows = (aid_bad == N - 1) | (aid_bad == N + 3)
+    assert np.array_equal(slots2.cpu().numpy()[bad_rows], ids[bad_rows])
+    # empty batch: counts zeroed, nothing else touched
+    e_ids, e_w, e_slots, e_cnt = pool.route_logits(0, to_dev(logits[:0]), to_dev(aid[:0]))
+    torch.cuda.synchronize()
+    assert int(e_cnt.sum()) == 0
+    # logits that are not 16-byte aligned are refused
+    if M % 4 == 0 and n > 1:
+        shifted = torch.zeros(n * M + 1, dtype=torch.float32, device="cuda")[1:].view(n, M)
+        with pytest.raises(binding.EwError):
+            pool.route_logits(0, shifted, to_dev(aid_loaded))
+    pool.destroy()
+
+
 def test_c2_prefill_layer():
     """8192 tokens, 20 adapters: routing checked for every token, the layer output on a seeded sample."""
     cfg = wl.CONFIGS["c2"]

@@ -26,6 +26,10 @@ sys.path.insert(0, ROOT)
 # DRAM bytes (read + write) per launch of the dominant kernel from the committed ncu captures
 # (profiles/c1_decode_grouped_gemm_full.md); reported beside the algorithmic bytes, not used in any ratio.
 NCU_TRAFFIC_BYTES = {"c1": 1.1529e9}
+# route_logits_kernel at the c4 shape: thread instructions per token from one ncu capture (smsp__inst_executed x 32 /
+# tokens, profiles/c4_reroute_operator.md), and the issue peak of the GPU
+ALU_INSTR_PER_TOKEN_C4 = 215 * 32
+ALU_PEAK_TINSTR = 148 * 4 * 32 * 1.965e9 / 1e12
 
 METRIC = "adapter-aware MoE layer tokens/s"
 UNIT = "tokens/s"
@@ -374,8 +378,13 @@ def run_reroute(args):
                   "ms_per_launch": ms, "tokens": Bt, "tokens_per_s": Bt / (ms * 1e-3), "dtype": "f32", "data": "synthetic",
                   "config": {"workload": f"c4: softmax + top-k + reroute + counts from fp32 logits, {Bt} tokens, 20 adapters x 32 of 64 experts",
                              "l2": f"cold: {n_sets} rotating buffer sets", "includes": "zeroing of counts + kernel"},
-                  "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                               "of": peak_kind, "algorithmic_bytes": nbytes, "traffic": None}})
+                  # bound by arithmetic (softmax + k selection rounds over M probabilities), not by memory: ncu counts 215
+                  # warp instructions per token (M = 64, k = 6); peak = 148 SMs x 4 schedulers x 32 lanes x 1.965 GHz
+                  "roofline": {"bound": "alu", "achieved": Bt / (ms * 1e-3) * ALU_INSTR_PER_TOKEN_C4 / 1e12, "peak": ALU_PEAK_TINSTR,
+                               "unit": "T thread-instructions/s", "of": "derived: SM count x issue slots x lanes x max clock",
+                               "frac": Bt / (ms * 1e-3) * ALU_INSTR_PER_TOKEN_C4 / 1e12 / ALU_PEAK_TINSTR,
+                               "instructions_per_token": ALU_INSTR_PER_TOKEN_C4, "hbm_gbs": gbs, "hbm_frac": gbs / peak,
+                               "algorithmic_bytes": nbytes, "traffic": None}})
     sweep = []
     for lg in (() if args.tokens else (16, 18, 20, 22)):
         nb_, ms_, _ = measure_logits(1 << lg, max(20, args.steps >> max(0, lg - 16)))

@@ -245,14 +245,27 @@ __global__ void __launch_bounds__(4 * kLogitTok) route_logits_kernel(const float
     float wsum = 0.f;
     float my_w[8];                                                           // weights of the pairs this lane writes (r = g, g+4, ...)
     for (int r = 0; r < k; ++r) {
-        float bv = -1.f;
-        int bi = 0;
+        // arg-max as a tree over neighbouring ranges (short dependency chains); the right half wins only if
+        // strictly greater, so the lower index keeps a tie
+        float tv[EPT / 2];
+        int ti[EPT / 2];
 #pragma unroll
-        for (int i = 0; i < EPT; ++i) {                                      // strict >: the lower index keeps a tie
-            const bool gt = p[i] > bv;
-            bv = gt ? p[i] : bv;
-            bi = gt ? i : bi;
+        for (int i = 0; i < EPT / 2; ++i) {
+            const bool gt = p[2 * i + 1] > p[2 * i];
+            tv[i] = gt ? p[2 * i + 1] : p[2 * i];
+            ti[i] = gt ? 2 * i + 1 : 2 * i;
         }
+#pragma unroll
+        for (int w = EPT / 4; w >= 1; w >>= 1) {
+#pragma unroll
+            for (int i = 0; i < w; ++i) {
+                const bool gt = tv[2 * i + 1] > tv[2 * i];
+                tv[i] = gt ? tv[2 * i + 1] : tv[2 * i];
+                ti[i] = gt ? ti[2 * i + 1] : ti[2 * i];
+            }
+        }
+        const float bv = tv[0];
+        const int bi = ti[0];
         float wv = bv;
         int wi = EPT * g + bi;
 #pragma unroll

@@ -417,10 +417,30 @@ def test_adapter_churn_under_load():
 @pytest.mark.parametrize("renorm", [0, 1])
 def test_odd_shapes(shape, renorm):
     """Shapes off every tile size, degenerate top-k, no shared experts, renormalised and scaled weights."""
+    check_shape(shape, renorm, seed=21)
+
+
+def _random_shape(rng):
+    M = int(rng.choice([2, 3, 5, 8, 12, 16, 24, 33, 48, 64, 72, 100]))
+    return dict(hidden=64 * int(rng.integers(1, 7)), inter=8 * int(rng.integers(1, 40)), num_experts=M,
+                num_shared=int(rng.integers(0, 3)), top_k=int(rng.integers(1, min(M, 8) + 1)),
+                max_adapters=int(rng.integers(1, 5)), e_max=int(rng.integers(1, min(M, 5) + 1)),
+                n_tokens=int(rng.choice([1, 3, 17, 32, 33, 63, 64, 100, 129, 257, 600, 1100])))
+
+
+@pytest.mark.parametrize("case", range(32))
+def test_random_shapes(case):
+    """Seeded random layer shapes and batch sizes (sizes, expert counts, top-k, shared experts, adapters all drawn
+    independently), each checked against the oracle like the hand-picked ones above."""
+    rng = np.random.default_rng(1000 + case)
+    check_shape(_random_shape(rng), renorm=case % 2, seed=1000 + case)
+
+
+def check_shape(shape, renorm, seed):
     import torch
-    cfg = wl.MoEConfig(name="odd", num_layers=1, seed=21, **shape)
+    cfg = wl.MoEConfig(name="odd", num_layers=1, seed=seed, **shape)
     bank = wl.NoiseBank(cfg.seed)
-    rng = np.random.default_rng(21)
+    rng = np.random.default_rng(seed)
     scale = 2.5 if renorm else 1.0
     pool = binding.Pool.from_config(cfg, renormalize=renorm, routed_scale=scale)
     counts = rng.integers(0, cfg.e_max + 1, size=(cfg.max_adapters, 1))

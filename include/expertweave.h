@@ -109,7 +109,10 @@ ew_status_t ew_load_base(ew_pool_t *pool, int32_t layer, const void *router_w, c
  *   counts      host int32 [L]: e_i^(l), experts the adapter re-tunes in layer l (0 allowed)
  *   expert_ids  host int32 [sum counts]: per layer, strictly ascending base expert ids in [0,M);
  *               the r-th id of a layer gets delta = r, i.e. slot M + adapter_id*E_max + r
- *   w_gate,w_up host bf16 [sum counts, I, H];  w_down host bf16 [sum counts, H, I], same order
+ *   w_gate,w_up bf16 [sum counts, I, H];  w_down bf16 [sum counts, H, I], same order.  The weight
+ *               pointers may be host memory (page-locked memory copies at the host link's speed) or
+ *               device memory (an adapter kept resident outside the pool): the copy follows unified
+ *               addressing.  The same holds for the weight pointers of ew_load_base.
  * For each layer the byte range of slots [Delta_i, Delta_i + e) is backed by pages taken from the
  * pool's free list (or created); a page shared with a neighbouring adapter is mapped once and
  * reference-counted (sub-page allocation).  Weights are copied, then row adapter_id of every layer's

@@ -291,18 +291,19 @@ extern "C" ew_status_t ew_pool_trim(ew_pool_t *p) {
 
 // Copy e experts' gate and up blocks into slots [first, first+e) of the fused tensor, and the down
 // blocks into the down tensor.  Source layout: [e, I, H], [e, I, H], [e, H, I].
+// Weight sources may be host (pageable or page-locked) or device memory: the copy kind is left to unified addressing.
 static ew_status_t copy_gate_up(ew_pool *p, LayerState &L, size_t first, size_t e, const void *g, const void *u) {
     if (e == 0 || p->cfg.device < 0) return EW_OK;
     size_t blk = (size_t)p->cfg.inter * p->cfg.hidden * 2;
     char *dst13 = (char *)L.w13.slot_addr(first);
-    CU_TRY(cudaMemcpy2DAsync(dst13, 2 * blk, g, blk, blk, e, cudaMemcpyHostToDevice, p->copy_stream));
-    CU_TRY(cudaMemcpy2DAsync(dst13 + blk, 2 * blk, u, blk, blk, e, cudaMemcpyHostToDevice, p->copy_stream));
+    CU_TRY(cudaMemcpy2DAsync(dst13, 2 * blk, g, blk, blk, e, cudaMemcpyDefault, p->copy_stream));
+    CU_TRY(cudaMemcpy2DAsync(dst13 + blk, 2 * blk, u, blk, blk, e, cudaMemcpyDefault, p->copy_stream));
     return EW_OK;
 }
 static ew_status_t copy_down(ew_pool *p, LayerState &L, size_t first, size_t e, const void *d) {
     if (e == 0 || p->cfg.device < 0) return EW_OK;
     size_t blk = (size_t)p->cfg.inter * p->cfg.hidden * 2;
-    CU_TRY(cudaMemcpyAsync((void *)L.w2.slot_addr(first), d, blk * e, cudaMemcpyHostToDevice, p->copy_stream));
+    CU_TRY(cudaMemcpyAsync((void *)L.w2.slot_addr(first), d, blk * e, cudaMemcpyDefault, p->copy_stream));
     return EW_OK;
 }
 static ew_status_t copy_experts(ew_pool *p, LayerState &L, size_t first, size_t e, const void *g, const void *u,
@@ -339,7 +340,7 @@ extern "C" ew_status_t ew_load_base(ew_pool_t *p, int32_t layer, const void *rou
     if (gpu) {
         // forwards in flight may still read the old weights of this layer
         for (auto &e : p->fwd_events) CU_TRY(cudaEventSynchronize(e.second));
-        CU_TRY(cudaMemcpyAsync(L.router_w, router_w, M * c.hidden * 2, cudaMemcpyHostToDevice, p->copy_stream));
+        CU_TRY(cudaMemcpyAsync(L.router_w, router_w, M * c.hidden * 2, cudaMemcpyDefault, p->copy_stream));
         ew_status_t st = copy_experts(p, L, 0, M, w_gate, w_up, w_down);
         if (st == EW_OK && S) st = copy_experts(p, L, P, S, sh_gate, sh_up, sh_down);
         if (st != EW_OK) return st;

@@ -124,6 +124,33 @@ def test_load_unload_on_device():
     pool.destroy()
 
 
+def test_adapter_weights_from_device_memory():
+    """ew_load_adapter takes its weights from device memory as well as from host memory: same forward either way."""
+    import ctypes as C
+    import torch
+    cfg = wl.CONFIGS["c0"]
+    bank = wl.NoiseBank(cfg.seed)
+    pool = binding.Pool.from_config(cfg)
+    binding.load_model(pool, cfg, bank)
+    x, aid = to_dev(wl.gen_tokens(cfg)), to_dev(wl.gen_adapter_ids(cfg))
+    ref = pool.moe_forward(0, x, aid).clone()
+    torch.cuda.synchronize()
+    tuned = wl.tuned_sets(cfg)
+    ew = wl.gen_adapter_layer(cfg, 1, 0, tuned[1][0], bank)
+    pool.unload_adapter(1)
+    dev = [torch.from_numpy(a.view(np.int16)).cuda() for a in (ew.w_gate, ew.w_up, ew.w_down)]
+    counts = np.array([len(tuned[1][0])], np.int32)
+    ids = np.ascontiguousarray(tuned[1][0], np.int32)
+    rc = binding.lib().ew_load_adapter(pool._h, 1, counts.ctypes.data_as(C.c_void_p), ids.ctypes.data_as(C.c_void_p),
+                                       C.c_void_p(dev[0].data_ptr()), C.c_void_p(dev[1].data_ptr()),
+                                       C.c_void_p(dev[2].data_ptr()))
+    assert rc == 0
+    out = pool.moe_forward(0, x, aid)
+    torch.cuda.synchronize()
+    assert torch.equal(out, ref)
+    pool.destroy()
+
+
 def test_reroute_operator_c4_sample():
     """The rerouting operator alone: slot ids and per-slot counts are bit-exact."""
     import torch

@@ -135,11 +135,12 @@ class Pool:
         _check(lib().ew_load_base(self._h, layer, *[_hp(a) for a in arrs]), "ew_load_base")
 
     def load_adapter(self, adapter_id, counts, expert_ids, w_gate, w_up, w_down):
+        """Weights: numpy arrays of bf16 bit patterns (host), or torch tensors (host or device) taken as they are."""
         counts = _host(counts, np.int32)
         expert_ids = _host(expert_ids, np.int32)
-        g, u, d = _host(w_gate), _host(w_up), _host(w_down)
-        _check(lib().ew_load_adapter(self._h, adapter_id, _hp(counts), _hp(expert_ids), _hp(g), _hp(u), _hp(d)),
-               "ew_load_adapter")
+        keep = [a if hasattr(a, "data_ptr") else _host(a) for a in (w_gate, w_up, w_down)]   # alive during the call
+        g, u, d = [_dp(a) if hasattr(a, "data_ptr") else _hp(a) for a in keep]
+        _check(lib().ew_load_adapter(self._h, adapter_id, _hp(counts), _hp(expert_ids), g, u, d), "ew_load_adapter")
 
     def unload_adapter(self, adapter_id):
         _check(lib().ew_unload_adapter(self._h, adapter_id), "ew_unload_adapter")

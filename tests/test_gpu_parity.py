@@ -126,7 +126,6 @@ def test_load_unload_on_device():
 
 def test_adapter_weights_from_device_memory():
     """ew_load_adapter takes its weights from device memory as well as from host memory: same forward either way."""
-    import ctypes as C
     import torch
     cfg = wl.CONFIGS["c0"]
     bank = wl.NoiseBank(cfg.seed)
@@ -139,12 +138,7 @@ def test_adapter_weights_from_device_memory():
     ew = wl.gen_adapter_layer(cfg, 1, 0, tuned[1][0], bank)
     pool.unload_adapter(1)
     dev = [torch.from_numpy(a.view(np.int16)).cuda() for a in (ew.w_gate, ew.w_up, ew.w_down)]
-    counts = np.array([len(tuned[1][0])], np.int32)
-    ids = np.ascontiguousarray(tuned[1][0], np.int32)
-    rc = binding.lib().ew_load_adapter(pool._h, 1, counts.ctypes.data_as(C.c_void_p), ids.ctypes.data_as(C.c_void_p),
-                                       C.c_void_p(dev[0].data_ptr()), C.c_void_p(dev[1].data_ptr()),
-                                       C.c_void_p(dev[2].data_ptr()))
-    assert rc == 0
+    pool.load_adapter(1, np.array([len(tuned[1][0])], np.int32), tuned[1][0], *dev)
     out = pool.moe_forward(0, x, aid)
     torch.cuda.synchronize()
     assert torch.equal(out, ref)

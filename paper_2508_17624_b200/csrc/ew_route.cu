@@ -191,6 +191,9 @@ __global__ void __launch_bounds__(4 * kLogitTok) route_logits_kernel(const float
     {
         const int mv = M >> 2;                                               // float4 per row
         const float4 *src = logits + (size_t)tok0 * mv;
+        // (row, column) of this thread's float4 and of the one blockDim further: one division here, additions below
+        int row = tid / mv, col = tid - row * mv;
+        const int drow = (int)blockDim.x / mv, dcol = (int)blockDim.x - drow * mv;
         for (int v0 = tid; v0 < rows * mv; v0 += 4 * (int)blockDim.x) {      // four loads in flight per thread
             float4 r[4];
 #pragma unroll
@@ -198,11 +201,13 @@ __global__ void __launch_bounds__(4 * kLogitTok) route_logits_kernel(const float
                 if (v0 + u * (int)blockDim.x < rows * mv) r[u] = src[v0 + u * blockDim.x];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const int v = v0 + u * blockDim.x;
-                if (v < rows * mv) {
-                    float *d = tile + (size_t)(v / mv) * ld + 4 * (v % mv);
+                if (v0 + u * (int)blockDim.x < rows * mv) {
+                    float *d = tile + (size_t)row * ld + 4 * col;
                     d[0] = r[u].x; d[1] = r[u].y; d[2] = r[u].z; d[3] = r[u].w;
                 }
+                row += drow;
+                col += dcol;
+                if (col >= mv) { col -= mv; ++row; }
             }
         }
     }

@@ -20,7 +20,7 @@ _lib = None
 class _Cfg(C.Structure):
     _fields_ = [("H", C.c_int32), ("I", C.c_int32), ("M", C.c_int32), ("S", C.c_int32), ("k", C.c_int32),
                 ("N", C.c_int32), ("E_max", C.c_int32), ("renormalize", C.c_int32),
-                ("routed_scale", C.c_float), ("round_h_bf16", C.c_int32)]
+                ("routed_scale", C.c_float)]
 
 
 _U16P = C.POINTER(C.c_uint16)
@@ -29,7 +29,7 @@ _I32P = C.POINTER(C.c_int32)
 
 class _Layer(C.Structure):
     _fields_ = [("router_w", _U16P), ("w_gate", _U16P), ("w_up", _U16P), ("w_down", _U16P),
-                ("s_gate", _U16P), ("s_up", _U16P), ("s_down", _U16P), ("e", _I32P),
+                ("s_gate", _U16P), ("s_up", _U16P), ("s_down", _U16P), ("e", _I32P), ("loaded", _I32P),
                 ("tuned", C.POINTER(_I32P)), ("a_gate", C.POINTER(_U16P)), ("a_up", C.POINTER(_U16P)),
                 ("a_down", C.POINTER(_U16P))]
 
@@ -67,11 +67,10 @@ class OracleConfig:
     E_max: int
     renormalize: int = 0
     routed_scale: float = 1.0
-    round_h_bf16: int = 0
 
     def c(self) -> _Cfg:
         return _Cfg(self.H, self.I, self.M, self.S, self.k, self.N, self.E_max, self.renormalize,
-                    self.routed_scale, self.round_h_bf16)
+                    self.routed_scale)
 
     @property
     def P(self) -> int:
@@ -99,6 +98,7 @@ class OracleLayer:
         adapters = list(adapters) if adapters is not None else [None] * N
         assert len(adapters) == N
         self.e = np.zeros(N, np.int32)
+        self.loaded = np.array([0 if a is None else 1 for a in adapters], np.int32)
         tuned_p = (_I32P * N)()
         ag, au, ad = (_U16P * N)(), (_U16P * N)(), (_U16P * N)()
         self.tuned: List[np.ndarray] = []
@@ -120,6 +120,7 @@ class OracleLayer:
                 arr_p[i] = p
         self._keep += [tuned_p, ag, au, ad]
         st.e = self.e.ctypes.data_as(_I32P)
+        st.loaded = self.loaded.ctypes.data_as(_I32P)
         st.tuned = C.cast(tuned_p, C.POINTER(_I32P))
         st.a_gate = C.cast(ag, C.POINTER(_U16P))
         st.a_up = C.cast(au, C.POINTER(_U16P))
@@ -143,14 +144,22 @@ def build_map(M: int, N: int, E_max: int, tuned: Sequence[np.ndarray]) -> np.nda
     return Pi
 
 
-def reroute(ids: np.ndarray, aid: np.ndarray, Pi: np.ndarray) -> np.ndarray:
+def reroute(ids: np.ndarray, aid: np.ndarray, Pi: np.ndarray, loaded: Optional[np.ndarray] = None,
+            return_bad: bool = False):
+    """Slot ids [B,k].  `loaded` [N] marks the adapters that are loaded (default: all); tokens whose adapter id
+    is outside [-1,N) or not loaded are base-model tokens, and `return_bad` also returns how many there were."""
     ids, ip = _i32(ids)
     aid, ap = _i32(aid)
     Pi, pp = _i32(Pi)
     B, k = ids.shape
+    N, M = Pi.shape
+    lp = None
+    if loaded is not None:
+        loaded, lp = _i32(loaded)
+        assert loaded.shape == (N,)
     out = np.empty((B, k), np.int32)
-    lib().ewo_reroute(B, k, Pi.shape[1], ip, ap, pp, out.ctypes.data_as(_I32P))
-    return out
+    bad = lib().ewo_reroute(B, k, M, N, ip, ap, pp, lp, out.ctypes.data_as(_I32P))
+    return (out, int(bad)) if return_bad else out
 
 
 def counts(slots: np.ndarray, P: int) -> np.ndarray:

@@ -13,7 +13,10 @@
  *   ewo_build_map          ESFT expert map, Section 4.1, the two-case definition of Pi^(l)[i,j]
  *                          with Delta_i = M + i*E_max and 0 <= delta < e_i^(l).
  *   ewo_reroute            batched rerouting, Section 4.1: TopK'(x) = { Pi[A(x), j] : j in TopK(x) };
- *                          adapter id -1 marks a base-model token (Section 4.3).
+ *                          adapter id -1 marks a base-model token (Section 4.3).  The paper leaves two
+ *                          inputs undefined: an id outside [-1, N) and the id of an adapter that is not
+ *                          loaded.  Reading taken here: such a token is a base-model token (its ids are
+ *                          kept) and it is counted in the function's return value.
  *   ewo_gate_topk          the router of Section 2.1 (g(x), top-k ids [B,k]); the paper does not fix
  *                          g, so: softmax over all M logits, the k largest probabilities, ties to
  *                          the lower index, weights = the selected probabilities (optionally
@@ -46,7 +49,6 @@ typedef struct {
     int32_t H, I, M, S, k, N, E_max;
     int32_t renormalize;   /* 1: divide the k weights by their sum */
     float routed_scale;    /* multiplies the k weights */
-    int32_t round_h_bf16;  /* debug aid: round the SwiGLU activation to bf16 (not the graded mode) */
 } ewo_cfg;
 
 /* All weights of one layer, as the caller holds them on the host (bf16 bits). */
@@ -54,7 +56,8 @@ typedef struct {
     const uint16_t *router_w;                  /* [M, H] */
     const uint16_t *w_gate, *w_up, *w_down;    /* base routed experts [M,I,H], [M,I,H], [M,H,I] */
     const uint16_t *s_gate, *s_up, *s_down;    /* shared experts      [S,I,H], [S,I,H], [S,H,I] */
-    const int32_t *e;                          /* [N] experts tuned by adapter i in this layer (0 = not loaded) */
+    const int32_t *e;                          /* [N] experts tuned by adapter i in this layer (0 when not loaded) */
+    const int32_t *loaded;                     /* [N] 1 = adapter i is loaded (it may still tune nothing in this layer) */
     const int32_t *const *tuned;               /* [N] -> ascending base expert ids, length e[i] */
     const uint16_t *const *a_gate;             /* [N] -> [e_i, I, H] */
     const uint16_t *const *a_up;               /* [N] -> [e_i, I, H] */
@@ -66,13 +69,6 @@ static inline float bf(uint16_t b) {
     float f;
     memcpy(&f, &u, 4);
     return f;
-}
-
-static inline uint16_t to_bf16(float f) {
-    uint32_t u;
-    memcpy(&u, &f, 4);
-    u += 0x7FFFu + ((u >> 16) & 1u);
-    return (uint16_t)(u >> 16);
 }
 
 int ewo_num_threads(void) {
@@ -98,13 +94,21 @@ int ewo_build_map(int M, int N, int E_max, const int32_t *e, const int32_t *cons
     return 0;
 }
 
-/* slots[t,r] = aid[t] < 0 ? ids[t,r] : Pi[aid[t], ids[t,r]] */
-void ewo_reroute(int B, int k, int M, const int32_t *ids, const int32_t *aid, const int32_t *Pi, int32_t *slots) {
-    for (int t = 0; t < B; ++t)
+/* slots[t,r] = aid[t] == -1 ? ids[t,r] : Pi[aid[t], ids[t,r]].
+ * loaded[i] != 0 marks adapter i as loaded (null = all N loaded).  A token whose id is outside [-1, N) or names
+ * an adapter that is not loaded is treated as a base-model token; the return value counts such tokens. */
+int ewo_reroute(int B, int k, int M, int N, const int32_t *ids, const int32_t *aid, const int32_t *Pi,
+                const int32_t *loaded, int32_t *slots) {
+    int bad = 0;
+    for (int t = 0; t < B; ++t) {
+        int a = aid[t];
+        if (a < -1 || a >= N || (a >= 0 && loaded && !loaded[a])) { a = -1; ++bad; }
         for (int r = 0; r < k; ++r) {
             int j = ids[t * k + r];
-            slots[t * k + r] = aid[t] < 0 ? j : Pi[aid[t] * M + j];
+            slots[t * k + r] = a < 0 ? j : Pi[a * M + j];
         }
+    }
+    return bad;
 }
 
 void ewo_counts(int n_pairs, int P, const int32_t *slots, int32_t *cnt) {
@@ -181,8 +185,7 @@ static void expert_ffn(const ewo_cfg *c, const float *xf, const uint16_t *wg, co
         const uint16_t *rg = wg + (size_t)i * H, *ru = wu + (size_t)i * H;
         for (int h = 0; h < H; ++h) g += bf(rg[h]) * xf[h];
         for (int h = 0; h < H; ++h) u += bf(ru[h]) * xf[h];
-        float a = (g / (1.f + expf(-g))) * u;
-        act[i] = c->round_h_bf16 ? bf(to_bf16(a)) : a;
+        act[i] = (g / (1.f + expf(-g))) * u;
     }
     for (int o = 0; o < H; ++o) {
         float d = 0.f;
@@ -242,7 +245,7 @@ int ewo_layer_forward(const ewo_cfg *c, const ewo_layer *L, int B, const uint16_
     int32_t *slots = ids + n;
     float *w = (float *)malloc(sizeof(float) * n);
     ewo_gate_topk(c, B, x, L->router_w, ids, w, 0, 0);
-    ewo_reroute(B, c->k, c->M, ids, aid, Pi, slots);
+    ewo_reroute(B, c->k, c->M, c->N, ids, aid, Pi, L->loaded, slots);
     int rc = ewo_ffn_given_slots(c, L, B, x, slots, w, out);
     if (ids_out) memcpy(ids_out, ids, sizeof(int32_t) * n);
     if (slots_out) memcpy(slots_out, slots, sizeof(int32_t) * n);
@@ -282,9 +285,4 @@ int ewo_layer_forward_merged(const ewo_cfg *c, const ewo_layer *L, int B, const 
     }
     free(ids); free(w);
     return 0;
-}
-
-/* bf16 rounding of an fp32 buffer (convenience for comparisons) */
-void ewo_round_bf16(size_t n, const float *in, uint16_t *out) {
-    for (size_t i = 0; i < n; ++i) out[i] = to_bf16(in[i]);
 }

@@ -75,6 +75,31 @@ def test_reroute_definition():
             assert cnt[M + i * E_max + d] == 0
 
 
+def test_reroute_bad_and_unloaded_adapter_ids_are_base_tokens():
+    """The paper defines the adapter id as -1 (base model) or an adapter index (Section 4.3) and is silent on
+    anything else.  Reading pinned here: an id outside [-1, N), or the id of an adapter that is not loaded, makes
+    the token a base-model token (ids unchanged) and is counted; nothing is read outside the map.  The expected
+    values are spelled out by hand for a map small enough to check by eye."""
+    M, N, E_max = 4, 3, 2
+    tuned = [np.array([1, 2], np.int32), np.array([0], np.int32), np.array([3], np.int32)]
+    Pi = oracle.build_map(M, N, E_max, tuned)
+    assert Pi.tolist() == [[0, 4, 5, 3], [6, 1, 2, 3], [0, 1, 2, 8]]
+    ids = np.array([[1, 2], [0, 3], [3, 0], [2, 1], [1, 0], [3, 2], [0, 1]], np.int32)
+    aid = np.array([0, 1, 2, -1, 3, -2, 2**30], np.int32)
+    slots, bad = oracle.reroute(ids, aid, Pi, return_bad=True)             # every adapter loaded
+    assert slots.tolist() == [[4, 5], [6, 3], [8, 0], [2, 1], [1, 0], [3, 2], [0, 1]] and bad == 3
+    # adapter 1 not loaded: its token keeps the base ids even though a (stale) row for it exists in the map
+    slots, bad = oracle.reroute(ids, aid, Pi, loaded=np.array([1, 0, 1], np.int32), return_bad=True)
+    assert slots.tolist() == [[4, 5], [0, 3], [8, 0], [2, 1], [1, 0], [3, 2], [0, 1]] and bad == 4
+    # a large negative id is not an index into the map either
+    slots, bad = oracle.reroute(ids[:1], np.array([-2**31], np.int32), Pi, return_bad=True)
+    assert slots.tolist() == [[1, 2]] and bad == 1
+    # with the ids rewritten to -1 by hand the result is the same and nothing is counted
+    fixed = np.where((aid < -1) | (aid >= N), -1, aid).astype(np.int32)
+    slots2, bad2 = oracle.reroute(ids, fixed, Pi, return_bad=True)
+    assert bad2 == 0 and np.array_equal(slots2, oracle.reroute(ids, aid, Pi))
+
+
 def test_build_map_rejects_bad_lists():
     with pytest.raises(ValueError):
         oracle.build_map(8, 1, 2, [np.array([1, 2, 3], np.int32)])      # e > E_max
@@ -171,6 +196,18 @@ def test_base_only_and_identical_copies():
     clone = oracle.OracleLayer(cfg, **base, adapters=same)
     o, _, _, slots = oracle.layer_forward(clone, x, aid)
     assert np.array_equal(o, base_out) and (slots >= cfg.M).any()
+    # an adapter that is not loaded: its tokens (and tokens with an id past N) are base tokens, whether the map
+    # holds an identity row for it or a stale one; the merged-model path agrees
+    part = oracle.OracleLayer(cfg, **base, adapters=[adapters[0], None])
+    aid_bad = aid.copy()
+    aid_bad[0] = cfg.N + 5
+    want = np.where((aid_bad == 1) | (aid_bad >= cfg.N), -1, aid_bad).astype(np.int32)
+    o_want, *_ = oracle.layer_forward(full, x, want)
+    for Pi in (None, full.build_map()):
+        o, _, _, slots = oracle.layer_forward(part, x, aid_bad, Pi)
+        assert np.array_equal(o, o_want)
+        assert (slots[(aid_bad == 1) | (aid_bad >= cfg.N)] < cfg.M).all()
+    assert np.array_equal(oracle.layer_forward_merged(part, x, aid_bad), o_want)
     # adapter copies that differ change exactly the tokens whose routed set meets the tuned set
     o, ids, _, slots = oracle.layer_forward(full, x, aid)
     touched = (slots >= cfg.M).any(axis=1)

@@ -6,7 +6,7 @@ import oracle
 from paper_2508_17624_b200 import binding, build
 from paper_2508_17624_b200 import workloads as wl
 
-from helpers import bf16_to_f32, check_output, check_routing, oracle_layer, to_dev
+from helpers import WEIGHT_RTOL, bf16_to_f32, check_output, check_routing, oracle_layer, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -19,21 +19,39 @@ def _built():
     binding.lib()
 
 
+def edge_tokens(r, n_extra, seed):
+    """Tokens that own the first and the last row of every live slot's chunk (so that every slot's first and last
+    token block, ragged tails included, is compared), plus `n_extra` seeded random ones."""
+    inv = r["inv"].cpu().numpy()
+    off = r["offsets"].cpu().numpy()
+    B, k = inv.shape
+    row_tok = np.empty(B * k, np.int64)
+    row_tok[inv.reshape(-1)] = np.repeat(np.arange(B), k)
+    live = np.nonzero(off[1:] > off[:-1])[0]
+    picks = set(row_tok[off[live]].tolist()) | set(row_tok[off[live + 1] - 1].tolist())
+    picks |= set(np.random.default_rng(seed).choice(B, size=min(B, n_extra), replace=False).tolist())
+    return np.array(sorted(picks))
+
+
 def run_layer(cfg, layer=0, n_tokens=None, aid_mode=None, adapters=None, sample=None, pool=None, bank=None,
-              tuned=None, bases=None):
+              tuned=None, bases=None, **pool_kw):
+    """One debug forward against the oracle.  `sample`: None = the output of every token is compared; an index
+    array; or a function of the debug results that returns one."""
     import torch
     bank = bank or wl.NoiseBank(cfg.seed)
     own = pool is None
     if own:
-        pool = binding.Pool.from_config(cfg, max_tokens=n_tokens or cfg.n_tokens)
+        pool = binding.Pool.from_config(cfg, max_tokens=n_tokens or cfg.n_tokens, **pool_kw)
         tuned, bases = binding.load_model(pool, cfg, bank, adapters=adapters)
-    olayer = oracle_layer(cfg, layer, bank, tuned, base=bases[layer], adapters=adapters)
+    olayer = oracle_layer(cfg, layer, bank, tuned, base=(bases or {}).get(layer), adapters=adapters)
     x = wl.gen_tokens(cfg, layer, n_tokens)
     aid = wl.gen_adapter_ids(cfg, n_tokens, aid_mode)
     r = pool.moe_forward_debug(layer, to_dev(x), to_dev(aid))
     torch.cuda.synchronize()
     assert pool.last_device_error() == 0
     ids, w, slots, flips = check_routing(cfg, olayer, x, aid, r)
+    if callable(sample):
+        sample = sample(r)
     rel, mx = check_output(olayer, x, slots, w, bf16_to_f32(r["out"]), sample)
     # the plain entry point gives the same bits as the debug one
     out2 = pool.moe_forward(layer, to_dev(x), to_dev(aid))
@@ -41,7 +59,8 @@ def run_layer(cfg, layer=0, n_tokens=None, aid_mode=None, adapters=None, sample=
     assert torch.equal(out2, r["out"])
     if own:
         pool.destroy()
-    return dict(flips=flips, rel=rel, max_abs=mx, slots=slots, out=r["out"])
+    return dict(flips=flips, rel=rel, max_abs=mx, slots=slots, out=r["out"],
+                n_checked=x.shape[0] if sample is None else len(sample))
 
 
 def test_c0_tiny_layer():
@@ -85,15 +104,32 @@ def test_zero_tokens_and_errors():
     with pytest.raises(binding.EwError):
         pool.moe_forward(0, torch.zeros((cfg.n_tokens + 1, cfg.hidden), dtype=torch.bfloat16, device="cuda"),
                          torch.zeros(cfg.n_tokens + 1, dtype=torch.int32, device="cuda"))
-    # adapter 1 is not loaded and 5 is out of range: both behave as base tokens and raise the device flag
-    xb = to_dev(wl.gen_tokens(cfg, 0, 4))
-    bad = pool.moe_forward(0, xb, torch.tensor([1, 5, -7, -1], dtype=torch.int32, device="cuda"))
+    pool.destroy()
+
+
+def test_bad_and_unloaded_adapter_ids_against_the_oracle():
+    """Adapter 1 is not loaded, 5 and 2^30 are past N, -7 is below -1: the oracle's reading makes all of them base
+    tokens; the GPU must give the oracle's slots, counts and output for them and raise its flag."""
+    import torch
+    cfg = wl.CONFIGS["c0"]
+    bank = wl.NoiseBank(cfg.seed)
+    pool = binding.Pool.from_config(cfg)
+    tuned, bases = binding.load_model(pool, cfg, bank, adapters=[0])
+    olayer = oracle_layer(cfg, 0, bank, tuned, base=bases[0], adapters=[0])
+    x = wl.gen_tokens(cfg)
+    aid = np.resize(np.array([1, 5, -7, -1, 0, 2**30, 0, 1, -2**31, 0], np.int32), cfg.n_tokens)
+    r = pool.moe_forward_debug(0, to_dev(x), to_dev(aid))
     torch.cuda.synchronize()
     assert pool.last_device_error() == 8
-    good = pool.moe_forward(0, xb, torch.full((4,), -1, dtype=torch.int32, device="cuda"))
+    ids, w, slots, _ = check_routing(cfg, olayer, x, aid, r)
+    check_output(olayer, x, slots, w, bf16_to_f32(r["out"]))
+    _, n_bad = oracle.reroute(ids, aid, olayer.build_map(), loaded=olayer.loaded, return_bad=True)
+    assert n_bad == int(((aid != 0) & (aid != -1)).sum()) > 30
+    assert (slots[aid == 0] >= cfg.num_experts).any() and (slots[aid != 0] < cfg.num_experts).all()
+    good = pool.moe_forward(0, to_dev(x), to_dev(np.where(aid == 0, 0, -1).astype(np.int32)))
     torch.cuda.synchronize()
     assert pool.last_device_error() == 0
-    assert torch.equal(bad, good)
+    assert torch.equal(r["out"], good)
     pool.destroy()
 
 
@@ -188,6 +224,29 @@ def test_reroute_operator_c4_sample():
     assert int(slots3[5, 2]) == cfg.num_experts + 7
     assert torch.equal(slots3[9], bad_ids[9])
     assert pool.last_device_error() in (1, 8)
+    # bad adapter ids against the oracle's reading (base tokens), with counts; adapter 3 evicted = not loaded
+    pool.unload_adapter(3)
+    loaded = np.ones(cfg.max_adapters, np.int32)
+    loaded[3] = 0
+    aid4 = aid.copy()
+    aid4[[0, 17, 4098]] = [cfg.max_adapters, -5, 2**30]
+    Pi4 = pool.get_expert_map(0)
+    assert np.array_equal(Pi4[3], np.arange(cfg.num_experts))
+    slots4, cnt4 = pool.reroute(0, to_dev(ids), to_dev(aid4))
+    torch.cuda.synchronize()
+    want4, n_bad = oracle.reroute(ids, aid4, Pi, loaded=loaded, return_bad=True)     # Pi: the stale map, row 3 included
+    assert n_bad == 3 + int((aid4 == 3).sum())
+    assert np.array_equal(slots4.cpu().numpy(), want4)
+    assert np.array_equal(cnt4.cpu().numpy(), oracle.counts(want4, cfg.num_slots))
+    assert pool.last_device_error() == 8
+    # in place, on a batch whose pair count is not a multiple of four (vector body + scalar tail on the same buffer)
+    n_odd = 4097
+    assert (n_odd * cfg.top_k) % 4 != 0
+    buf = to_dev(ids[:n_odd]).clone()
+    pool.reroute(0, buf, to_dev(aid4[:n_odd]), slot_ids=buf, want_counts=False)
+    torch.cuda.synchronize()
+    assert np.array_equal(buf.cpu().numpy(), want4[:n_odd])
+    assert pool.last_device_error() == 8
     pool.destroy()
 
 
@@ -233,8 +292,12 @@ def test_route_from_logits(M, k, n, renorm):
     torch.cuda.synchronize()
     assert pool.last_device_error() in (1, 8)
     assert np.array_equal(ids2.cpu().numpy(), ids)
-    bad_rows = (aid_bad == N - 1) | (aid_bad == N + 3)
-    assert np.array_equal(slots2.cpu().numpy()[bad_rows], ids[bad_rows])
+    loaded = np.ones(N, np.int32)
+    loaded[N - 1] = 0
+    want2, n_bad = oracle.reroute(ids, aid_bad, Pi, loaded=loaded, return_bad=True)
+    assert n_bad == int(((aid_bad == N - 1) | (aid_bad == N + 3)).sum()) > 0
+    assert np.array_equal(slots2.cpu().numpy(), want2)
+    assert np.array_equal(cnt2.cpu().numpy(), oracle.counts(want2, M + N * e_max))
     # empty batch: counts zeroed, nothing else touched
     e_ids, e_w, e_slots, e_cnt = pool.route_logits(0, to_dev(logits[:0]), to_dev(aid[:0]))
     torch.cuda.synchronize()
@@ -248,11 +311,11 @@ def test_route_from_logits(M, k, n, renorm):
 
 
 def test_c2_prefill_layer():
-    """8192 tokens, 20 adapters: routing checked for every token, the layer output on a seeded sample."""
+    """8192 tokens, 20 adapters: routing and the layer output are checked for every token."""
     cfg = wl.CONFIGS["c2"]
-    sample = np.random.default_rng(2).choice(cfg.n_tokens, size=192, replace=False)
-    res = run_layer(cfg, sample=np.sort(sample))
-    print("c2", {k: v for k, v in res.items() if k in ("flips", "rel", "max_abs")})
+    res = run_layer(cfg)
+    assert res["n_checked"] == cfg.n_tokens
+    print("c2", {k: v for k, v in res.items() if k in ("flips", "rel", "max_abs", "n_checked")})
     assert res["flips"] <= 40
     counts = np.bincount(res["slots"].reshape(-1), minlength=cfg.num_slots)
     assert counts[:cfg.num_experts].min() > 256            # base slots are fat (several token blocks) ...
@@ -298,7 +361,9 @@ def test_c4_reroute_full_size():
 
 def test_c3_stacked_layers():
     """26 layers of the decode shape resident in one pool through the virtual weight tensors (fewer layers
-    if the device has less free memory), 20 adapters, Zipf adapter popularity; three layers are checked."""
+    if the device has less free memory), 20 adapters, Zipf adapter popularity.  Every layer is checked against the
+    oracle: routing for all 1024 tokens, the output for the tokens that own the first and the last row of every
+    live slot plus 160 random ones (about 450 tokens per layer)."""
     import torch
     cfg = wl.CONFIGS["c3"]
     per_layer = (66 + 20 * 9) * 3 * cfg.inter * cfg.hidden * 2
@@ -309,14 +374,11 @@ def test_c3_stacked_layers():
     bank = wl.NoiseBank(cfg.seed)
     pool = binding.Pool.from_config(cfg)
     tuned = wl.tuned_sets(cfg)
-    check = sorted({0, L // 2, L - 1})
-    bases = {}
     for l in range(L):
         b = wl.gen_base_layer(cfg, l, bank)
         pool.load_base(l, b.router_w, b.routed.w_gate, b.routed.w_up, b.routed.w_down,
                        b.shared.w_gate, b.shared.w_up, b.shared.w_down)
-        if l in check:
-            bases[l] = b
+        del b
     for i in range(cfg.max_adapters):
         per = [wl.gen_adapter_layer(cfg, i, l, tuned[i][l], bank) for l in range(L)]
         pool.load_adapter(i, np.array([len(tuned[i][l]) for l in range(L)], np.int32),
@@ -330,17 +392,21 @@ def test_c3_stacked_layers():
     assert st["physical_bytes"] - st["live_expert_bytes"] < 0.02 * st["live_expert_bytes"]   # page rounding only
     aid = wl.gen_adapter_ids(cfg)
     assert aid.min() >= 0                                              # every token belongs to an adapter
-    sample = np.sort(np.random.default_rng(3).choice(cfg.n_tokens, size=48, replace=False))
-    for l in check:
-        res = run_layer(cfg, layer=l, sample=sample, pool=pool, bank=bank, tuned=tuned, bases=bases)
-        print("c3 layer", l, {k: v for k, v in res.items() if k in ("flips", "rel", "max_abs")})
-    # all layers back to back on one stream, each on its own input
+    single = []
+    for l in range(L):                   # the oracle's copy of a layer's weights is regenerated from the seed
+        res = run_layer(cfg, layer=l, sample=lambda r, l=l: edge_tokens(r, 160, 300 + l), pool=pool, bank=bank,
+                        tuned=tuned)
+        assert res["n_checked"] >= 128
+        single.append(res["out"].clone())
+        if l in (0, L // 2, L - 1):
+            print("c3 layer", l, {k: v for k, v in res.items() if k in ("flips", "rel", "max_abs", "n_checked")})
+    # all layers back to back on one stream, each on its own input: the same bits as one at a time
     xs = [to_dev(wl.gen_tokens(cfg, l)) for l in range(L)]
     d_aid = to_dev(aid)
     outs = [pool.moe_forward(l, xs[l], d_aid) for l in range(L)]
     torch.cuda.synchronize()
     assert pool.last_device_error() == 0
-    assert all(torch.isfinite(o.float()).all() for o in outs)
+    assert all(torch.equal(o, s_) for o, s_ in zip(outs, single))
     pool.destroy()
 
 
@@ -471,19 +537,28 @@ def check_shape(shape, renorm, seed):
     olayer = oracle_layer(cfg, 0, bank, tuned, base=bases[0])
     olayer.cfg.renormalize, olayer.cfg.routed_scale = renorm, scale
     x = wl.gen_tokens(cfg)
+    x_scale = 1.0
     if cfg.num_experts > 64:      # spread the logits so that the 1e-5 near-tie window stays rare with many experts
-        x = wl.f32_to_bf16_bits(wl.bf16_bits_to_f32(x) * 6.0)
+        x_scale = 6.0
+        x = wl.f32_to_bf16_bits(wl.bf16_bits_to_f32(x) * x_scale)
     aid = wl.gen_adapter_ids(cfg, mode="uniform")
+    # The absolute bound of 2e-2 is stated for outputs the size of the five workloads' (|y| < 4): the final rounding
+    # to bf16 alone is half an ulp = 1.6e-2 for |y| in [4, 8) and 3.1e-2 beyond.  So the inputs are drawn to stay
+    # there instead of the bound being stretched: while the oracle's output reaches 3.5 the activations are halved
+    # (exact in bf16; decided by the oracle alone, before the GPU runs).
+    for _ in range(8):
+        ref_full, *_ = oracle.layer_forward(olayer, x, aid)
+        if float(np.abs(ref_full).max()) < 3.5:
+            break
+        x = wl.f32_to_bf16_bits(wl.bf16_bits_to_f32(x) * np.float32(0.5))
+        x_scale *= 0.5
+    assert float(np.abs(ref_full).max()) < 3.5
     r = pool.moe_forward_debug(0, to_dev(x), to_dev(aid))
     torch.cuda.synchronize()
     assert pool.last_device_error() == 0
-    ids, w, slots, flips = check_routing(cfg, olayer, x, aid, r)
+    ids, w, slots, flips = check_routing(cfg, olayer, x, aid, r, weight_rtol=WEIGHT_RTOL * max(1.0, x_scale))
     assert flips <= max(2, cfg.n_tokens // 20)
-    ref = oracle.ffn_given_slots(olayer, x, slots, w)
-    got = bf16_to_f32(r["out"])
-    tol = 2e-2 * max(1.0, float(np.abs(ref).max()) / 2.0)      # the absolute bound scales with the output magnitude
-    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 1e-2
-    assert np.abs(got - ref).max() <= tol
+    check_output(olayer, x, slots, w, bf16_to_f32(r["out"]))
     pool.destroy()
 
 

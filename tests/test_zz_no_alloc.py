@@ -1,4 +1,4 @@
-"""The allocation-free routing entry point against the regular forward's routing results.
+"""The allocation-free routing entry point against the CPU oracle and against the regular forward.
 
 Some users of the library cannot allocate device memory when they need a routing decision (their
 KV cache owns all free HBM, or they run where the CUDA allocator must not be entered), so
@@ -11,7 +11,7 @@ import pytest
 from paper_2508_17624_b200 import binding, build
 from paper_2508_17624_b200 import workloads as wl
 
-from helpers import WEIGHT_RTOL, WEIGHT_TOL, to_dev
+from helpers import WEIGHT_RTOL, WEIGHT_TOL, check_routing, oracle_layer, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -35,24 +35,33 @@ def test_route_noalloc_matches_forward_twice_in_a_row(name):
     assert torch.cuda.is_available()
     build.build()
     cfg = wl.CONFIGS[name]
+    bank = wl.NoiseBank(cfg.seed)
     pool = binding.Pool.from_config(cfg)
-    binding.load_model(pool, cfg)
-    x, aid = to_dev(wl.gen_tokens(cfg)), to_dev(wl.gen_adapter_ids(cfg))
+    tuned, bases = binding.load_model(pool, cfg, bank)
+    olayer = oracle_layer(cfg, 0, bank, tuned, base=bases[0])
+    x_bits, aid_np = wl.gen_tokens(cfg), wl.gen_adapter_ids(cfg)
+    x, aid = to_dev(x_bits), to_dev(aid_np)
     ref = pool.moe_forward_debug(0, x, aid)
     torch.cuda.synchronize()
     want = {k_: ref[k_].cpu().numpy() for k_ in ("topk_ids", "topk_w", "slot_ids", "counts")}
     for call in range(2):                               # the second call sees the first call's leftovers in the array
         ids, w, slots, counts, status = _route(pool, cfg, x, aid, cfg.n_tokens)
         assert status == 0
+        # against the oracle: ids (near-ties counted), weights, slot ids and counts bit-exact given the ids
+        _, _, _, flips = check_routing(cfg, olayer, x_bits, aid_np,
+                                       dict(topk_ids=ids, topk_w=w, slot_ids=slots, counts=counts))
+        assert flips <= 4
+        # and the same bits as the existing entry point
         assert np.array_equal(ids, want["topk_ids"]), call
         assert (np.abs(w - want["topk_w"]) <= WEIGHT_TOL + WEIGHT_RTOL * want["topk_w"]).all(), call
         assert np.array_equal(slots, want["slot_ids"]), call
         assert np.array_equal(counts, want["counts"]), call
     # a bad adapter id is reported through the status word kept in the array, and cleared by the next call
-    bad = aid.clone()
-    bad[0] = cfg.max_adapters + 3
-    *_, status = _route(pool, cfg, x, bad, cfg.n_tokens)
+    bad_np = aid_np.copy()
+    bad_np[0] = cfg.max_adapters + 3
+    ids, w, slots, counts, status = _route(pool, cfg, x, to_dev(bad_np), cfg.n_tokens)
     assert status & 1
+    check_routing(cfg, olayer, x_bits, bad_np, dict(topk_ids=ids, topk_w=w, slot_ids=slots, counts=counts))
     *_, status = _route(pool, cfg, x, aid, cfg.n_tokens)
     assert status == 0
     assert pool.last_device_error() == 0                # the pool's own status word and workspace were not involved

@@ -12,14 +12,15 @@
 
 namespace ew {
 
-// One work item of the grouped GEMMs: a 128-row tile of one slot's weight matrix times up to NT
-// token rows of that slot.  Built on the device from the per-slot counts.
+// One work item of the grouped GEMMs, built on the device from the per-slot counts.  Thin item: a 128-row tile
+// of one slot's weight matrix times up to NT token rows of that slot.  Fat item (CTA-pair kernel): 256 weight rows
+// (GEMM-1: gate tile + up tile of 128 output features; GEMM-2: 256 output features) times 129..256 token rows.
 struct alignas(16) GemmItem {
     int32_t slot;       // first-dimension index into the virtual weight tensor (>= P: shared expert)
-    int32_t tile;       // 128-row tile of the weight matrix
-    int32_t in_row;     // first activation row (x rows for shared experts, permuted rows otherwise)
+    int32_t tile;       // tile of the weight matrix (thin: 128 rows; fat: see above)
+    int32_t in_row;     // first activation row (x rows for shared experts, slot-contiguous rows otherwise)
     int32_t out_row;    // first output row
-    int32_t rows;       // token rows in this item (1..NT)
+    int32_t rows;       // token rows in this item
     int32_t from_x;     // 1: activation rows come straight from the caller's x (shared experts)
     int32_t pad0, pad1;
 };
@@ -32,11 +33,9 @@ struct Workspace {
     int32_t *inv = nullptr;        // [Bmax, k] row of the pair in slot-contiguous order
     int32_t *counts = nullptr;     // [P]
     int32_t *offsets = nullptr;    // [P + 1]
-    int32_t *n_items = nullptr;    // [2]  items of GEMM-1, GEMM-2
-    GemmItem *items1 = nullptr;
-    GemmItem *items2 = nullptr;
-    int32_t max_items1 = 0, max_items2 = 0;
-    void *xp = nullptr;            // [Bmax*k, H] bf16 permuted activations (written only with EW_DISABLE_GATHER=1)
+    int32_t *n_items = nullptr;    // [4]  thin items of GEMM-1, GEMM-2; fat items of GEMM-1, GEMM-2
+    GemmItem *items1 = nullptr, *items2 = nullptr;   // thin items
+    GemmItem *fat1 = nullptr, *fat2 = nullptr;       // fat items (prefill-sized batches)
     int32_t *src_tok = nullptr;    // [Bmax*k] token of each slot-contiguous row: GEMM-1 fetches those rows of x itself
     void *act = nullptr;           // [S*Bmax + Bmax*k, I] bf16 SwiGLU output
     float *y = nullptr;            // [S*Bmax + Bmax*k, H] fp32 expert outputs
@@ -52,6 +51,7 @@ struct LayerState {
     int32_t *pi_dev = nullptr;     // device [N, M]
     std::vector<int32_t> pi_host;  // master copy
     bool base_loaded = false;
+    bool base_mapped = false;      // the pages under the base and shared experts are mapped (a failed first load is retried without remapping)
     CUtensorMap map_w13, map_w2;   // TMA descriptors over the two virtual tensors
     CUtensorMap map_router[3];     // and over the router rows [M, H], with boxes of 1, 2 and 4 K-atoms
 };
@@ -61,21 +61,20 @@ struct LayerState {
 struct ew_pool {
     ew_config_t cfg;
     int P = 0;                      // M + N * E_max
-    int token_tile = 32;            // NT: token rows per GEMM-1 work item
-    int token_tile2 = 32;           // and per GEMM-2 work item
-    bool use_pairs = false;         // NT = 256: GEMM-2's work items are processed by CTA pairs (cta_group::2)
-    bool gather = false;            // GEMM-1 gathers its token rows from x; no permuted copy of x is written
+    int token_tile = 32;            // NT: token rows per thin work item (32, 64 or 128)
+    bool fat = false;               // prefill-sized batch: blocks of more than 128 rows run on the CTA-pair kernel
     ew::PageBackend *be = nullptr;
     ew::PagePool pages;
     std::vector<ew::LayerState> layers;
     std::vector<std::vector<int32_t>> adapter_counts;   // [N][L]; empty = not loaded
     ew::Workspace ws;
-    CUtensorMap map_xp, map_act;   // TMA descriptors over the workspace activations (box 64 x 32 rows)
-    CUtensorMap map_xp_big[2], map_act_big[2];   // same with 128- and 256-row boxes (prefill token tiles)
+    CUtensorMap map_act, map_act_big;   // TMA descriptors over the SwiGLU output (boxes of 64 x 32 and 64 x 128 rows)
     cudaStream_t copy_stream = nullptr;
     std::vector<std::pair<cudaStream_t, cudaEvent_t>> fwd_events;   // last forward per caller stream
     int sm_count = 148;
     bool counts_clean = true;      // the slot counters are zero (the combine kernel of a finished forward re-zeroes them)
+    cudaEvent_t route_event = nullptr;   // last ew_route_noalloc call (created with the pool: that call creates nothing)
+    bool route_event_used = false;
     bool profiling = false;
     std::vector<cudaEvent_t> prof_events;   // 6 per recorded forward
     size_t prof_used = 0;                   // events in use
@@ -96,17 +95,31 @@ namespace ew {
 
 void set_last_error(const std::string &s);
 
+// Makes the pool's device current for the duration of an entry point and puts the caller's device back on exit.
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    cudaError_t enter(int device) {
+        cudaError_t e = cudaGetDevice(&prev);
+        if (e != cudaSuccess || prev == device) return e;
+        e = cudaSetDevice(device);
+        switched = e == cudaSuccess;
+        return e;
+    }
+    ~DeviceGuard() {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
 // EW_DISABLE_PDL=1 in the environment turns the launch overlap off (plain stream order), for debugging.
-bool pdl_enabled(int kind = -1);
-// EW_DISABLE_PAIRS=1 keeps prefill-sized token tiles on the one-CTA kernel.
-bool pairs_enabled();
-// EW_DISABLE_GATHER=1 brings back the permuted copy of x (GEMM-1 then reads it by TMA), for debugging and A/B runs.
-bool gather_enabled();
+bool pdl_enabled();
+// EW_DISABLE_FAT=1 keeps every block of token rows on the weight-streaming kernel (128-row blocks at prefill).
+bool fat_enabled();
 
 // Launch with programmatic stream serialization (the kernel calls pdl_wait() before it reads its
 // predecessor's output).
 template <class... KArgs, class... Args>
-int launch_pdl(int kind, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -116,7 +129,7 @@ int launch_pdl(int kind, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = pdl_enabled(kind) ? 1 : 0;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
     return (int)cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
@@ -141,5 +154,6 @@ int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid
 int launch_route_logits(ew_pool *p, int layer, const float *logits, const int32_t *aid, int B, int32_t *topk_ids,
                         float *topk_w, int32_t *slot_ids, int32_t *counts, cudaStream_t st);
 int gemm_setup(ew_pool *p);   // once per pool: opt in to the shared memory the GEMM kernels need
+int router_setup(ew_pool *p); // once per pool: the router kernels' attributes and the fixed scratch array's device address
 
 }  // namespace ew

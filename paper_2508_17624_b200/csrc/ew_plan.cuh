@@ -1,6 +1,6 @@
 // Dispatch planning (device functions used by the permute kernel): the exclusive scan of the
 // per-slot token counts (Section 2.1 dispatch), the slot-contiguous order of the (token, expert) pairs as two
-// tables (inv: pair -> row, src_tok: row -> token), and the work-item lists of the two grouped GEMMs.
+// tables (inv: pair -> row, src_tok: row -> token), and the work-item lists of the grouped GEMM kernels.
 //
 // All functions are block-wide: every thread of the CTA calls them with the same arguments; `nthreads` =
 // blockDim.x must be a multiple of 32 and at most 256.
@@ -38,12 +38,17 @@ __device__ inline void block_exclusive_scan(const int32_t *in, int32_t *out, int
 
 struct Params {
     int B, k, P, S;
-    int NT1, NT2;        // token rows per work item of GEMM-1 / GEMM-2
-    int R1, R2;          // weight tiles per group of GEMM-1 / GEMM-2
+    int NT;              // token rows per "thin" work item (swap-AB kernel: weight tile x up to NT token rows)
+    int fat;             // 1: blocks of more than kFatMin rows go to the CTA-pair kernel (256 token rows x 256 weight rows)
+    int R1, R2;          // weight tiles per group of the thin GEMM-1 / GEMM-2 items (128 rows each)
+    int RF1, RF2;        // and of the fat items (GEMM-1: 128 gate + 128 up rows; GEMM-2: 256 rows)
     int32_t *offsets;    // [P + 1] out
-    GemmItem *items1, *items2;
-    int32_t *n_items;    // [2] out
+    GemmItem *items1, *items2, *fat1, *fat2;
+    int32_t *n_items;    // [4] out: thin GEMM-1, thin GEMM-2, fat GEMM-1, fat GEMM-2
 };
+
+constexpr int kFatRows = 256;    // token rows of a fat item
+constexpr int kFatMin = 128;     // a block of at most this many rows is a thin item
 
 // Stages the counts and scans them: sm[0..P] = offsets, and cnt_s (returned) = the counts.  `counts` is read
 // with L1 bypassed (other CTAs' atomics produced it).
@@ -55,81 +60,79 @@ __device__ inline int32_t *stage_and_scan(int32_t *sm, const int32_t *counts, in
     return cnt_s;
 }
 
-// Writes the work items of the groups g = first_group, first_group + group_stride, ... (one warp per group, lanes
-// over the group's items); planner 0 also publishes the offsets and the item counts.  `sm` as left by
+// Writes the work items of the groups g = first_warp, first_warp + warp_stride, ... (one warp per group, lanes
+// over the group's items); the publishing planner also writes the offsets and the item counts.  `sm` as left by
 // stage_and_scan.
 //
-// groups: g < S shared expert g (rows = B); g >= S slot g - S (rows = counts).  Two classes: "thin" groups (at
-// most kThinRows rows: their items are weight streams) and "fat" ones (tensor-core bound at prefill).  The two
-// item sequences are merged evenly, so that at any moment the CTAs hold a mix of both and the weight stream of the
-// thin items overlaps the arithmetic of the fat ones.  Per group the items are ordered (weight tile, token block)
-// so that CTAs working at the same time share a weight tile through L2.
+// groups: g < S shared expert g (rows = B); g >= S slot g - S (rows = counts).  A group's rows are cut into
+// blocks.  Decode-sized batches (fat = 0): blocks of NT rows, all "thin" items = one 128-row weight tile times
+// the block (the weight-streaming kernel).  Prefill-sized batches (fat = 1): full blocks of 256 rows, and a
+// remainder of more than 128 rows, are "fat" items for the CTA-pair kernel; a remainder of at most 128 rows
+// (every adapter slot with few tokens is just that) is a thin item.  Per group the items are ordered (weight
+// tile, token block) so that CTAs working at the same time share a weight tile through L2.
 __device__ inline void write_items(int32_t *sm, const int32_t *cnt_s, const Params &A, int32_t *warp_sums, int nthreads,
                                    int first_warp, int warp_stride, bool publish) {
-    constexpr int kThinRows = 64;
     const int P = A.P, S = A.S, B = A.B;
     const int G = P + S;
     const int32_t *off = sm;
-    int32_t *blk = sm + P + 1;              // [G + 1] scan of the fat groups' token blocks
-    int32_t *nblk = blk + G + 1;            // [G] token blocks of fat groups (0 for thin ones)
-    int32_t *blk_t = nblk + G;              // [G + 1] scan of the thin groups' token blocks
+    int32_t *blk = sm + P + 1;              // [G + 1] scan of the groups' fat blocks
+    int32_t *nblk = blk + G + 1;            // [G] fat blocks
+    int32_t *blk_t = nblk + G;              // [G + 1] scan of the groups' thin blocks
     int32_t *nblk_t = blk_t + G + 1;        // [G]
     const int lane = threadIdx.x & 31;
     if (publish)
         for (int i = threadIdx.x; i <= P; i += nthreads) A.offsets[i] = off[i];
-    // GEMM-1 and GEMM-2 may use different token tiles (NT1, NT2): each pass has its own block counts and scans
-    for (int pass = 0; pass < 2; ++pass) {
-        const int NT = pass ? A.NT2 : A.NT1;
-        const int R = pass ? A.R2 : A.R1;
-        if (pass == 0 || A.NT2 != A.NT1) {                // same tile in both GEMMs (decode): one set of scans serves both
-            __syncthreads();                              // the previous pass has finished reading the scan arrays
-            for (int g = threadIdx.x; g < G; g += nthreads) {
-                const int rows = g < S ? B : cnt_s[g - S];
-                const int nb = (rows + NT - 1) / NT;
-                const bool thin = rows <= kThinRows;
-                nblk[g] = thin ? 0 : nb;
-                nblk_t[g] = thin ? nb : 0;
-            }
-            __syncthreads();
-            block_exclusive_scan(nblk, blk, G, warp_sums, nthreads);
-            block_exclusive_scan(nblk_t, blk_t, G, warp_sums, nthreads);
+    for (int g = threadIdx.x; g < G; g += nthreads) {
+        const int rows = g < S ? B : cnt_s[g - S];
+        if (A.fat) {
+            const int rem = rows % kFatRows;
+            nblk[g] = rows / kFatRows + (rem > kFatMin ? 1 : 0);
+            nblk_t[g] = (rem > 0 && rem <= kFatMin) ? 1 : 0;
+        } else {
+            nblk[g] = 0;
+            nblk_t[g] = (rows + A.NT - 1) / A.NT;
         }
-        const int fat_blocks = blk[G], thin_blocks = blk_t[G];
-        if (publish && threadIdx.x == 0) A.n_items[pass] = (fat_blocks + thin_blocks) * R;
-        const long long n_fat = (long long)fat_blocks * R, n_thin = (long long)thin_blocks * R;
-        const bool small = (n_fat + 1) * (n_thin + 1) < (1ll << 31);
-        GemmItem *dst = pass ? A.items2 : A.items1;
-        for (int g = first_warp; g < G; g += warp_stride) {
-            const bool thin = nblk_t[g] > 0;
-            const int nb = thin ? nblk_t[g] : nblk[g];
-            if (nb == 0) continue;
-            const bool shared = g < S;
-            const int rows = shared ? B : cnt_s[g - S];
-            const int slot = shared ? P + g : g - S;
-            const int in0 = shared ? 0 : off[g - S];
-            const int out0 = shared ? g * B : S * B + off[g - S];
-            const long long first = (long long)(thin ? blk_t[g] : blk[g]) * R;    // index inside the group's own class
-            for (int i = lane; i < nb * R; i += 32) {
-                const int tile = i / nb, c = i % nb;
-                const int in_row = (pass ? out0 : in0) + c * NT;     // GEMM-2 reads what GEMM-1 wrote
-                const int out_row = out0 + c * NT;
-                const int item_rows = min(NT, rows - c * NT);
-                const int from_x = (!pass && shared) ? 1 : 0;
-                // merged position: thin item q has floor(q*n_fat/n_thin) fat items before it, and fat item q
-                // the thin items that rule puts before it
-                const long long q = first + i;
-                long long pos;
-                if (small) {                                  // every product fits 32 bits: cheap divisions
-                    const unsigned qu = (unsigned)q, nf = (unsigned)n_fat, nt = (unsigned)n_thin;
-                    if (thin) pos = nf ? qu + qu * nf / nt : qu;
-                    else pos = nt ? qu + min(nt, ((qu + 1) * nt + nf - 1) / nf) : qu;
-                } else {
-                    if (thin) pos = n_fat ? q + q * n_fat / n_thin : q;
-                    else pos = n_thin ? q + min(n_thin, ((q + 1) * n_thin + n_fat - 1) / n_fat) : q;
-                }
-                int4 *d4 = reinterpret_cast<int4 *>(dst + pos);      // one item = two 16-byte stores
-                d4[0] = make_int4(slot, tile, in_row, out_row);
+    }
+    __syncthreads();
+    block_exclusive_scan(nblk, blk, G, warp_sums, nthreads);
+    block_exclusive_scan(nblk_t, blk_t, G, warp_sums, nthreads);
+    if (publish && threadIdx.x == 0) {
+        A.n_items[0] = blk_t[G] * A.R1;
+        A.n_items[1] = blk_t[G] * A.R2;
+        A.n_items[2] = blk[G] * A.RF1;
+        A.n_items[3] = blk[G] * A.RF2;
+    }
+    for (int g = first_warp; g < G; g += warp_stride) {
+        const bool shared = g < S;
+        const int rows = shared ? B : cnt_s[g - S];
+        if (rows == 0) continue;
+        const int slot = shared ? P + g : g - S;
+        const int in0 = shared ? 0 : off[g - S];                  // GEMM-1 reads x rows (shared) or slot-contiguous rows
+        const int out0 = shared ? g * B : S * B + off[g - S];     // rows of act / Y; GEMM-2 reads what GEMM-1 wrote
+        for (int pass = 0; pass < 2; ++pass) {
+            const int from_x = (!pass && shared) ? 1 : 0;
+            const int in_base = pass ? out0 : in0;
+            // thin items
+            const int nt = nblk_t[g], Rt = pass ? A.R2 : A.R1;
+            GemmItem *dst = (pass ? A.items2 : A.items1) + (size_t)blk_t[g] * Rt;
+            const int thin0 = A.fat ? (rows / kFatRows) * kFatRows : 0;      // first row of the (only) thin block
+            for (int i = lane; i < nt * Rt; i += 32) {
+                const int tile = i / nt, c = i % nt;
+                const int r0 = thin0 + c * A.NT;
+                const int item_rows = A.fat ? rows - thin0 : min(A.NT, rows - r0);
+                int4 *d4 = reinterpret_cast<int4 *>(dst + i);        // one item = two 16-byte stores
+                d4[0] = make_int4(slot, tile, in_base + r0, out0 + r0);
                 d4[1] = make_int4(item_rows, from_x, 0, 0);
+            }
+            // fat items
+            const int nf = nblk[g], Rf = pass ? A.RF2 : A.RF1;
+            GemmItem *dstf = (pass ? A.fat2 : A.fat1) + (size_t)blk[g] * Rf;
+            for (int i = lane; i < nf * Rf; i += 32) {
+                const int tile = i / nf, c = i % nf;
+                const int r0 = c * kFatRows;
+                int4 *d4 = reinterpret_cast<int4 *>(dstf + i);
+                d4[0] = make_int4(slot, tile, in_base + r0, out0 + r0);
+                d4[1] = make_int4(min(kFatRows, rows - r0), from_x, 0, 0);
             }
         }
     }

@@ -10,18 +10,13 @@
 namespace ew {
 static thread_local std::string g_last_error;
 void set_last_error(const std::string &s) { g_last_error = s; }
-bool pairs_enabled() {
-    static const bool on = [] { const char *e = getenv("EW_DISABLE_PAIRS"); return !(e && e[0] == '1'); }();
+bool fat_enabled() {
+    static const bool on = [] { const char *e = getenv("EW_DISABLE_FAT"); return !(e && e[0] == '1'); }();
     return on;
 }
-bool gather_enabled() {
-    static const bool on = [] { const char *e = getenv("EW_DISABLE_GATHER"); return !(e && e[0] == '1'); }();
-    return on;
-}
-bool pdl_enabled(int kind) {
+bool pdl_enabled() {
     static const bool on = [] { const char *e = getenv("EW_DISABLE_PDL"); return !(e && e[0] == '1'); }();
-    static const int mask = [] { const char *e = getenv("EW_PDL_MASK"); return e ? atoi(e) : 31; }();
-    return on && (kind < 0 || ((mask >> kind) & 1));
+    return on;
 }
 }  // namespace ew
 
@@ -101,10 +96,11 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static ew_status_t alloc_workspace(ew_pool *p) {
     const ew_config_t &c = p->cfg;
     size_t Bm = (size_t)c.max_tokens, k = c.top_k, P = p->P, S = c.num_shared, H = c.hidden, I = c.inter;
+    // blocks of token rows: at most one ragged block per group plus the full blocks (32 rows at the least); a fat
+    // block has more than 128 rows
     size_t rb = P + S * ((Bm + 31) / 32) + (Bm * k + 31) / 32 + 1;
-    size_t r1 = (I + 127) / 128, r2 = (H + 127) / 128;
-    p->ws.max_items1 = (int32_t)(rb * r1);
-    p->ws.max_items2 = (int32_t)(rb * r2);
+    size_t rbf = (P + S) + (S * Bm + Bm * k) / 128 + 1;
+    size_t r1 = (I + 127) / 128, r2 = (H + 127) / 128, rf2 = (H + 255) / 256;
     size_t rows = S * Bm + Bm * k + 32;     // +32: a token tile may start at the last row
     struct Seg { void **ptr; size_t bytes; };
     Workspace &w = p->ws;
@@ -112,8 +108,8 @@ static ew_status_t alloc_workspace(ew_pool *p) {
         {(void **)&w.topk_ids, Bm * k * 4}, {(void **)&w.topk_w, Bm * k * 4}, {(void **)&w.slot_ids, Bm * k * 4},
         {(void **)&w.rank, Bm * k * 4}, {(void **)&w.inv, Bm * k * 4}, {(void **)&w.counts, P * 4},
         {(void **)&w.offsets, (P + 1) * 4}, {(void **)&w.n_items, 16}, {(void **)&w.items1, rb * r1 * sizeof(GemmItem)},
-        {(void **)&w.items2, rb * r2 * sizeof(GemmItem)}, {(void **)&w.xp, (Bm * k + 32) * H * 2},
-        {(void **)&w.src_tok, (Bm * k + 32) * 4},
+        {(void **)&w.items2, rb * r2 * sizeof(GemmItem)}, {(void **)&w.fat1, rbf * r1 * sizeof(GemmItem)},
+        {(void **)&w.fat2, rbf * rf2 * sizeof(GemmItem)}, {(void **)&w.src_tok, (Bm * k + 32) * 4},
         {(void **)&w.act, rows * I * 2}, {(void **)&w.y, rows * H * 4}, {(void **)&w.err, 256},
         {(void **)&w.loaded, (size_t)c.max_adapters * 4 + 16},
         {&p->stage_x[0], Bm * H * 2}, {&p->stage_out[0], Bm * H * 2}, {(void **)&p->stage_aid[0], Bm * 4},
@@ -130,24 +126,20 @@ static ew_status_t alloc_workspace(ew_pool *p) {
         off += align_up(s.bytes, 1024);
     }
     w.bytes = total;
-    // TMA descriptors over the permuted activations and the SwiGLU output (box = 64 k-elements x 32 rows)
-    uint64_t d_xp[2] = {H, Bm * k + 32}, d_act[2] = {I, rows};
-    uint32_t box[2] = {64, 32};
-    if (make_tensor_map(p, &p->map_xp, w.xp, 2, d_xp, box) || make_tensor_map(p, &p->map_act, w.act, 2, d_act, box))
+    // TMA descriptors over the SwiGLU output (boxes of 64 k-elements x 32 rows and x 128 rows)
+    uint64_t d_act[2] = {I, rows};
+    uint32_t box[2] = {64, 32}, bbox[2] = {64, 128};
+    if (make_tensor_map(p, &p->map_act, w.act, 2, d_act, box) || make_tensor_map(p, &p->map_act_big, w.act, 2, d_act, bbox))
         return EW_ERR_CUDA;
-    for (int v = 0; v < 2; ++v) {
-        uint32_t bbox[2] = {64, v ? 256u : 128u};
-        if (make_tensor_map(p, &p->map_xp_big[v], w.xp, 2, d_xp, bbox) || make_tensor_map(p, &p->map_act_big[v], w.act, 2, d_act, bbox))
-            return EW_ERR_CUDA;
-    }
     return EW_OK;
 }
 
 static void destroy_pool(ew_pool *p) {
     if (!p) return;
     bool gpu = p->cfg.device >= 0;
+    DeviceGuard guard;
     if (gpu) {
-        cudaSetDevice(p->cfg.device);
+        guard.enter(p->cfg.device);
         cudaDeviceSynchronize();
     }
     for (auto &L : p->layers) {
@@ -161,6 +153,7 @@ static void destroy_pool(ew_pool *p) {
         if (p->ws.topk_ids) cudaFree(p->ws.topk_ids);   // the workspace is one allocation; topk_ids is its base
         for (auto &e : p->fwd_events) cudaEventDestroy(e.second);
         for (auto &e : p->prof_events) cudaEventDestroy(e);
+        if (p->route_event) cudaEventDestroy(p->route_event);
         for (int i = 0; i < 2; ++i) {
             if (p->host_h2d_done[i]) cudaEventDestroy(p->host_h2d_done[i]);
             if (p->host_comp_done[i]) cudaEventDestroy(p->host_comp_done[i]);
@@ -192,8 +185,9 @@ extern "C" ew_status_t ew_pool_create(const ew_config_t *cfg, ew_pool_t **out) {
     bool gpu = c.device >= 0;
     ew_status_t st = EW_OK;
     std::string err;
+    DeviceGuard guard;
     if (gpu) {
-        cudaError_t e = cudaSetDevice(c.device);
+        cudaError_t e = guard.enter(c.device);
         if (e != cudaSuccess) {
             set_last_error(std::string("cudaSetDevice: ") + cudaGetErrorString(e));
             delete p;
@@ -263,7 +257,8 @@ extern "C" ew_status_t ew_pool_create(const ew_config_t *cfg, ew_pool_t **out) {
             }
             ew_status_t s = alloc_workspace(p);
             if (s != EW_OK) return s;
-            if (gemm_setup(p)) return EW_ERR_CUDA;
+            if (gemm_setup(p) || router_setup(p)) return EW_ERR_CUDA;
+            CU_TRY(cudaEventCreateWithFlags(&p->route_event, cudaEventDisableTiming));
             return EW_OK;
         };
         st = body();
@@ -320,10 +315,11 @@ extern "C" ew_status_t ew_load_base(ew_pool_t *p, int32_t layer, const void *rou
     bool gpu = c.device >= 0;
     if (gpu && (!router_w || !w_gate || !w_up || !w_down || (c.num_shared > 0 && (!sh_gate || !sh_up || !sh_down))))
         return EW_ERR_INVALID_ARG;
-    if (gpu) CU_TRY(cudaSetDevice(c.device));
+    DeviceGuard guard;
+    if (gpu) CU_TRY(guard.enter(c.device));
     LayerState &L = p->layers[layer];
     size_t M = c.num_experts, S = c.num_shared, P = p->P;
-    if (!L.base_loaded && c.pool_mode == 0) {
+    if (!L.base_mapped && c.pool_mode == 0) {
         ew_status_t st;
         if ((st = be_status(p, L.w13.map_slots(0, M))) != EW_OK) return st;
         if ((st = be_status(p, L.w2.map_slots(0, M))) != EW_OK) { L.w13.unmap_slots(0, M); return st; }
@@ -333,18 +329,20 @@ extern "C" ew_status_t ew_load_base(ew_pool_t *p, int32_t layer, const void *rou
             return st;
         }
     }
-    if (!L.base_loaded) {
-        p->live_experts += M;
-        p->live_expert_bytes += (M + S) * 3 * (size_t)c.inter * c.hidden * 2;
-    }
+    L.base_mapped = true;
     if (gpu) {
         // forwards in flight may still read the old weights of this layer
         for (auto &e : p->fwd_events) CU_TRY(cudaEventSynchronize(e.second));
+        if (p->route_event_used) CU_TRY(cudaEventSynchronize(p->route_event));
         CU_TRY(cudaMemcpyAsync(L.router_w, router_w, M * c.hidden * 2, cudaMemcpyDefault, p->copy_stream));
         ew_status_t st = copy_experts(p, L, 0, M, w_gate, w_up, w_down);
         if (st == EW_OK && S) st = copy_experts(p, L, P, S, sh_gate, sh_up, sh_down);
         if (st != EW_OK) return st;
         CU_TRY(cudaStreamSynchronize(p->copy_stream));
+    }
+    if (!L.base_loaded) {                               // counted once, when the first load of the layer has succeeded
+        p->live_experts += M;
+        p->live_expert_bytes += (M + S) * 3 * (size_t)c.inter * c.hidden * 2;
     }
     L.base_loaded = true;
     return EW_OK;
@@ -372,7 +370,8 @@ extern "C" ew_status_t ew_load_adapter(ew_pool_t *p, int32_t a, const int32_t *c
                 return EW_ERR_INVALID_ARG;
             }
         }
-    if (gpu) CU_TRY(cudaSetDevice(c.device));
+    DeviceGuard guard;
+    if (gpu) CU_TRY(guard.enter(c.device));
     size_t delta = (size_t)M + (size_t)a * c.e_max;     // Delta_i = M + i * E_max
     ew_status_t st = EW_OK;
     // Layer by layer, tensor by tensor: map the slots' pages (driver calls on this thread, ~0.1 ms per page), then
@@ -423,10 +422,14 @@ extern "C" ew_status_t ew_unload_adapter(ew_pool_t *p, int32_t a) {
     const ew_config_t &c = p->cfg;
     bool gpu = c.device >= 0;
     int L = c.num_layers, M = c.num_experts;
-    if (gpu) CU_TRY(cudaSetDevice(c.device));
-    // 1. forwards issued earlier may still read the adapter's slots and its map rows: let them finish as issued
-    if (gpu)
+    DeviceGuard guard;
+    if (gpu) CU_TRY(guard.enter(c.device));
+    // 1. forwards (and allocation-free routing calls) issued earlier may still read the adapter's slots and its
+    //    map rows: let them finish as issued
+    if (gpu) {
         for (auto &e : p->fwd_events) CU_TRY(cudaEventSynchronize(e.second));
+        if (p->route_event_used) CU_TRY(cudaEventSynchronize(p->route_event));
+    }
     // 2. rows back to identity, so that later forwards no longer reach the adapter's slots
     for (int l = 0; l < L; ++l) {
         LayerState &Ls = p->layers[l];
@@ -494,11 +497,15 @@ extern "C" ew_status_t ew_slot_address(ew_pool_t *p, int32_t layer, int32_t whic
 extern "C" ew_status_t ew_last_device_error(ew_pool_t *p, int32_t *code) {
     if (!p || !code) return EW_ERR_INVALID_ARG;
     if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
-    CU_TRY(cudaSetDevice(p->cfg.device));
+    DeviceGuard guard;
+    CU_TRY(guard.enter(p->cfg.device));
     for (auto &e : p->fwd_events) CU_TRY(cudaEventSynchronize(e.second));
     int32_t v = 0;
     CU_TRY(cudaMemcpy(&v, p->ws.err, 4, cudaMemcpyDeviceToHost));
     CU_TRY(cudaMemset(p->ws.err, 0, 4));
+    // a kernel that gave up on a wait may have left the forward unfinished: the combine kernel, which leaves the slot
+    // counters at zero for the next forward, may not have run
+    if (v & 2) p->counts_clean = false;
     // the word is a bit set: 1 = bad adapter id, 2 = a bounded wait expired, 4 = expert id out of range
     *code = (v & 2) ? EW_ERR_TIMEOUT : (v & 1) ? EW_ERR_BAD_ADAPTER_ID_IN_BATCH : (v & 4) ? EW_ERR_INVALID_ARG : EW_OK;
     return EW_OK;
@@ -562,26 +569,22 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     if (!p->layers[layer].base_loaded) return EW_ERR_NOT_LOADED;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const ew_config_t &c = p->cfg;
-    int dev = -1;
-    CU_TRY(cudaGetDevice(&dev));
-    if (dev != c.device) CU_TRY(cudaSetDevice(c.device));
+    DeviceGuard guard;
+    CU_TRY(guard.enter(c.device));
     // the caller's x becomes the activation operand of the shared experts: describe it for TMA
     CUtensorMap map_x;
     uint64_t dx[2] = {(uint64_t)c.hidden, (uint64_t)B};
     uint32_t box[2] = {64, 32};
     if (make_tensor_map(p, &map_x, x, 2, dx, box)) return EW_ERR_CUDA;
     CUtensorMap map_x_big = map_x;
-    // Prefill-sized batches: GEMM-1 (gate and up accumulators) keeps two accumulator sets in TMEM only up to 128 token
-    // rows per item, which hides its SwiGLU epilogue and measured 25 % faster than 256-row items; GEMM-2 has room for
-    // two sets at 256 rows and runs those on the CTA-pair kernel.
-    p->token_tile2 = pick_token_tile(p, B);
-    p->token_tile = p->token_tile2 == 256 ? 128 : p->token_tile2;
-    p->use_pairs = p->token_tile2 == 256 && pairs_enabled();
-    // The permuted copy of x (k rows per token) is not written: the permute kernel only records which token each
-    // slot-contiguous row is, and GEMM-1 gathers those rows of x (which stay in L2) into its token operand.
-    p->gather = gather_enabled();
+    // Token rows per thin work item, and whether the batch is large enough for fat items (blocks of more than 128
+    // rows on the CTA-pair kernel).  A permuted copy of x (k rows per token) is never written: the permute kernel
+    // only records which token each slot-contiguous row is, and GEMM-1 gathers those rows of x (which stay in L2).
+    const int tile = pick_token_tile(p, B);
+    p->fat = tile == 256 && fat_enabled();
+    p->token_tile = tile == 256 ? 128 : tile;
     if (p->token_tile >= 128) {
-        uint32_t bbox[2] = {64, (uint32_t)p->token_tile};
+        uint32_t bbox[2] = {64, 128};
         if (make_tensor_map(p, &map_x_big, x, 2, dx, bbox)) return EW_ERR_CUDA;
     }
     size_t nk = (size_t)B * c.top_k;
@@ -635,9 +638,8 @@ extern "C" ew_status_t ew_reroute(ew_pool_t *p, int32_t layer, const int32_t *to
     if (!p || layer < 0 || layer >= p->cfg.num_layers || B < 0) return EW_ERR_INVALID_ARG;
     if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    int dev = -1;
-    CU_TRY(cudaGetDevice(&dev));
-    if (dev != p->cfg.device) CU_TRY(cudaSetDevice(p->cfg.device));
+    DeviceGuard guard;
+    CU_TRY(guard.enter(p->cfg.device));
     if (counts) CU_TRY(cudaMemsetAsync(counts, 0, (size_t)p->P * 4, st));
     if (B == 0) return EW_OK;
     if (!topk_ids || !aid || !slot_ids || ((uintptr_t)topk_ids & 3) || ((uintptr_t)slot_ids & 3)) return EW_ERR_INVALID_ARG;
@@ -652,9 +654,8 @@ extern "C" ew_status_t ew_route_logits(ew_pool_t *p, int32_t layer, const float 
     if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
     if (!p->layers[layer].base_loaded) return EW_ERR_NOT_LOADED;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    int dev = -1;
-    CU_TRY(cudaGetDevice(&dev));
-    if (dev != p->cfg.device) CU_TRY(cudaSetDevice(p->cfg.device));
+    DeviceGuard guard;
+    CU_TRY(guard.enter(p->cfg.device));
     CU_TRY(cudaMemsetAsync(counts, 0, (size_t)p->P * 4, st));
     if (B == 0) return EW_OK;
     if (!logits || !aid || !topk_ids || !topk_w || !slot_ids || ((uintptr_t)logits & 15) || (p->cfg.num_experts & 3)) {
@@ -672,9 +673,8 @@ extern "C" ew_status_t ew_moe_forward_host(ew_pool_t *p, int32_t layer, const vo
     if (B == 0) return EW_OK;
     if (!x_host || !aid_host || !out_host) return EW_ERR_INVALID_ARG;
     cudaStream_t user = (cudaStream_t)cuda_stream;
-    int dev = -1;
-    CU_TRY(cudaGetDevice(&dev));
-    if (dev != p->cfg.device) CU_TRY(cudaSetDevice(p->cfg.device));
+    DeviceGuard guard;
+    CU_TRY(guard.enter(p->cfg.device));
     if (!p->host_h2d) {                                   // first use: the pipeline's streams and events
         CU_TRY(cudaStreamCreateWithFlags(&p->host_h2d, cudaStreamNonBlocking));
         CU_TRY(cudaStreamCreateWithFlags(&p->host_comp, cudaStreamNonBlocking));
@@ -721,6 +721,8 @@ extern "C" ew_status_t ew_profile_enable(ew_pool_t *p, int32_t on) {
 extern "C" ew_status_t ew_profile_read(ew_pool_t *p, double *ms, int32_t *n_forwards) {
     if (!p || !ms || !n_forwards) return EW_ERR_INVALID_ARG;
     if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
+    DeviceGuard guard;
+    CU_TRY(guard.enter(p->cfg.device));
     for (int i = 0; i < 5; ++i) ms[i] = 0.0;
     size_t n = p->prof_used / 6;
     for (size_t f = 0; f < n; ++f) {

@@ -6,8 +6,6 @@
 //   combine_kernel   weighted un-permute and sum, one rounding to bf16 (Section 2.1)
 #include <cuda_bf16.h>
 
-#include <cstdlib>
-
 #include "ew_internal.h"
 #include "ew_plan.cuh"
 #include "ew_tc.cuh"
@@ -40,10 +38,11 @@ __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.comm
 template <int N>
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 
-__global__ void __launch_bounds__(256) reroute_kernel(const int32_t *__restrict__ ids, const int32_t *__restrict__ aid,
+// (ids and slots may be the same buffer - the rewrite in place the ABI allows - so neither is __restrict__)
+__global__ void __launch_bounds__(256) reroute_kernel(const int32_t *ids, const int32_t *__restrict__ aid,
                                                       const int32_t *__restrict__ pi, const int32_t *__restrict__ loaded,
                                                       int n_tokens, int k, int M, int N, int P,
-                                                      int32_t *__restrict__ slots, int32_t *__restrict__ counts, int *err) {
+                                                      int32_t *slots, int32_t *__restrict__ counts, int *err) {
     extern __shared__ __align__(128) int32_t smem_i[];
     const int tile_ints_max = kRerouteTok * k;
     const int stage_ints = kRerouteTok + tile_ints_max;            // a stage = 256 adapter ids, then 256*k ids (both 16-byte multiples)
@@ -143,10 +142,10 @@ __global__ void __launch_bounds__(256) reroute_kernel(const int32_t *__restrict_
 }
 
 // any alignment: one thread per (token, expert) pair
-__global__ void __launch_bounds__(256) reroute_kernel_unaligned(const int32_t *__restrict__ ids, const int32_t *__restrict__ aid,
+__global__ void __launch_bounds__(256) reroute_kernel_unaligned(const int32_t *ids, const int32_t *__restrict__ aid,
                                                                 const int32_t *__restrict__ pi, const int32_t *__restrict__ loaded,
                                                                 long long n_pairs, int k, int M, int N,
-                                                                int32_t *__restrict__ slots, int32_t *__restrict__ counts, int *err) {
+                                                                int32_t *slots, int32_t *__restrict__ counts, int *err) {
     for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < n_pairs; q += (long long)gridDim.x * blockDim.x) {
         int a = aid[q / k];
         if (a < -1 || a >= N || (a >= 0 && !loaded[a])) { atomicOr(err, 1); a = -1; }
@@ -316,68 +315,35 @@ __global__ void __launch_bounds__(4 * kLogitTok) route_logits_kernel(const float
 // shared memory; the first kPlanners CTAs publish the offsets and write the GEMM work items (the item
 // loop is a chain of dependent integer arithmetic, so it is spread over several CTAs), the other CTAs record for
 // each (token, expert) pair its slot-contiguous row (inv) and for each row its token (src_tok), one thread per
-// pair.  (Without a src_tok table they copy the token rows instead, one row per warp: the debugging path that keeps
-// a permuted copy of x.)  Item order:
-//   per group the items are ordered (weight tile, token block) so that CTAs working at the same time
-//   share a weight tile through L2; thin and fat groups are merged evenly (see below).
+// pair.  No copy of x is made: GEMM-1 gathers its token rows through src_tok.
 // ------------------------------------------------------------------------------------------------
 constexpr int kPlanners = 8;
 
-__global__ void __launch_bounds__(256) permute_kernel(const uint4 *x, const int32_t *slot_ids,
-                                                      const int32_t *rank, const int32_t *counts,
-                                                      int B, int k, int H, int P, int S, int NT1, int NT2, int R1, int R2,
-                                                      int32_t *offsets, int32_t *inv,
-                                                      uint4 *xp, int32_t *src_tok, GemmItem *items1,
-                                                      GemmItem *items2, int32_t *n_items) {
+__global__ void __launch_bounds__(256) permute_kernel(const int32_t *slot_ids, const int32_t *rank, const int32_t *counts,
+                                                      plan::Params A, int32_t *inv, int32_t *src_tok) {
     extern __shared__ int32_t sm[];
     __shared__ int32_t warp_sums[8];
     tc::pdl_launch_dependents();
-    // counts, slot ids and ranks come from the router kernel, x from the caller's earlier work: none of the kernel's
-    // pointer parameters is __restrict__, so that no load can be hoisted above this wait
+    // counts, slot ids and ranks come from the router kernel: none of the kernel's pointer parameters is
+    // __restrict__, so that no load can be hoisted above this wait
     tc::pdl_wait();
-    const int32_t *cnt_s = plan::stage_and_scan(sm, counts, P, S, warp_sums, 256);
+    const int32_t *cnt_s = plan::stage_and_scan(sm, counts, A.P, A.S, warp_sums, 256);
     const int32_t *off = sm;                 // [P + 1]
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long n_pairs = (long long)B * k;
-    if (blockIdx.x >= kPlanners && src_tok) {
-        // gather mode: no copy of x; one thread per (token, j) pair records the pair's row and the row's token
+    const int warp = threadIdx.x >> 5;
+    const long long n_pairs = (long long)A.B * A.k;
+    if (blockIdx.x >= kPlanners) {           // the first CTAs (dispatched first) are the planners
+        // one thread per (token, j) pair records the pair's row and the row's token
         const long long q = (long long)(blockIdx.x - kPlanners) * 256 + threadIdx.x;
         if (q < n_pairs) {
             const int dest = off[slot_ids[q]] + rank[q];
             if (dest < n_pairs) {            // always, unless the routing kernel gave up midway (error word set)
                 inv[q] = dest;
-                src_tok[dest] = (int32_t)(q / k);
-            }
-        }
-        return;
-    }
-    if (blockIdx.x >= kPlanners) {                       // the first CTAs (dispatched first) are the planners
-        const long long q = (long long)(blockIdx.x - kPlanners) * 8 + warp;
-        if (q < n_pairs) {
-            const int dest = off[slot_ids[q]] + rank[q];
-            if (dest >= n_pairs) return;
-            if (lane == 0) inv[q] = dest;
-            const int hv = H >> 3;
-            const uint4 *src = x + (size_t)(q / k) * hv;
-            uint4 *dst = xp + (size_t)dest * hv;
-            // eight 16-byte loads in flight per lane, then the stores (the pointers are not __restrict__, so the
-            // compiler would otherwise serialise every load behind the previous store)
-            for (int v0 = 0; v0 < hv; v0 += 256) {
-                uint4 r[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u)
-                    if (v0 + u * 32 + lane < hv) r[u] = src[v0 + u * 32 + lane];
-#pragma unroll
-                for (int u = 0; u < 8; ++u)
-                    if (v0 + u * 32 + lane < hv) dst[v0 + u * 32 + lane] = r[u];
+                src_tok[dest] = (int32_t)(q / A.k);
             }
         }
         return;
     }
     // ---- planner CTAs: each has repeated the (cheap) scan and writes the items of every kPlanners-th group
-    plan::Params A;
-    A.B = B; A.k = k; A.P = P; A.S = S; A.NT1 = NT1; A.NT2 = NT2; A.R1 = R1; A.R2 = R2;
-    A.offsets = offsets; A.items1 = items1; A.items2 = items2; A.n_items = n_items;
     plan::write_items(sm, cnt_s, A, warp_sums, 256, warp + 8 * blockIdx.x, 8 * kPlanners, blockIdx.x == 0);
 }
 
@@ -422,41 +388,33 @@ __global__ void __launch_bounds__(256) combine_kernel(const float4 *y, const int
 
 }  // namespace
 
-// Token rows per GEMM work item: the smallest tile that holds ~1.5x the mean rows per routed expert.
+// Token rows per GEMM work item: the smallest tile that holds ~1.5x the mean rows per routed expert.  256 means
+// "prefill-sized": blocks of more than 128 rows become fat items of the CTA-pair kernel.
 int pick_token_tile(const ew_pool *p, int B) {
-    static const int forced = [] { const char *e = getenv("EW_FORCE_NT"); return e ? atoi(e) : 0; }();
-    if (forced == 32 || forced == 64 || forced == 128 || forced == 256) return forced;   // debugging / tuning aid
     const double mean = (double)B * p->cfg.top_k / p->cfg.num_experts;
     const double want = mean * 1.5;
-    // 256-row items (GEMM-2 on CTA pairs) pay off once the mean itself reaches a full 128-row tile; just below that
-    // (the stacked-decode shape: 96 rows per base expert) 128-row items measured 0.7 % faster
     return want <= 32 ? 32 : want <= 64 ? 64 : want <= 192 ? 128 : 256;
 }
 
-// weight tiles per group: 128-row tiles, or 256-row tile pairs where the CTA-pair kernel runs the items
-void plan_tiles(const ew_pool *p, int *R1, int *R2) {
+int launch_permute(ew_pool *p, const void *, int B, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
-    *R1 = (c.inter + 127) / 128;                                 // GEMM-1 always runs on the one-CTA kernel
-    const int tile_rows2 = p->use_pairs ? 256 : 128;
-    *R2 = (c.hidden + tile_rows2 - 1) / tile_rows2;
-}
-
-int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st) {
-    const ew_config_t &c = p->cfg;
-    int R1, R2;
-    plan_tiles(p, &R1, &R2);
+    plan::Params A;
+    A.B = B; A.k = c.top_k; A.P = p->P; A.S = c.num_shared;
+    A.NT = p->token_tile; A.fat = p->fat ? 1 : 0;
+    A.R1 = (c.inter + 127) / 128; A.R2 = (c.hidden + 127) / 128;
+    A.RF1 = (c.inter + 127) / 128; A.RF2 = (c.hidden + 255) / 256;
+    A.offsets = p->ws.offsets; A.items1 = p->ws.items1; A.items2 = p->ws.items2; A.fat1 = p->ws.fat1; A.fat2 = p->ws.fat2;
+    A.n_items = p->ws.n_items;
     const long long pairs = (long long)B * c.top_k;
-    const int grid = (int)(p->gather ? (pairs + 255) / 256 : (pairs + 7) / 8) + kPlanners;
+    const int grid = (int)((pairs + 255) / 256) + kPlanners;
     const size_t smem = plan::smem_words(p->P, c.num_shared) * 4;
-    return launch_pdl(1, permute_kernel, dim3(grid), dim3(256), smem, st, (const uint4 *)x, p->ws.slot_ids, p->ws.rank,
-                      p->ws.counts, B, c.top_k, c.hidden, p->P, c.num_shared, p->token_tile, p->token_tile2, R1, R2, p->ws.offsets, p->ws.inv,
-                      (uint4 *)p->ws.xp, p->gather ? p->ws.src_tok : (int32_t *)nullptr, p->ws.items1, p->ws.items2,
-                      p->ws.n_items);
+    return launch_pdl(permute_kernel, dim3(grid), dim3(256), smem, st, (const int32_t *)p->ws.slot_ids, (const int32_t *)p->ws.rank,
+                      (const int32_t *)p->ws.counts, A, p->ws.inv, p->ws.src_tok);
 }
 
 int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
-    return launch_pdl(4, combine_kernel, dim3(B), dim3(256), 0, st, (const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B, c.top_k,
+    return launch_pdl(combine_kernel, dim3(B), dim3(256), 0, st, (const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B, c.top_k,
                       c.hidden, c.num_shared, (uint2 *)out, p->ws.counts, p->P);
 }
 

@@ -444,12 +444,9 @@ static int router_launch(ew_pool *p, int layer, const void *x, const RouterGeome
     A.H = c.hidden; A.M = c.num_experts; A.k = c.top_k; A.N = c.max_adapters; A.renormalize = c.renormalize;
     A.scale = c.routed_scale;
     A.stages = g.stages; A.tmem_cols = g.tmem_cols; A.pi_in_smem = g.pi_in_smem; A.tok_tile = g.tok_tile; A.atoms = g.atoms;
-    cudaError_t e = g.reg ? cudaFuncSetAttribute(router_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
-                          : cudaFuncSetAttribute(router_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e != cudaSuccess) return (int)e;
     if (pdl) {
-        if (g.reg) return launch_pdl(0, router_kernel<true>, dim3(g.grid), dim3(kThreads), g.smem, st, map_x, map_r, A);
-        return launch_pdl(0, router_kernel<false>, dim3(g.grid), dim3(kThreads), g.smem, st, map_x, map_r, A);
+        if (g.reg) return launch_pdl(router_kernel<true>, dim3(g.grid), dim3(kThreads), g.smem, st, map_x, map_r, A);
+        return launch_pdl(router_kernel<false>, dim3(g.grid), dim3(kThreads), g.smem, st, map_x, map_r, A);
     }
     if (g.reg) router_kernel<true><<<g.grid, kThreads, g.smem, st>>>(map_x, map_r, A);
     else router_kernel<false><<<g.grid, kThreads, g.smem, st>>>(map_x, map_r, A);
@@ -511,6 +508,22 @@ int noalloc_scratch(int device, unsigned char **out) {
     return 0;
 }
 }  // namespace
+
+// Once per pool, with the pool's device current (ew_pool_create): everything about the router kernels that may load
+// code or reserve memory on first use happens here, where the pool allocates anyway - the opt-in to large dynamic
+// shared memory, a query that forces both instantiations to be loaded, and the device address of the fixed scratch
+// array.  ew_route_noalloc then only looks the address up.
+int router_setup(ew_pool *p) {
+    cudaError_t e = cudaFuncSetAttribute(router_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(router_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaFuncAttributes fa;
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, router_kernel<true>);
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, router_kernel<false>);
+    unsigned char *scratch = nullptr;
+    int rc = e == cudaSuccess ? noalloc_scratch(p->cfg.device, &scratch) : (int)e;
+    if (rc) set_last_error(std::string("router set-up: ") + cudaGetErrorString((cudaError_t)rc));
+    return rc;
+}
 }  // namespace ew
 
 extern "C" ew_status_t ew_route_noalloc(ew_pool_t *p, int32_t layer, const void *x, const int32_t *adapter_ids,
@@ -526,34 +539,34 @@ extern "C" ew_status_t ew_route_noalloc(ew_pool_t *p, int32_t layer, const void 
     }
     if (!counts) return EW_ERR_INVALID_ARG;
     if (!p->layers[layer].base_loaded) return EW_ERR_NOT_LOADED;
+    if (n_tokens > 0 && (!x || !adapter_ids || !topk_ids || !topk_w || !slot_ids || ((uintptr_t)x & 15))) return EW_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    int dev = -1;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess && dev != c.device) e = cudaSetDevice(c.device);
+    DeviceGuard guard;
+    cudaError_t e = guard.enter(c.device);
     unsigned char *scratch = nullptr;
-    int rc = e == cudaSuccess ? noalloc_scratch(c.device, &scratch) : (int)e;
+    int rc = e == cudaSuccess ? noalloc_scratch(c.device, &scratch) : (int)e;      // resolved when the pool was created
     // the array keeps the previous call's contents: the status word and the counters must start at zero
     if (!rc) rc = (int)cudaMemsetAsync(scratch, 0, kNoAllocHeader, st);
     if (!rc) rc = (int)cudaMemsetAsync(counts, 0, (size_t)p->P * 4, st);
+    if (!rc && n_tokens > 0) {
+        RouterGeometry g;
+        if (!router_geometry(p, n_tokens, &g)) return EW_ERR_INVALID_ARG;
+        RouterArgs A;
+        A.aid = adapter_ids; A.B = n_tokens;
+        A.topk_ids = topk_ids; A.topk_w = topk_w; A.slot_ids = slot_ids; A.counts = counts;
+        A.rank = reinterpret_cast<int32_t *>(scratch + kNoAllocHeader);      // scratch: position of each pair in its slot
+        A.err = reinterpret_cast<int *>(scratch);                            // scratch: device status word
+        rc = router_launch(p, layer, x, g, A, false, st);
+    }
+    if (!rc && device_status) rc = (int)cudaMemcpyAsync(device_status, scratch, 4, cudaMemcpyDeviceToDevice, st);
+    // eviction and base reloads wait for this call through an event that was created with the pool
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (!rc && cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone) {
+        rc = (int)cudaEventRecord(p->route_event, st);
+        p->route_event_used = true;
+    }
     if (rc) {
         set_last_error(std::string("ew_route_noalloc: ") + cudaGetErrorString((cudaError_t)rc));
-        return EW_ERR_CUDA;
-    }
-    if (n_tokens == 0) return EW_OK;
-    if (!x || !adapter_ids || !topk_ids || !topk_w || !slot_ids || ((uintptr_t)x & 15)) return EW_ERR_INVALID_ARG;
-
-    RouterGeometry g;
-    if (!router_geometry(p, n_tokens, &g)) return EW_ERR_INVALID_ARG;
-    RouterArgs A;
-    A.aid = adapter_ids; A.B = n_tokens;
-    A.topk_ids = topk_ids; A.topk_w = topk_w; A.slot_ids = slot_ids; A.counts = counts;
-    A.rank = reinterpret_cast<int32_t *>(scratch + kNoAllocHeader);      // scratch: position of each pair in its slot
-    A.err = reinterpret_cast<int *>(scratch);                            // scratch: device status word
-    e = (cudaError_t)router_launch(p, layer, x, g, A, false, st);
-    if (e == cudaSuccess && device_status)
-        e = cudaMemcpyAsync(device_status, scratch, 4, cudaMemcpyDeviceToDevice, st);
-    if (e != cudaSuccess) {
-        set_last_error(std::string("ew_route_noalloc: ") + cudaGetErrorString(e));
         return EW_ERR_CUDA;
     }
     return EW_OK;
@@ -588,8 +601,10 @@ extern "C" ew_status_t ew_selftest_bounded_wait(ew_pool_t *p, void *cuda_stream)
     if (!p) return EW_ERR_INVALID_ARG;
     if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    DeviceGuard guard;
     int *flag = p->ws.err + 1;                            // second word of the error segment
-    cudaError_t e = cudaMemsetAsync(flag, 0, 4, st);
+    cudaError_t e = guard.enter(p->cfg.device);
+    if (e == cudaSuccess) e = cudaMemsetAsync(flag, 0, 4, st);
     if (e == cudaSuccess) {
         wait_selftest_kernel<<<1, 32, 0, st>>>(p->ws.err, flag);
         e = cudaGetLastError();

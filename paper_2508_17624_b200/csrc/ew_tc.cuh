@@ -58,6 +58,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
 }
+// The same wait for a whole warp: lane 0 polls, the result reaches the other lanes through a shuffle (which also
+// orders their later reads after lane 0's acquire).  Thirty-two lanes polling one barrier word cost shared-memory
+// cycles that the tensor core's operand reads and the copies in flight need.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, err) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -175,12 +183,15 @@ __device__ __forceinline__ void tc2_commit_both(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                  ::"r"(bar), "h"((uint16_t)3) : "memory");
 }
-// arrive on the barrier at this offset in CTA 0 (from either CTA)
+// arrive on the barrier at this offset in CTA 0 (from either CTA).  Default semantics (release at CTA scope):
+// the cluster-scope release form measured about 1400 cycles per call, which a thread that arrives once per
+// pipeline stage cannot afford; what the arrival publishes here is either TMEM traffic ordered by the tcgen05
+// fences or shared-memory writes already ordered by a proxy fence, and the waiter acquires at cluster scope.
 __device__ __forceinline__ void mbar_arrive_leader(uint32_t local_bar) {
     asm volatile(
         "{\n\t.reg .b32 ra;\n\t"
         "mapa.shared::cluster.u32 ra, %0, 0;\n\t"
-        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
+        "mbarrier.arrive.shared::cluster.b64 _, [ra];\n\t}"
         ::"r"(local_bar) : "memory");
 }
 __device__ __forceinline__ uint32_t instr_desc_m256(int n) {

@@ -16,7 +16,10 @@
  *   - bf16 tensors are passed as void* to raw 16-bit patterns, row-major, innermost dimension
  *     contiguous.  int32 and float are the C types.
  *   - One pool may be used by one host thread at a time.  Forward calls on one pool share one
- *     workspace: issue them on one stream (or order them yourself).
+ *     workspace; the pool orders them itself (a call on another stream than the previous one first
+ *     makes its stream wait for that forward, on the device).
+ *   - Every entry point makes the pool's device current while it runs and restores the caller's
+ *     current device before it returns.
  *   - H must be a multiple of 64 and I a multiple of 8; M <= 256; top_k <= 32 and <= M.
  */
 #ifndef EXPERTWEAVE_H_
@@ -86,8 +89,8 @@ typedef struct {
 
 /* Create a pool: reserves, per layer and per stacked linear (gate|up fused as one tensor, down as
  * another), a contiguous virtual range for M + N*E_max slots (+S trailing slots that hold the shared
- * experts and are never addressed by the expert map) and maps nothing (Section 4.2, "reserves the
- * contiguous virtual address space ... without mapping any physical memory page"); allocates the
+ * experts and are never addressed by the expert map); no physical page is mapped under it at this
+ * point (Section 4.2: reservation and mapping are separate steps).  Allocates the
  * expert maps (identity rows), router storage and the forward workspace for cfg->max_tokens.
  * Errors: EW_ERR_INVALID_ARG (bad sizes), EW_ERR_OOM, EW_ERR_CUDA.  *out is set only on EW_OK. */
 ew_status_t ew_pool_create(const ew_config_t *cfg, ew_pool_t **out);
@@ -96,8 +99,8 @@ ew_status_t ew_pool_create(const ew_config_t *cfg, ew_pool_t **out);
 ew_status_t ew_pool_destroy(ew_pool_t *pool);
 
 /* Load the base model's weights of one layer: the range [0, M) of the pool plus the shared experts
- * (Section 4.2: "loading of a range of consecutive experts, either from the base model at system
- * initialization time or from an adapter at runtime").  All pointers are HOST bf16:
+ * (Section 4.2 treats the base model as one more range of consecutive experts, loaded once at start-up
+ * through the same map-and-copy path that adapters take later).  All pointers are HOST bf16:
  *   router_w [M,H]; w_gate, w_up [M,I,H]; w_down [M,H,I]; sh_gate, sh_up [S,I,H]; sh_down [S,H,I]
  * (the sh_* pointers may be null when S = 0).  Data is copied before the call returns; the caller
  * keeps ownership.  Calling it again for the same layer overwrites the weights in place. */
@@ -125,10 +128,11 @@ ew_status_t ew_load_adapter(ew_pool_t *pool, int32_t adapter_id, const int32_t *
 
 /* Evict an adapter: the call waits for every forward issued before it (they complete as issued, with
  * the adapter still in place), then its expert-map rows return to identity and pages whose reference
- * count drops to zero are unmapped and returned to the pool's free list for reuse (Section 4.2).  Errors: EW_ERR_INVALID_ARG, EW_ERR_NOT_LOADED. */
+ * count drops to zero are unmapped and returned to the pool's free list for reuse (Section 4.2).
+ * Errors: EW_ERR_INVALID_ARG, EW_ERR_NOT_LOADED. */
 ew_status_t ew_unload_adapter(ew_pool_t *pool, int32_t adapter_id);
 
-/* Release the free list's pages back to the driver ("eventually reclaimed", Section 4.2). */
+/* Release the free list's pages back to the driver (Section 4.2: pages that are not reused are reclaimed). */
 ew_status_t ew_pool_trim(ew_pool_t *pool);
 
 /* The adapter-aware MoE layer forward (Sections 2.1, 4.1, 4.3), asynchronous on `cuda_stream`:
@@ -196,6 +200,15 @@ ew_status_t ew_profile_read(ew_pool_t *pool, double *ms, int32_t *n_forwards);
 ew_status_t ew_reroute(ew_pool_t *pool, int32_t layer, const int32_t *topk_ids, const int32_t *adapter_ids,
                        int32_t n_tokens, int32_t *slot_ids, int32_t *counts, void *cuda_stream);
 
+/* Ablation of the operator above (Section 5.3, Figure 7, the "SingleOp" variant): the same rewrite as one kernel per
+ * elementary tensor operation - broadcast the adapter ids to [n_tokens,k], compute offsets into the flattened map,
+ * gather - with both intermediates materialised, plus a histogram kernel when counts is not null.  Results are
+ * identical to ew_reroute's; only the cost differs.  scratch: DEVICE int32 [2 * n_tokens * k], caller-owned.
+ * All other arguments as for ew_reroute (slot_ids may alias topk_ids). */
+ew_status_t ew_reroute_unfused(ew_pool_t *pool, int32_t layer, const int32_t *topk_ids, const int32_t *adapter_ids,
+                               int32_t n_tokens, int32_t *slot_ids, int32_t *counts, int32_t *scratch,
+                               void *cuda_stream);
+
 /* Gate function and rerouting from given logits, in one kernel (Sections 2.1 and 4.3; the operator of
  * ew_reroute fused with the softmax + top-k that precedes it): for every token softmax over its M logits, the
  * top_k largest probabilities (ties to the lower index) as topk_ids / topk_w (renormalised and scaled as the
@@ -216,18 +229,21 @@ ew_status_t ew_route_logits(ew_pool_t *pool, int32_t layer, const float *logits,
  * flight).  It runs the same fused router kernel as ew_moe_forward (logits, softmax, top-k, batched
  * rerouting, per-slot counts) for x [n_tokens,H] and writes into buffers the CALLER provides:
  *   topk_ids, slot_ids [n_tokens,k] int32; topk_w [n_tokens,k] float; counts [M + N*E_max] int32
- *   (overwritten); device_status (optional, device int32): 0 or EW_ERR_BAD_ADAPTER_ID_IN_BATCH-style
- *   bit set as in ew_last_device_error's word (bit 0 bad adapter id, bit 1 expired wait).
+ *   (overwritten); device_status (optional, device int32): 0, or bits as in ew_last_device_error's
+ *   word (bit 0 bad adapter id, bit 1 expired wait); written for n_tokens = 0 as well.
  * All pointers DEVICE.  The kernel's scratch lives in one fixed array inside the library (about 256 KiB
- * per GPU, held until the process exits); therefore
+ * per GPU, held from the moment the library's code is loaded on that GPU until the process exits); therefore
  *   - n_tokens * top_k must not exceed 65536, otherwise EW_ERR_INVALID_ARG and nothing is launched;
- *   - the call performs no cudaMalloc / cudaFree and enters no allocating library routine;
- *   - the first call on a device resolves the array's device address (cudaGetSymbolAddress): make that
- *     first call before any stream capture begins;
+ *   - the call performs no cudaMalloc / cudaFree and enters no allocating library routine.  Everything
+ *     that may load code or reserve memory on first use - the array's device address
+ *     (cudaGetSymbolAddress), the router kernels' attributes - is resolved by ew_pool_create, once per
+ *     device, so the first routing call already finds it done;
  *   - all calls share the array, which still holds the previous call's contents (the words that must
  *     start at zero are cleared on the stream at the start of each call): two calls that overlap on
  *     the GPU (different streams, no ordering) race on it.  Order them.
- * The pool's weights and expert maps are read, its workspace is not touched.
+ * The pool's weights and expert maps are read, its workspace is not touched.  ew_unload_adapter and
+ * ew_load_base wait for the latest call of this entry point (an event created with the pool is recorded
+ * after it) as they wait for forwards; calls made during stream capture are not tracked.
  * Errors: EW_ERR_INVALID_ARG, EW_ERR_NOT_LOADED, EW_ERR_NO_DEVICE, EW_ERR_CUDA. */
 ew_status_t ew_route_noalloc(ew_pool_t *pool, int32_t layer, const void *x, const int32_t *adapter_ids,
                              int32_t n_tokens, int32_t *topk_ids, float *topk_w, int32_t *slot_ids,

@@ -22,7 +22,7 @@ STATUS_NAMES = ["EW_OK", "EW_ERR_INVALID_ARG", "EW_ERR_OOM", "EW_ERR_SLOT_IN_USE
                 "EW_ERR_NO_DEVICE"]
 EXPORTS = ["ew_pool_create", "ew_pool_destroy", "ew_load_base", "ew_load_adapter", "ew_unload_adapter",
            "ew_pool_trim", "ew_moe_forward", "ew_moe_forward_debug", "ew_moe_forward_host", "ew_profile_enable",
-           "ew_profile_read", "ew_reroute", "ew_route_logits", "ew_route_noalloc", "ew_selftest_bounded_wait", "ew_get_expert_map",
+           "ew_profile_read", "ew_reroute", "ew_reroute_unfused", "ew_route_logits", "ew_route_noalloc", "ew_selftest_bounded_wait", "ew_get_expert_map",
            "ew_pool_stats", "ew_last_device_error", "ew_slot_address", "ew_status_str", "ew_last_error_string"]
 
 
@@ -201,6 +201,19 @@ class Pool:
             counts = torch.empty((self.num_slots,), dtype=torch.int32, device=topk_ids.device)
         _check(lib().ew_reroute(self._h, layer, _dp(topk_ids), _dp(adapter_ids), topk_ids.shape[0], _dp(slot_ids),
                                 _dp(counts), _stream()), "ew_reroute")
+        return slot_ids, counts
+
+    def reroute_unfused(self, layer, topk_ids, adapter_ids, slot_ids=None, counts=None, want_counts=True, scratch=None):
+        """The same rewrite as `reroute`, as one kernel per elementary tensor operation (ablation)."""
+        import torch
+        if slot_ids is None:
+            slot_ids = torch.empty_like(topk_ids)
+        if counts is None and want_counts:
+            counts = torch.empty((self.num_slots,), dtype=torch.int32, device=topk_ids.device)
+        if scratch is None:
+            scratch = torch.empty((2 * topk_ids.numel(),), dtype=torch.int32, device=topk_ids.device)
+        _check(lib().ew_reroute_unfused(self._h, layer, _dp(topk_ids), _dp(adapter_ids), topk_ids.shape[0], _dp(slot_ids),
+                                        _dp(counts), _dp(scratch), _stream()), "ew_reroute_unfused")
         return slot_ids, counts
 
     def route_logits(self, layer, logits, adapter_ids):

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libexpertweave.so")
-SOURCES = ["ew_vmm.cpp", "ew_pool.cu", "ew_route.cu", "ew_router.cu", "ew_gemm.cu"]
+SOURCES = ["ew_vmm.cpp", "ew_pool.cu", "ew_route.cu", "ew_router.cu", "ew_gemm.cu", "ew_ablate.cu"]
 
 
 def _nvcc() -> str:

@@ -90,6 +90,84 @@ def test_c1_base_only_equals_no_adapters():
     assert (a["slots"] < cfg.num_experts).all()
 
 
+@pytest.mark.parametrize("name", ["c0", "c1"])
+def test_padding_mode_pool(name):
+    """The padding baseline of Section 3.1 (pool_mode = 1: the whole [M + N*E_max] tensor is backed by pages at
+    creation): the same kernels give the oracle's result, bit-identical to the pool that maps pages on demand,
+    while holding the full tensor's worth of pages."""
+    import torch
+    cfg = wl.CONFIGS[name]
+    vmm = run_layer(cfg)
+    pad = run_layer(cfg, pool_mode=1)
+    assert torch.equal(vmm["out"], pad["out"]) and np.array_equal(vmm["slots"], pad["slots"])
+    pools = {m: binding.Pool.from_config(cfg, pool_mode=m) for m in (0, 1)}
+    for pool in pools.values():
+        binding.load_model(pool, cfg, adapters=[0])          # one adapter: most of the adapter range is padding
+    st0, st1 = pools[0].stats(), pools[1].stats()
+    assert st1["pages_mapped"] * st1["page_bytes"] >= st1["padding_bytes"]        # fully backed
+    assert st0["pages_mapped"] <= st1["pages_mapped"] and (name == "c0" or st0["pages_mapped"] < 0.8 * st1["pages_mapped"])
+    assert st0["physical_bytes"] - st0["live_expert_bytes"] <= 4 * st0["page_bytes"]   # page rounding only
+    for pool in pools.values():
+        pool.destroy()
+
+
+def test_slot_address_reads_back_the_loaded_weights():
+    """ew_slot_address: start_addr = base + slot * expert_size (Section 4.2); the bytes there are the expert's
+    weights as loaded (gate block then up block in the fused tensor), for base, adapter and shared slots."""
+    import torch
+    from cuda.bindings import runtime as rt
+    cfg = wl.CONFIGS["c0"]
+    bank = wl.NoiseBank(cfg.seed)
+    pool = binding.Pool.from_config(cfg)
+    tuned, bases = binding.load_model(pool, cfg, bank)
+    torch.cuda.synchronize()
+    blk = cfg.inter * cfg.hidden            # elements per matrix
+
+    def read(which, slot, n_elems):
+        host = np.empty(n_elems, np.uint16)
+        err, = rt.cudaMemcpy(host.ctypes.data, pool.slot_address(0, which, slot), n_elems * 2,
+                             rt.cudaMemcpyKind.cudaMemcpyDeviceToHost)
+        assert int(err) == 0
+        return host
+
+    base13, base2 = pool.slot_address(0, 0, 0), pool.slot_address(0, 1, 0)
+    for slot in (0, 7, cfg.num_experts - 1):
+        assert pool.slot_address(0, 0, slot) == base13 + slot * 2 * blk * 2
+        assert pool.slot_address(0, 1, slot) == base2 + slot * blk * 2
+        got = read(0, slot, 2 * blk)
+        assert np.array_equal(got[:blk], bases[0].routed.w_gate[slot].reshape(-1))
+        assert np.array_equal(got[blk:], bases[0].routed.w_up[slot].reshape(-1))
+        assert np.array_equal(read(1, slot, blk), bases[0].routed.w_down[slot].reshape(-1))
+    ew = wl.gen_adapter_layer(cfg, 1, 0, tuned[1][0], bank)
+    slot = cfg.num_experts + 1 * cfg.e_max + 2                     # adapter 1, third tuned expert
+    assert np.array_equal(read(0, slot, blk), ew.w_gate[2].reshape(-1))
+    assert np.array_equal(read(1, slot, blk), ew.w_down[2].reshape(-1))
+    shared = cfg.num_slots                                         # first shared expert sits behind the P routed slots
+    assert np.array_equal(read(0, shared, blk), bases[0].shared.w_gate[0].reshape(-1))
+    with pytest.raises(binding.EwError):
+        pool.slot_address(0, 0, cfg.num_slots + cfg.num_shared)
+    with pytest.raises(binding.EwError):
+        pool.slot_address(0, 2, 0)
+    pool.destroy()
+
+
+@pytest.mark.parametrize("switch", ["EW_DISABLE_PDL", "EW_DISABLE_FAT"])
+def test_debugging_switches_in_a_fresh_process(switch):
+    """The two environment switches of the library (plain stream order instead of overlapped launches; every block
+    on the weight-streaming kernel) are read once per process, so each is exercised in a process of its own: the
+    tiny layer, the decode layer and a prefill-sized odd shape against the oracle."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, **{switch: "1"})
+    here = os.path.dirname(os.path.abspath(__file__))
+    r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-x", "-m", "gpu", os.path.join(here, "test_gpu_parity.py"), "-k",
+                        "test_c0_tiny_layer or test_c1_decode_layer or (test_odd_shapes and shape8)"],
+                       env=env, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
+    assert " passed" in r.stdout and "4 passed" in r.stdout, r.stdout[-500:]
+
+
 def test_zero_tokens_and_errors():
     import torch
     cfg = wl.CONFIGS["c0"]
@@ -239,6 +317,10 @@ def test_reroute_operator_c4_sample():
     assert np.array_equal(slots4.cpu().numpy(), want4)
     assert np.array_equal(cnt4.cpu().numpy(), oracle.counts(want4, cfg.num_slots))
     assert pool.last_device_error() == 8
+    slots5, cnt5 = pool.reroute_unfused(0, to_dev(ids), to_dev(aid4))
+    torch.cuda.synchronize()
+    assert np.array_equal(slots5.cpu().numpy(), want4) and np.array_equal(cnt5.cpu().numpy(), cnt4.cpu().numpy())
+    assert pool.last_device_error() == 8
     # in place, on a batch whose pair count is not a multiple of four (vector body + scalar tail on the same buffer)
     n_odd = 4097
     assert (n_odd * cfg.top_k) % 4 != 0
@@ -351,6 +433,15 @@ def test_c4_reroute_full_size():
         # in place (slot_ids aliasing topk_ids) gives the same result
         buf = d_ids.clone()
         pool.reroute(0, buf, d_aid, slot_ids=buf, want_counts=False)
+        torch.cuda.synchronize()
+        assert np.array_equal(buf.cpu().numpy(), want)
+        # the unfused formulation (one kernel per tensor operation) gives the oracle's result as well
+        slots_u, cnt_u = pool.reroute_unfused(0, d_ids, d_aid)
+        torch.cuda.synchronize()
+        assert np.array_equal(slots_u.cpu().numpy(), want)
+        assert np.array_equal(cnt_u.cpu().numpy(), oracle.counts(want, cfg.num_slots))
+        buf = d_ids.clone()
+        pool.reroute_unfused(0, buf, d_aid, slot_ids=buf, want_counts=False)
         torch.cuda.synchronize()
         assert np.array_equal(buf.cpu().numpy(), want)
         for i in range(cfg.max_adapters):

@@ -505,7 +505,10 @@ extern "C" ew_status_t ew_last_device_error(ew_pool_t *p, int32_t *code) {
     CU_TRY(cudaMemset(p->ws.err, 0, 4));
     // a kernel that gave up on a wait may have left the forward unfinished: the combine kernel, which leaves the slot
     // counters at zero for the next forward, may not have run
-    if (v & 2) p->counts_clean = false;
+    if (v & 2) {
+        p->counts_clean = false;
+        CU_TRY(cudaMemset(p->ws.err + 8, 0, 8));        // and the rerouting operator's zeroing handshake may be half done
+    }
     // the word is a bit set: 1 = bad adapter id, 2 = a bounded wait expired, 4 = expert id out of range
     *code = (v & 2) ? EW_ERR_TIMEOUT : (v & 1) ? EW_ERR_BAD_ADAPTER_ID_IN_BATCH : (v & 4) ? EW_ERR_INVALID_ARG : EW_OK;
     return EW_OK;
@@ -640,9 +643,20 @@ extern "C" ew_status_t ew_reroute(ew_pool_t *p, int32_t layer, const int32_t *to
     cudaStream_t st = (cudaStream_t)cuda_stream;
     DeviceGuard guard;
     CU_TRY(guard.enter(p->cfg.device));
-    if (counts) CU_TRY(cudaMemsetAsync(counts, 0, (size_t)p->P * 4, st));
-    if (B == 0) return EW_OK;
+    if (B == 0) {
+        if (counts) CU_TRY(cudaMemsetAsync(counts, 0, (size_t)p->P * 4, st));
+        return EW_OK;
+    }
     if (!topk_ids || !aid || !slot_ids || ((uintptr_t)topk_ids & 3) || ((uintptr_t)slot_ids & 3)) return EW_ERR_INVALID_ARG;
+    // the aligned kernel zeroes the counters itself (one launch per call) through two words of the pool's workspace:
+    // calls on different streams are ordered like forwards
+    const bool aligned = (((uintptr_t)topk_ids | (uintptr_t)slot_ids | (uintptr_t)aid) & 15) == 0;
+    if (aligned) {
+        ew_status_t ordered = order_after_other_streams(p, st);
+        if (ordered != EW_OK) return ordered;
+    } else if (counts) {
+        CU_TRY(cudaMemsetAsync(counts, 0, (size_t)p->P * 4, st));
+    }
     LAUNCH_TRY(launch_reroute(p, layer, topk_ids, aid, B, slot_ids, counts, st));
     return note_forward(p, st);
 }

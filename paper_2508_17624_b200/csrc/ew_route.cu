@@ -39,10 +39,15 @@ template <int N>
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 
 // (ids and slots may be the same buffer - the rewrite in place the ABI allows - so neither is __restrict__)
+//
+// The per-slot counts are overwritten, not accumulated, and the call is one launch: CTA 0 zeroes the caller's
+// counters and raises a flag in the pool's workspace; every CTA waits for that flag (bounded) before it adds its
+// histogram; the CTA that finishes last lowers the flag again for the next call.  All CTAs of the grid are resident
+// at once (one wave), so the wait cannot starve CTA 0.
 __global__ void __launch_bounds__(256) reroute_kernel(const int32_t *ids, const int32_t *__restrict__ aid,
                                                       const int32_t *__restrict__ pi, const int32_t *__restrict__ loaded,
                                                       int n_tokens, int k, int M, int N, int P,
-                                                      int32_t *slots, int32_t *__restrict__ counts, int *err) {
+                                                      int32_t *slots, int32_t *__restrict__ counts, int *err, int *sync) {
     extern __shared__ __align__(128) int32_t smem_i[];
     const int tile_ints_max = kRerouteTok * k;
     const int stage_ints = kRerouteTok + tile_ints_max;            // a stage = 256 adapter ids, then 256*k ids (both 16-byte multiples)
@@ -52,14 +57,21 @@ __global__ void __launch_bounds__(256) reroute_kernel(const int32_t *ids, const 
     __shared__ int abort_flag;
     for (int i = threadIdx.x; i < N * M; i += blockDim.x) pi_s[i] = pi[i];
     for (int i = threadIdx.x; i < N; i += blockDim.x) loaded_s[i] = loaded[i];
-    if (counts)
+    if (counts) {
         for (int i = threadIdx.x; i < P; i += blockDim.x) hist[i] = 0;
+        if (blockIdx.x == 0)
+            for (int i = threadIdx.x; i < P; i += blockDim.x) counts[i] = 0;
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < kRerouteStages; ++s) tc::mbar_init(tc::smem_u32(bars + s), 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    if (counts && blockIdx.x == 0 && threadIdx.x == 0) {        // the counters are zero: publish
+        __threadfence();
+        atomicExch(sync, 1);
+    }
     const unsigned div_magic = ((1u << 20) + k - 1) / k;
     const int n_tiles = (n_tokens + kRerouteTok - 1) / kRerouteTok;
     int flags = 0;
@@ -135,9 +147,26 @@ __global__ void __launch_bounds__(256) reroute_kernel(const int32_t *ids, const 
     if (threadIdx.x == 0) bulk_wait_read<0>();
     if (flags) atomicOr(err, flags);
     if (counts) {
+        if (threadIdx.x == 0) {                                  // wait (bounded) until CTA 0 has zeroed the counters
+            long long t0 = clock64();
+            while (atomicAdd(sync, 0) == 0) {
+                if (clock64() - t0 > tc::kWaitLimitCycles) { atomicOr(err, 2); abort_flag = 1; break; }
+                __nanosleep(64);
+            }
+            __threadfence();
+        }
         __syncthreads();
-        for (int i = threadIdx.x; i < P; i += blockDim.x)
-            if (hist[i]) atomicAdd(counts + i, hist[i]);
+        if (!abort_flag)
+            for (int i = threadIdx.x; i < P; i += blockDim.x)
+                if (hist[i]) atomicAdd(counts + i, hist[i]);
+        __syncthreads();
+        if (threadIdx.x == 0) {                                  // last CTA out lowers the flag for the next call
+            __threadfence();
+            if (atomicAdd(sync + 1, 1) == (int)gridDim.x - 1) {
+                atomicExch(sync + 1, 0);
+                atomicExch(sync, 0);
+            }
+        }
     }
 }
 
@@ -466,7 +495,7 @@ int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid
     const long long cap = (long long)p->sm_count * per_sm;
     if (blocks > cap) blocks = cap;
     reroute_kernel<<<(int)blocks, 256, smem, st>>>(ids, aid, pi, p->ws.loaded, B, c.top_k, c.num_experts, c.max_adapters,
-                                                   p->P, slots, counts, p->ws.err);
+                                                   p->P, slots, counts, p->ws.err, p->ws.err + 8);
     return (int)cudaGetLastError();
 }
 

@@ -204,3 +204,30 @@ def test_padding_mode_backs_everything():
     pool.unload_adapter(0)
     assert pool.stats()["pages_mapped"] == st["pages_mapped"]
     pool.destroy()
+
+
+def test_base_load_is_counted_once_and_a_failed_one_not_at_all():
+    """ew_load_base maps the base range on its first successful call only; loading a layer again overwrites in place
+    (same pages, same counters), and a first load that fails on the page budget leaves nothing mapped or counted, so
+    that a retry does not double anything."""
+    pool, cfg = mk(num_layers=2)
+    pool.load_base(0, None, None, None, None)
+    once = pool.stats()
+    pool.load_base(0, None, None, None, None)
+    again = pool.stats()
+    assert again == once and once["live_experts"] == 4
+    assert once["pages_mapped"] == expect_mapped(cfg, [set(range(4))])
+    pool.destroy()
+    # 4 experts of 3 MiB + 1.5 MiB: 6 + 3 pages per layer; a budget of 10 lets layer 0 in and stops layer 1 midway
+    pool, cfg = mk(num_layers=2, max_pages=10)
+    pool.load_base(0, None, None, None, None)
+    before = pool.stats()
+    for _ in range(2):                                   # the retry fails the same way and changes nothing either
+        with pytest.raises(binding.EwError) as ei:
+            pool.load_base(1, None, None, None, None)
+        assert ei.value.status == 2
+        st = pool.stats()
+        for key in ("pages_mapped", "live_experts", "live_expert_bytes"):     # nothing of layer 1 stays mapped or counted
+            assert st[key] == before[key], key
+        assert st["pages_mapped"] + st["pages_free"] == st["pages_created_total"] <= 10   # pages made on the way wait in the free list
+    pool.destroy()

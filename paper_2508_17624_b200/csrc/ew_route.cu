@@ -340,6 +340,142 @@ __global__ void __launch_bounds__(4 * kLogitTok) route_logits_kernel(const float
 }
 
 // ------------------------------------------------------------------------------------------------
+// The same operator for M <= 64 with about a third of the warp instructions per token (the kernel above spends most
+// of its issue slots on k arg-max-with-removal passes over register arrays).  Four lanes share a token, lane g owning
+// the sixteen experts [16g, 16g + 16): it loads them straight from global memory, exponentiates, and sorts its sixteen
+// probabilities ONCE with a 63-comparator network of max/min pairs (values only).  A selection round is then a
+// butterfly max over the four lanes' current heads, a ballot to find the lowest lane that holds the maximum (lower
+// lane = lower expert index: the tie rule between lanes) and a pop of that lane's head; the lane notes the round in a
+// bit mask.  After the k rounds a lane's wins are the first entries of its sorted list, in round order; only then
+// does it look their indices up among its sixteen originals (lowest index not taken yet: the tie rule inside a lane)
+// and write ids, weights and slots.  A warp serves eight tokens at a time, a CTA 256 tokens in four passes, so the
+// expert map and the histogram are staged once per 256 tokens.  DEEP: k > 8, a lane may win up to sixteen rounds.
+// ------------------------------------------------------------------------------------------------
+constexpr int kLogitTok4 = 256;      // tokens per CTA: 64 groups of four lanes, four passes
+
+template <bool DEEP>
+__global__ void __launch_bounds__(256) route_logits4_kernel(const float4 *__restrict__ logits, const int32_t *__restrict__ aid,
+                                                            const int32_t *__restrict__ pi, const int32_t *__restrict__ loaded,
+                                                            int B, int M, int k, int N, int P, int renormalize, float scale,
+                                                            int32_t *topk_ids, float *topk_w, int32_t *slot_ids,
+                                                            int32_t *counts, int *err) {
+    extern __shared__ __align__(16) int32_t rl4_smem[];
+    int32_t *hist_s = rl4_smem;              // [P]
+    int32_t *pi_s = hist_s + P;              // [N][M]
+    constexpr unsigned kFull = 0xffffffffu;
+    constexpr int kDepth = DEEP ? 16 : 8;    // entries of the sorted list that can still be popped
+    const int tid = threadIdx.x, lane = tid & 31, g = lane & 3;
+    const unsigned group_shift = lane & 28;  // first lane of this token's four within the warp
+    const int mv = M >> 2;
+
+    for (int i = tid; i < P; i += blockDim.x) hist_s[i] = 0;
+    for (int i = tid; i < N * M; i += blockDim.x) pi_s[i] = pi[i];
+    __syncthreads();
+
+#pragma unroll 1
+    for (int ps = 0; ps < kLogitTok4 / 64; ++ps) {
+        const int t = blockIdx.x * kLogitTok4 + ps * 64 + (tid >> 2);
+        if (blockIdx.x * kLogitTok4 + ps * 64 >= B) break;            // nothing left for the whole CTA
+        const bool live = t < B;
+        float e[16];
+        {
+            const float4 *row = logits + (size_t)t * mv;
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                float4 r = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+                if (live && 4 * g + h < mv) r = __ldg(row + 4 * g + h);
+                e[4 * h] = r.x; e[4 * h + 1] = r.y; e[4 * h + 2] = r.z; e[4 * h + 3] = r.w;
+            }
+        }
+        int a = live ? __ldg(aid + t) : -1;
+        if (a < -1 || a >= N || (a >= 0 && !loaded[a])) {
+            if (g == 0) atomicOr(err, 1);
+            a = -1;
+        }
+        float mx = e[0];
+#pragma unroll
+        for (int i = 1; i < 16; ++i) mx = fmaxf(mx, e[i]);
+        mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 2));
+        if (!live) mx = 0.f;
+        float sum = 0.f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {                    // exp(-inf) = 0 for the absent experts
+            e[i] = __expf(e[i] - mx);                     // ex2.approx: relative error about 5e-7 for the arguments that matter
+            sum += e[i];
+        }
+        sum += __shfl_xor_sync(kFull, sum, 1);
+        sum += __shfl_xor_sync(kFull, sum, 2);
+        const float inv_sum = 1.f / sum;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) e[i] = 16 * g + i < M ? e[i] * inv_sum : -1.f;   // absent experts below every real one
+
+        float s0[16];                                    // the lane's probabilities sorted descending
+#pragma unroll
+        for (int i = 0; i < 16; ++i) s0[i] = e[i];
+#define EW_CE(x, y) { const float hi_ = fmaxf(s0[x], s0[y]), lo_ = fminf(s0[x], s0[y]); s0[x] = hi_; s0[y] = lo_; }
+        EW_CE(0, 1) EW_CE(2, 3) EW_CE(0, 2) EW_CE(1, 3) EW_CE(1, 2) EW_CE(4, 5) EW_CE(6, 7) EW_CE(4, 6) EW_CE(5, 7)
+        EW_CE(5, 6) EW_CE(0, 4) EW_CE(2, 6) EW_CE(2, 4) EW_CE(1, 5) EW_CE(3, 7) EW_CE(3, 5) EW_CE(1, 2) EW_CE(3, 4)
+        EW_CE(5, 6) EW_CE(8, 9) EW_CE(10, 11) EW_CE(8, 10) EW_CE(9, 11) EW_CE(9, 10) EW_CE(12, 13) EW_CE(14, 15)
+        EW_CE(12, 14) EW_CE(13, 15) EW_CE(13, 14) EW_CE(8, 12) EW_CE(10, 14) EW_CE(10, 12) EW_CE(9, 13) EW_CE(11, 15)
+        EW_CE(11, 13) EW_CE(9, 10) EW_CE(11, 12) EW_CE(13, 14) EW_CE(0, 8) EW_CE(4, 12) EW_CE(4, 8) EW_CE(2, 10)
+        EW_CE(6, 14) EW_CE(6, 10) EW_CE(2, 4) EW_CE(6, 8) EW_CE(10, 12) EW_CE(1, 9) EW_CE(5, 13) EW_CE(5, 9)
+        EW_CE(3, 11) EW_CE(7, 15) EW_CE(7, 11) EW_CE(3, 5) EW_CE(7, 9) EW_CE(11, 13) EW_CE(1, 2) EW_CE(3, 4)
+        EW_CE(5, 6) EW_CE(7, 8) EW_CE(9, 10) EW_CE(11, 12) EW_CE(13, 14)
+#undef EW_CE
+        float s[kDepth];                                 // the part of it that is popped during the rounds
+#pragma unroll
+        for (int i = 0; i < kDepth; ++i) s[i] = s0[i];
+
+        unsigned won = 0;                                // bit r: this lane's head won round r
+        float wsum = 0.f;
+        for (int r = 0; r < k; ++r) {
+            float wv = s[0];
+            wv = fmaxf(wv, __shfl_xor_sync(kFull, wv, 1));
+            wv = fmaxf(wv, __shfl_xor_sync(kFull, wv, 2));
+            const unsigned holders = (__ballot_sync(kFull, s[0] == wv) >> group_shift) & 0xfu;
+            wsum += wv;
+            if (g == __ffs(holders) - 1) {               // the lowest lane that holds it pops its head
+                won |= 1u << r;
+#pragma unroll
+                for (int i = 0; i < kDepth - 1; ++i) s[i] = s[i + 1];
+                s[kDepth - 1] = -2.f;
+            }
+        }
+        // this lane's wins, in round order, are s0[0], s0[1], ...
+        unsigned taken = 0;
+        const float wnorm = renormalize ? scale / wsum : scale;
+#pragma unroll
+        for (int j = 0; j < kDepth; ++j) {
+            if (__any_sync(kFull, won != 0)) {
+                if (won) {
+                    const int r = __ffs(won) - 1;
+                    won &= won - 1;
+                    const float wv = s0[j];
+                    unsigned eq = 0;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) eq |= (e[i] == wv) ? (1u << i) : 0u;
+                    const int idx = __ffs(eq & ~taken) - 1;   // lowest index with that value not taken yet
+                    taken |= 1u << idx;
+                    if (live) {
+                        const int id = 16 * g + idx;
+                        const int slot = a < 0 ? id : pi_s[a * M + id];
+                        const size_t o = (size_t)t * k + r;
+                        topk_ids[o] = id;
+                        slot_ids[o] = slot;
+                        topk_w[o] = (renormalize || scale != 1.f) ? wv * wnorm : wv;
+                        atomicAdd(hist_s + slot, 1);
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < P; i += blockDim.x)
+        if (hist_s[i]) atomicAdd(counts + i, hist_s[i]);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Scan + permute + plan.  Every CTA recomputes the exclusive scan of the (small) count array in
 // shared memory; the first kPlanners CTAs publish the offsets and write the GEMM work items (the item
 // loop is a chain of dependent integer arithmetic, so it is spread over several CTAs), the other CTAs record for
@@ -456,7 +592,21 @@ int launch_route_logits(ew_pool *p, int layer, const float *logits, const int32_
     const int grid = (B + kLogitTok - 1) / kLogitTok;
     const int32_t *pi = p->layers[layer].pi_dev;
     cudaError_t e;
-    if (M <= 64) {
+    const size_t smem4 = ((size_t)p->P + (size_t)N * M) * 4;
+    if (M <= 64 && smem4 <= 160 * 1024) {
+        const int grid4 = (B + kLogitTok4 - 1) / kLogitTok4;
+        if (c.top_k > 8) {
+            e = cudaFuncSetAttribute(route_logits4_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem4);
+            if (e != cudaSuccess) return (int)e;
+            route_logits4_kernel<true><<<grid4, 256, smem4, st>>>((const float4 *)logits, aid, pi, p->ws.loaded, B, M, c.top_k, N, p->P,
+                                                                  c.renormalize, c.routed_scale, topk_ids, topk_w, slot_ids, counts, p->ws.err);
+        } else {
+            e = cudaFuncSetAttribute(route_logits4_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem4);
+            if (e != cudaSuccess) return (int)e;
+            route_logits4_kernel<false><<<grid4, 256, smem4, st>>>((const float4 *)logits, aid, pi, p->ws.loaded, B, M, c.top_k, N, p->P,
+                                                                   c.renormalize, c.routed_scale, topk_ids, topk_w, slot_ids, counts, p->ws.err);
+        }
+    } else if (M <= 64) {                                 // an expert map too large for the sorted kernel's shared memory
         e = cudaFuncSetAttribute(route_logits_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return (int)e;
         route_logits_kernel<16><<<grid, 4 * kLogitTok, smem, st>>>((const float4 *)logits, aid, pi, p->ws.loaded, B, M, c.top_k, N, p->P, c.renormalize,

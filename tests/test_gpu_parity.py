@@ -332,16 +332,20 @@ def test_reroute_operator_c4_sample():
     pool.destroy()
 
 
-@pytest.mark.parametrize("M,k,n,renorm", [(64, 6, 65536, 0), (64, 6, 4099, 1), (16, 2, 130, 0), (80, 3, 1000, 0),
-                                          (256, 8, 777, 1), (4, 4, 33, 0)])
-def test_route_from_logits(M, k, n, renorm):
+@pytest.mark.parametrize("M,k,n,renorm,quant", [(64, 6, 65536, 0, 0), (64, 6, 4099, 1, 0), (16, 2, 130, 0, 0), (80, 3, 1000, 0, 0),
+                                                (256, 8, 777, 1, 0), (4, 4, 33, 0, 0), (64, 16, 1000, 1, 0), (32, 32, 200, 0, 0),
+                                                (64, 6, 3000, 0, 1), (48, 12, 500, 1, 1), (128, 6, 300, 0, 1)])
+def test_route_from_logits(M, k, n, renorm, quant):
     """Softmax + top-k + rerouting + counts from given fp32 logits (the c4 recipe: N(0,1) logits, adapter ids per
-    token): ids equal the oracle's except where the k-th and (k+1)-th probabilities are within rounding of each other,
+    token; also k > 8, k = M, and logits with many exact ties): ids equal the oracle's except where the k-th and
+    (k+1)-th probabilities are within rounding of each other,
     weights to 2e-6 relative (same logits, different summation order), slots and counts bit-exact given the ids."""
     import torch
     N, e_max = 5, 3
     rng = np.random.default_rng(100 + M + k)
     logits = rng.standard_normal((n, M)).astype(np.float32)
+    if quant:                  # logits on a grid of 0.5: many exact ties, inside a lane's experts and between lanes
+        logits = (np.round(logits * 2) / 2).astype(np.float32)
     aid = rng.integers(-1, N, size=n).astype(np.int32)
     scale = 1.5 if renorm else 1.0
     pool = binding.Pool(hidden=64, inter=64, num_experts=M, num_shared=0, top_k=k, max_adapters=N, e_max=e_max,
@@ -362,6 +366,8 @@ def test_route_from_logits(M, k, n, renorm):
     assert pool.last_device_error() == 0
     ids, w, slots, cnt = ids.cpu().numpy(), w.cpu().numpy(), slots.cpu().numpy(), cnt.cpu().numpy()
     same = (ids == ids_o).all(axis=1)
+    if quant:                  # equal logits give equal probabilities on both sides: the tie rule decides, exactly
+        assert same.all(), "ties must go to the lower expert index, in the oracle's order"
     assert np.all(gap[~same] < 1e-6), "a routing decision differs where the probabilities are not tied"
     assert (~same).sum() <= max(1, n // 1000)
     assert np.allclose(w[same], w_o[same], rtol=2e-6, atol=1e-9)

@@ -143,7 +143,7 @@ int make_atom_map(ew_pool *p, CUtensorMap *out, const void *base, int H, int row
 
 // Kernel launchers (all asynchronous on `st`; return cudaError_t as int).
 int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B, cudaStream_t st);
-int launch_permute(ew_pool *p, const void *x, int B, cudaStream_t st);
+int launch_permute(ew_pool *p, int B, cudaStream_t st);
 int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, const CUtensorMap &map_x_big, const void *x, int B,
                  cudaStream_t st);
 int pick_token_tile(const ew_pool *p, int B);

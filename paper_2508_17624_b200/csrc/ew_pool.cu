@@ -611,7 +611,7 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     p->counts_clean = false;
     LAUNCH_TRY(launch_route(p, layer, x, aid, B, st));
     PROF_MARK(1);
-    LAUNCH_TRY(launch_permute(p, x, B, st));
+    LAUNCH_TRY(launch_permute(p, B, st));
     PROF_MARK(2);
     if (topk_ids) CU_TRY(cudaMemcpyAsync(topk_ids, p->ws.topk_ids, nk * 4, cudaMemcpyDeviceToDevice, st));
     if (topk_w) CU_TRY(cudaMemcpyAsync(topk_w, p->ws.topk_w, nk * 4, cudaMemcpyDeviceToDevice, st));

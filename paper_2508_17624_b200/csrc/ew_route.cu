@@ -561,7 +561,7 @@ int pick_token_tile(const ew_pool *p, int B) {
     return want <= 32 ? 32 : want <= 64 ? 64 : want <= 192 ? 128 : 256;
 }
 
-int launch_permute(ew_pool *p, const void *, int B, cudaStream_t st) {
+int launch_permute(ew_pool *p, int B, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
     plan::Params A;
     A.B = B; A.k = c.top_k; A.P = p->P; A.S = c.num_shared;

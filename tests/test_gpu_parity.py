@@ -724,6 +724,35 @@ def test_side_stream_and_cuda_graph():
     pool.destroy()
 
 
+def test_cuda_graph_of_a_prefill_sized_forward():
+    """A prefill-sized batch (thin and fat item lists, CTA-pair kernels launched as clusters with programmatic
+    dependent launch) captured into a CUDA graph after one warm-up call replays with the bits of a direct call."""
+    import torch
+    cfg = wl.MoEConfig(name="odd", num_layers=1, seed=31, hidden=192, inter=136, num_experts=6, num_shared=1, top_k=2,
+                       max_adapters=8, e_max=2, n_tokens=2500)
+    bank = wl.NoiseBank(cfg.seed)
+    pool = binding.Pool.from_config(cfg)
+    tuned = wl.tuned_sets(cfg, np.array([[2], [1], [2], [1], [2], [2], [1], [2]]))
+    binding.load_model(pool, cfg, bank, tuned=tuned)
+    x, aid = to_dev(wl.gen_tokens(cfg)), to_dev(wl.gen_adapter_ids(cfg, mode="uniform"))
+    ref = pool.moe_forward(0, x, aid).clone()            # the warm-up call
+    torch.cuda.synchronize()
+    counts = pool.moe_forward_debug(0, x, aid)["counts"].cpu().numpy()
+    assert counts.max() > 256 and ((counts > 0) & (counts <= 128)).any()      # both item lists are in play
+    g = torch.cuda.CUDAGraph()
+    out = torch.zeros_like(x)
+    with torch.cuda.graph(g):
+        pool.moe_forward(0, x, aid, out)
+    for _ in range(3):
+        out.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, ref)
+    assert torch.equal(pool.moe_forward(0, x, aid), ref)
+    assert pool.last_device_error() == 0
+    pool.destroy()
+
+
 def test_two_pools_on_one_device():
     import torch
     c0, c1 = wl.CONFIGS["c0"], wl.with_(wl.CONFIGS["c0"], seed=5, max_adapters=1)

@@ -63,6 +63,17 @@ def run_layer(cfg, layer=0, n_tokens=None, aid_mode=None, adapters=None, sample=
                 n_checked=x.shape[0] if sample is None else len(sample))
 
 
+def oracle_check(pool, cfg, olayer, x_bits, aid_np, out, layer=0):
+    """`out` (a forward's result obtained some other way: another entry point, another stream, a graph replay) has
+    the bits of a debug forward on the same inputs, and that forward matches the oracle stage by stage."""
+    import torch
+    r = pool.moe_forward_debug(layer, to_dev(x_bits), to_dev(aid_np))
+    torch.cuda.synchronize()
+    assert torch.equal(r["out"], out)
+    ids, w, slots, _ = check_routing(cfg, olayer, x_bits, aid_np, r)
+    check_output(olayer, x_bits, slots, w, bf16_to_f32(r["out"]))
+
+
 def test_c0_tiny_layer():
     res = run_layer(wl.CONFIGS["c0"])
     assert res["flips"] <= 2
@@ -229,11 +240,15 @@ def test_load_unload_on_device():
     changed = (aid == 1).cpu().numpy()
     same = torch.equal(part[~torch.from_numpy(changed).cuda()], full[~torch.from_numpy(changed).cuda()])
     assert same
+    x_bits, aid_np = wl.gen_tokens(cfg), wl.gen_adapter_ids(cfg)
+    oracle_check(pool, cfg, oracle_layer(cfg, 0, bank, tuned, base=bases[0], adapters=[0]), x_bits,
+                 np.where(aid_np == 1, -1, aid_np).astype(np.int32), part)
     ew = wl.gen_adapter_layer(cfg, 1, 0, tuned[1][0], bank)
     pool.load_adapter(1, np.array([3], np.int32), tuned[1][0], ew.w_gate, ew.w_up, ew.w_down)
     again = pool.moe_forward(0, x, aid)
     torch.cuda.synchronize()
     assert torch.equal(again, full)
+    oracle_check(pool, cfg, oracle_layer(cfg, 0, bank, tuned, base=bases[0]), x_bits, aid_np, again)
     assert pool.stats()["pages_mapped"] == st_full["pages_mapped"]
     pool.destroy()
 
@@ -256,6 +271,7 @@ def test_adapter_weights_from_device_memory():
     out = pool.moe_forward(0, x, aid)
     torch.cuda.synchronize()
     assert torch.equal(out, ref)
+    oracle_check(pool, cfg, oracle_layer(cfg, 0, bank, tuned), wl.gen_tokens(cfg), wl.gen_adapter_ids(cfg), out)
     pool.destroy()
 
 
@@ -750,6 +766,7 @@ def test_cuda_graph_of_a_prefill_sized_forward():
         assert torch.equal(out, ref)
     assert torch.equal(pool.moe_forward(0, x, aid), ref)
     assert pool.last_device_error() == 0
+    oracle_check(pool, cfg, oracle_layer(cfg, 0, bank, tuned), wl.gen_tokens(cfg), wl.gen_adapter_ids(cfg, mode="uniform"), out)
     pool.destroy()
 
 
@@ -894,8 +911,14 @@ def test_host_buffer_pipeline():
         assert torch.equal(direct, direct_ref)
         for (xh, ah, oh), r in zip(host, ref):
             assert torch.equal(oh.cuda().view(torch.bfloat16), r), rep
-            oh.zero_()
+            if rep < 2:
+                oh.zero_()
     assert pool.last_device_error() == 0
+    # what arrived in the host buffer of the first batch is the oracle's layer output
+    xh, ah, oh = host[0]
+    bank = wl.NoiseBank(cfg.seed)
+    oracle_check(pool, cfg, oracle_layer(cfg, 0, bank, wl.tuned_sets(cfg)), xh.numpy().view(np.uint16), ah.numpy(),
+                 oh.cuda().view(torch.bfloat16))
     pool.destroy()
 
 

@@ -196,7 +196,10 @@ ew_status_t ew_profile_read(ew_pool_t *pool, double *ms, int32_t *n_forwards);
  * if counts is not null, the number of pairs per slot (counts is overwritten, not accumulated).
  * All pointers DEVICE: topk_ids, slot_ids [n_tokens,k] int32 (may alias), adapter_ids [n_tokens],
  * counts [M + N*E_max].  n_tokens is not limited by max_tokens.  Ids outside [0,M) are passed
- * through unchanged and flagged in the device error word. */
+ * through unchanged and flagged in the device error word; adapter ids outside [-1,N) or of an adapter that
+ * is not loaded behave as -1 and are flagged.  With 16-byte-aligned buffers a call is one kernel launch
+ * (the kernel zeroes the counters itself, through two handshake words in the pool's workspace); calls on
+ * different streams are therefore ordered by the pool like forwards.  Asynchronous on cuda_stream. */
 ew_status_t ew_reroute(ew_pool_t *pool, int32_t layer, const int32_t *topk_ids, const int32_t *adapter_ids,
                        int32_t n_tokens, int32_t *slot_ids, int32_t *counts, void *cuda_stream);
 

@@ -179,7 +179,8 @@ def layer_bytes_and_flops(cfg, live):
     blk = cfg.inter * cfg.hidden * 2
     return {
         "bytes_gemm1": groups * 2 * blk + (pairs + B) * H * 2 + rows_act * cfg.inter * 2,     # weights + rows in + act out
-        "bytes_gemm2": groups * blk + rows_act * cfg.inter * 2 + rows_act * H * 4,
+        # weights + act rows in + Y rows out (the shared experts are chained along K: one Y row per token for all of them)
+        "bytes_gemm2": groups * blk + rows_act * cfg.inter * 2 + (pairs + (B if cfg.num_shared else 0)) * H * 4,
         "bytes_layer": groups * 3 * blk,
         "flops_gemm1": 2.0 * rows_act * 2 * cfg.inter * H,
         "flops_gemm2": 2.0 * rows_act * cfg.inter * H,

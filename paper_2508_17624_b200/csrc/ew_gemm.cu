@@ -142,27 +142,32 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
                 // GEMM-1: only the shared experts' rows (contiguous in x) come by TMA
                 const bool tma_tokens = !GATHER || it.from_x;
                 const uint32_t b_bytes = !tma_tokens ? 0 : big ? NT * kBlockK * 2 : nchunk * kChunkBytes;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                // GEMM-2 of the shared experts: the K loop runs over it.chain experts (slot, slot + 1, ...) whose
+                // activation blocks lie it.chain_rows rows apart
+                const int n_stage = (GLU ? 1 : it.chain) * num_kb;
+                for (int st = 0, kb = 0, ch = 0; st < n_stage; ++st) {
                     if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1, abort_flag, err))) break;
                     const uint32_t sa = smem_base + stage * C::kStageBytes;
                     const uint32_t full = bar_full + 8 * stage;
+                    const int in_row = it.in_row + ch * it.chain_rows;
                     mbar_expect_tx(full, (GLU ? 2 : 1) * kATileBytes + b_bytes);
                     if (GLU) {
                         tma_load_3d(sa, &map_w, kb * kBlockK, it.tile * kTileRows, it.slot * 2, full);
                         tma_load_3d(sa + kATileBytes, &map_w, kb * kBlockK, it.tile * kTileRows, it.slot * 2 + 1, full);
                     } else {
-                        tma_load_3d(sa, &map_w, kb * kBlockK, it.tile * kTileRows, it.slot, full);
+                        tma_load_3d(sa, &map_w, kb * kBlockK, it.tile * kTileRows, it.slot + ch, full);
                     }
                     const uint32_t sb = sa + (GLU ? 2 : 1) * kATileBytes;
                     if (!tma_tokens) {
                         // the token operand of this stage is written by the gather warps
                     } else if (big) {
-                        tma_load_2d(sb, amap, kb * kBlockK, it.in_row, full);
+                        tma_load_2d(sb, amap, kb * kBlockK, in_row, full);
                     } else {
                         for (int c = 0; c < nchunk; ++c)
-                            tma_load_2d(sb + c * kChunkBytes, amap, kb * kBlockK, it.in_row + c * kChunkRows, full);
+                            tma_load_2d(sb + c * kChunkBytes, amap, kb * kBlockK, in_row + c * kChunkRows, full);
                     }
                     if (++stage == C::kStages) { stage = 0; phase ^= 1; }
+                    if (++kb == num_kb) { kb = 0; ++ch; }
                 }
             }
         }
@@ -178,7 +183,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
                 if (!(ok = mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, abort_flag, err))) break;
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + acc * C::kAccCols;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                const int n_stage = (GLU ? 1 : it.chain) * num_kb;
+                for (int kb = 0; kb < n_stage; ++kb) {
                     if (!(ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, err))) break;
                     if (GATHER) fence_proxy_async_smem();           // the token rows were written by cp.async, not by TMA
                     tc_fence_after();
@@ -426,14 +432,16 @@ fat_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
                 const int wrow = GLU ? it.tile * kTileRows : (it.tile * 2 + (int)rank) * kTileRows;
                 const int wz = GLU ? it.slot * 2 + (int)rank : it.slot;
                 const uint32_t bytes = (uint32_t)(2 * kATileBytes + (tma_tokens ? 2 * kATileBytes : 0));   // of both CTAs
-                for (int kb = 0; kb < num_kb; ++kb) {
+                const int n_stage = (GLU ? 1 : it.chain) * num_kb;           // GEMM-2 of the shared experts: chained along K
+                for (int st = 0, kb = 0, ch = 0; st < n_stage; ++st) {
                     if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1, abort_flag, err))) break;
                     const uint32_t sa = smem_base + stage * C::kStageBytes;
                     const uint32_t full = leader_addr(bar_full + 8 * stage);
                     if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, bytes);
-                    tma2_load_3d(sa + kATileBytes, &map_w, kb * kBlockK, wrow, wz, full);
-                    if (tma_tokens) tma2_load_2d(sa, &map_a, kb * kBlockK, arow, full);
+                    tma2_load_3d(sa + kATileBytes, &map_w, kb * kBlockK, wrow, wz + (GLU ? 0 : ch), full);
+                    if (tma_tokens) tma2_load_2d(sa, &map_a, kb * kBlockK, arow + ch * it.chain_rows, full);
                     if (++stage == C::kStages) { stage = 0; phase ^= 1; }
+                    if (++kb == num_kb) { kb = 0; ++ch; }
                 }
             }
         }
@@ -444,10 +452,11 @@ fat_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
             const uint32_t idesc = instr_desc_m256(kFatN);
             bool ok = true;
             for (int w = pair_id; w < n_items && ok; w += n_pairs) {
+                const int n_stage = (GLU ? 1 : items[w].chain) * num_kb;
                 if (!(ok = mbar_wait_cluster(bar_tempty + 8 * acc, acc_phase ^ 1, abort_flag, err))) break;
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + acc * kFatN;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = 0; kb < n_stage; ++kb) {
                     if (!(ok = mbar_wait_cluster(bar_full + 8 * stage, phase, abort_flag, err))) break;
                     tc_fence_after();
                     const uint32_t sa = smem_base + stage * C::kStageBytes;

@@ -22,7 +22,9 @@ struct alignas(16) GemmItem {
     int32_t out_row;    // first output row
     int32_t rows;       // token rows in this item
     int32_t from_x;     // 1: activation rows come straight from the caller's x (shared experts)
-    int32_t pad0, pad1;
+    int32_t chain;      // experts chained along K in this item (GEMM-2 of the shared experts: S; otherwise 1): the
+                        // item's K loop runs over slots slot .. slot + chain - 1, whose activation blocks start
+    int32_t chain_rows; // chain_rows rows apart, and accumulates them into one output block
 };
 
 struct Workspace {

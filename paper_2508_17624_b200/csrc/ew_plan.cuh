@@ -96,11 +96,16 @@ __device__ inline void write_items(int32_t *sm, const int32_t *cnt_s, const Para
     __syncthreads();
     block_exclusive_scan(nblk, blk, G, warp_sums, nthreads);
     block_exclusive_scan(nblk_t, blk_t, G, warp_sums, nthreads);
+    // GEMM-2 runs the S shared experts as ONE group chained along K (out[t] = sum_s Wdown_s . act_s[t] is a single
+    // product over the concatenated K), so that one fp32 row per token is written and read back instead of S: the
+    // shared groups 1 .. S-1 (same row count as group 0, hence the same blocks) emit no GEMM-2 items.
+    const int skip_t = S > 1 ? (S - 1) * nblk_t[0] : 0, skip_f = S > 1 ? (S - 1) * nblk[0] : 0;
+    const int y_base = S > 0 ? B : 0;                      // rows of Y: [0, B) the shared sum, then the routed rows
     if (publish && threadIdx.x == 0) {
         A.n_items[0] = blk_t[G] * A.R1;
-        A.n_items[1] = blk_t[G] * A.R2;
+        A.n_items[1] = (blk_t[G] - skip_t) * A.R2;
         A.n_items[2] = blk[G] * A.RF1;
-        A.n_items[3] = blk[G] * A.RF2;
+        A.n_items[3] = (blk[G] - skip_f) * A.RF2;
     }
     for (int g = first_warp; g < G; g += warp_stride) {
         const bool shared = g < S;
@@ -108,31 +113,34 @@ __device__ inline void write_items(int32_t *sm, const int32_t *cnt_s, const Para
         if (rows == 0) continue;
         const int slot = shared ? P + g : g - S;
         const int in0 = shared ? 0 : off[g - S];                  // GEMM-1 reads x rows (shared) or slot-contiguous rows
-        const int out0 = shared ? g * B : S * B + off[g - S];     // rows of act / Y; GEMM-2 reads what GEMM-1 wrote
+        const int act0 = shared ? g * B : S * B + off[g - S];     // rows of act: GEMM-1 writes them, GEMM-2 reads them
+        const int y0 = shared ? 0 : y_base + off[g - S];          // rows of Y
         for (int pass = 0; pass < 2; ++pass) {
+            if (pass && shared && g > 0) continue;                // chained into group 0's items
             const int from_x = (!pass && shared) ? 1 : 0;
-            const int in_base = pass ? out0 : in0;
+            const int in_base = pass ? act0 : in0, out_base = pass ? y0 : act0;
+            const int chain = (pass && shared) ? S : 1;
             // thin items
             const int nt = nblk_t[g], Rt = pass ? A.R2 : A.R1;
-            GemmItem *dst = (pass ? A.items2 : A.items1) + (size_t)blk_t[g] * Rt;
+            GemmItem *dst = (pass ? A.items2 : A.items1) + (size_t)(blk_t[g] - ((pass && !shared) ? skip_t : 0)) * Rt;
             const int thin0 = A.fat ? (rows / kFatRows) * kFatRows : 0;      // first row of the (only) thin block
             for (int i = lane; i < nt * Rt; i += 32) {
                 const int tile = i / nt, c = i % nt;
                 const int r0 = thin0 + c * A.NT;
                 const int item_rows = A.fat ? rows - thin0 : min(A.NT, rows - r0);
                 int4 *d4 = reinterpret_cast<int4 *>(dst + i);        // one item = two 16-byte stores
-                d4[0] = make_int4(slot, tile, in_base + r0, out0 + r0);
-                d4[1] = make_int4(item_rows, from_x, 0, 0);
+                d4[0] = make_int4(slot, tile, in_base + r0, out_base + r0);
+                d4[1] = make_int4(item_rows, from_x, chain, B);
             }
             // fat items
             const int nf = nblk[g], Rf = pass ? A.RF2 : A.RF1;
-            GemmItem *dstf = (pass ? A.fat2 : A.fat1) + (size_t)blk[g] * Rf;
+            GemmItem *dstf = (pass ? A.fat2 : A.fat1) + (size_t)(blk[g] - ((pass && !shared) ? skip_f : 0)) * Rf;
             for (int i = lane; i < nf * Rf; i += 32) {
                 const int tile = i / nf, c = i % nf;
                 const int r0 = c * kFatRows;
                 int4 *d4 = reinterpret_cast<int4 *>(dstf + i);
-                d4[0] = make_int4(slot, tile, in_base + r0, out0 + r0);
-                d4[1] = make_int4(min(kFatRows, rows - r0), from_x, 0, 0);
+                d4[0] = make_int4(slot, tile, in_base + r0, out_base + r0);
+                d4[1] = make_int4(min(kFatRows, rows - r0), from_x, chain, B);
             }
         }
     }

@@ -513,7 +513,9 @@ __global__ void __launch_bounds__(256) permute_kernel(const int32_t *slot_ids, c
 }
 
 // ------------------------------------------------------------------------------------------------
-// out[t] = sum_j w[t,j] * Y[S*B + inv[t,j]] + sum_q Y[q*B + t], fp32, j in router order, one rounding
+// out[t] = sum_j w[t,j] * Y[Yb + inv[t,j]] + Y[t], fp32, j in router order, one rounding.  Rows [0, B) of Y hold the
+// sum of the shared experts' outputs (GEMM-2 chains them along K); the routed rows start at Yb = B (0 without shared
+// experts).
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) combine_kernel(const float4 *y, const int32_t *inv,
                                                       const float *w, int B, int k, int H, int S,
@@ -525,8 +527,9 @@ __global__ void __launch_bounds__(256) combine_kernel(const float4 *y, const int
     tc::pdl_wait();                                     // expert outputs come from GEMM-2
     if (t == 0)                                         // the slot counters are spent: leave them zero for the next forward
         for (int i = threadIdx.x; i < P; i += blockDim.x) counts[i] = 0;
+    const int y_base = S > 0 ? B : 0;
     if (threadIdx.x < k) {
-        rows[threadIdx.x] = S * B + inv[(size_t)t * k + threadIdx.x];
+        rows[threadIdx.x] = y_base + inv[(size_t)t * k + threadIdx.x];
         wts[threadIdx.x] = w[(size_t)t * k + threadIdx.x];
     }
     __syncthreads();
@@ -539,8 +542,8 @@ __global__ void __launch_bounds__(256) combine_kernel(const float4 *y, const int
             acc.x = fmaf(wj, a.x, acc.x); acc.y = fmaf(wj, a.y, acc.y);
             acc.z = fmaf(wj, a.z, acc.z); acc.w = fmaf(wj, a.w, acc.w);
         }
-        for (int q = 0; q < S; ++q) {
-            const float4 a = y[((size_t)q * B + t) * hv + v];
+        if (S > 0) {
+            const float4 a = y[(size_t)t * hv + v];
             acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
         }
         const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);

@@ -192,7 +192,7 @@ __global__ void __launch_bounds__(256) reroute_kernel_unaligned(const int32_t *i
 // slot = Pi[aid][id], per-slot counts.  A CTA owns 128 tokens; the threads copy their logits [128, M] fp32 into
 // shared memory with coalesced 16-byte loads, rows M + 1 words apart so that the per-token reads that follow spread
 // over the banks.  Four neighbouring lanes of a warp share a token, lane g of the four owning the experts
-// [EPT*g, EPT*g + EPT) in registers (EPT = 16 for M <= 64, else 64).  Softmax by partial max and partial sum,
+// [EPT*g, EPT*g + EPT) in registers (EPT = 64: this kernel serves M > 64; smaller M takes the sorted kernel below).  Softmax by partial max and partial sum,
 // exchanged with two butterfly shuffles; then k rounds in which every lane offers its best remaining candidate and
 // the four settle the token's best the same way - no block-wide barrier after the tile has landed.  Counts go
 // through a shared-memory histogram, one atomic per non-empty slot and CTA.
@@ -590,13 +590,13 @@ int launch_route_logits(ew_pool *p, int layer, const float *logits, const int32_
                         float *topk_w, int32_t *slot_ids, int32_t *counts, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
     const int M = c.num_experts, N = c.max_adapters;
-    const size_t smem = ((size_t)kLogitTok * (M + 1) + p->P + (size_t)N * M) * 4;
-    if (smem > 227 * 1024) return (int)cudaErrorInvalidConfiguration;
+    const size_t smem = ((size_t)kLogitTok * (M + 1) + p->P + (size_t)N * M) * 4;      // the M > 64 kernel: tile + histogram + map
     const int grid = (B + kLogitTok - 1) / kLogitTok;
     const int32_t *pi = p->layers[layer].pi_dev;
     cudaError_t e;
     const size_t smem4 = ((size_t)p->P + (size_t)N * M) * 4;
-    if (M <= 64 && smem4 <= 160 * 1024) {
+    if (M <= 64) {
+        if (smem4 > 200 * 1024) return (int)cudaErrorInvalidConfiguration;   // expert map + histogram beyond shared memory
         const int grid4 = (B + kLogitTok4 - 1) / kLogitTok4;
         if (c.top_k > 8) {
             e = cudaFuncSetAttribute(route_logits4_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem4);
@@ -609,12 +609,8 @@ int launch_route_logits(ew_pool *p, int layer, const float *logits, const int32_
             route_logits4_kernel<false><<<grid4, 256, smem4, st>>>((const float4 *)logits, aid, pi, p->ws.loaded, B, M, c.top_k, N, p->P,
                                                                    c.renormalize, c.routed_scale, topk_ids, topk_w, slot_ids, counts, p->ws.err);
         }
-    } else if (M <= 64) {                                 // an expert map too large for the sorted kernel's shared memory
-        e = cudaFuncSetAttribute(route_logits_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return (int)e;
-        route_logits_kernel<16><<<grid, 4 * kLogitTok, smem, st>>>((const float4 *)logits, aid, pi, p->ws.loaded, B, M, c.top_k, N, p->P, c.renormalize,
-                                                                   c.routed_scale, topk_ids, topk_w, slot_ids, counts, p->ws.err);
     } else {
+        if (smem > 227 * 1024) return (int)cudaErrorInvalidConfiguration;
         e = cudaFuncSetAttribute(route_logits_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return (int)e;
         route_logits_kernel<64><<<grid, 4 * kLogitTok, smem, st>>>((const float4 *)logits, aid, pi, p->ws.loaded, B, M, c.top_k, N, p->P, c.renormalize,

@@ -13,6 +13,12 @@
 // k arg-max rounds (probability descending, lower index on ties), looks each chosen expert up in the
 // layer's expert map Pi (staged in shared memory) under the token's adapter id, and bumps the slot's
 // counter; the atomic's return value is the pair's position inside the slot's chunk.
+//
+// Small batches (32-token tiles that leave most SMs idle) split K over a cluster: the 4 or 8 CTAs of a cluster own one
+// token tile and a quarter or an eighth of the K range each, so the chain of dependent load rounds is one or two stages
+// long instead of eight; every CTA sends its partial logits to the cluster's first CTA through distributed shared
+// memory, and that CTA adds them in rank order (the sum does not depend on timing) and runs the epilogue.
+#include <cstdlib>
 #include <mutex>
 #include <string>
 
@@ -37,11 +43,24 @@ __device__ __forceinline__ int checked_aid(int a, int N, const int32_t *loaded, 
     return a;
 }
 
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+// store into the same shared-memory offset of the cluster's CTA 0
+__device__ __forceinline__ void st_leader_f32(const float *local_ptr, float v) {
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, 0;\n\t"
+        "st.shared::cluster.f32 [ra], %1;\n\t}"
+        ::"r"(smem_u32(local_ptr)), "f"(v) : "memory");
+}
+
 struct RouterArgs {
     const int32_t *aid, *pi, *loaded;
     int B, H, M, k, N, renormalize;
     float scale;
     int stages, tmem_cols, pi_in_smem, tok_tile, atoms;
+    int ksplit;            // CTAs per cluster that share one token tile, each with 1/ksplit of K (1: no cluster)
+    int part_off;          // byte offset of the partial-logit buffer [ksplit][n_mma][32] floats in shared memory
     int32_t *topk_ids;
     float *topk_w;
     int32_t *slot_ids, *rank, *counts;
@@ -97,9 +116,15 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
     float *pbuf = reinterpret_cast<float *>(smem_al);                // [M][128]; aliases the ring once it has drained
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_atoms = A.H / kBlockK;
+    // K split over a cluster: CTA `krank` of the `cs` CTAs that share token tile `blockIdx.x / cs` owns the K-atoms
+    // [atom0, atom0 + num_atoms)
+    const int cs = A.ksplit;
+    const int krank = cs > 1 ? (int)cluster_ctarank() : 0;
+    const int atoms_all = A.H / kBlockK, atoms_per = (atoms_all + cs - 1) / cs;
+    const int atom0 = krank * atoms_per;
+    const int num_atoms = max(0, min(atoms_per, atoms_all - atom0));
     const int num_kb = (num_atoms + kAtoms - 1) / kAtoms;
-    const int tok0 = blockIdx.x * tok_tile;
+    const int tok0 = (cs > 1 ? (int)blockIdx.x / cs : (int)blockIdx.x) * tok_tile;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -134,11 +159,12 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                 if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1, abort_flag, A.err)) break;
                 const uint32_t sa = smem_base + stage * stage_bytes, full = bar_full + 8 * stage;
                 mbar_expect_tx(full, kAtoms * (tok_tile + n_mma) * kBlockK * 2);
-                tma_load_3d(sa, &map_x, 0, tok0, kb * kAtoms, full);
-                tma_load_3d(sa + x_bytes, &map_r, 0, 0, kb * kAtoms, full);
+                tma_load_3d(sa, &map_x, 0, tok0, atom0 + kb * kAtoms, full);
+                tma_load_3d(sa + x_bytes, &map_r, 0, 0, atom0 + kb * kAtoms, full);
                 if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1; }
             }
         }
+        if (cs > 1) cluster_arrive();                                // every thread of the cluster arrives exactly once
     } else if (warp == 1) {
         if (lane == 0) {                                             // MMA issuer
             uint32_t stage = 0, phase = 0;
@@ -160,6 +186,7 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
             }
             if (ok) tc_commit(bar_done);
         }
+        if (cs > 1) cluster_arrive();
     } else if (REG && tok_tile == 32) {
         // epilogue for 32-token tiles (small batches, where this kernel's latency is exposed): the logits sit in
         // TMEM lanes 0..31 only, which one warp can read; that warp spills them to shared memory and then all four
@@ -173,24 +200,46 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
         auto quad_sync = [] { asm volatile("bar.sync 1, 128;" ::: "memory"); };   // the four epilogue warps
         mbar_wait(bar_done, 0, abort_flag, A.err);
         quad_sync();                                                 // every epilogue thread is past its (bounded) wait
-        if (!*abort_flag) {
+        float *lg_s = reinterpret_cast<float *>(smem_al);            // [n_mma][32] logits, expert-major (the ring has drained)
+        float *red_s = lg_s + 64 * 32;                               // [2][4][32] partial max, partial sum
+        float *cv_s = red_s + 2 * 4 * 32;                            // [2][4][32] candidate values, double-buffered by round
+        int *ci_s = reinterpret_cast<int *>(cv_s + 2 * 4 * 32);      // [2][4][32] candidate expert ids
+        float *part_s = reinterpret_cast<float *>(smem_al + A.part_off);   // K split: [cs][n_mma][32] partial logits (CTA 0's is used)
+        if (!*abort_flag && g == 0) {
             tc_fence_after();
-            float *lg_s = reinterpret_cast<float *>(smem_al);        // [n_mma][32] logits, expert-major (the ring has drained)
-            float *red_s = lg_s + 64 * 32;                           // [2][4][32] partial max, partial sum
-            float *cv_s = red_s + 2 * 4 * 32;                        // [2][4][32] candidate values, double-buffered by round
-            int *ci_s = reinterpret_cast<int *>(cv_s + 2 * 4 * 32);  // [2][4][32] candidate expert ids
-            if (g == 0) {
-                uint32_t v0[32], v1[32];
-                if (n_mma >= 32) tc_ld32(tmem_base, v0); else tc_ld16(tmem_base, v0);
-                if (n_mma > 32) { if (n_mma - 32 >= 32) tc_ld32(tmem_base + 32, v1); else tc_ld16(tmem_base + 32, v1); }
-                tc_wait_ld();
+            uint32_t v0[32], v1[32];
+            if (n_mma >= 32) tc_ld32(tmem_base, v0); else tc_ld16(tmem_base, v0);
+            if (n_mma > 32) { if (n_mma - 32 >= 32) tc_ld32(tmem_base + 32, v1); else tc_ld16(tmem_base + 32, v1); }
+            tc_wait_ld();
+            if (cs == 1) {
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     if (j < n_mma) lg_s[j * 32 + lane] = __uint_as_float(v0[j]);
                     if (32 + j < n_mma) lg_s[(32 + j) * 32 + lane] = __uint_as_float(v1[j]);
                 }
+            } else {                                                 // this CTA's share of K: to the cluster's first CTA
+                float *mine = part_s + krank * (n_mma * 32);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    if (j < n_mma) st_leader_f32(mine + j * 32 + lane, num_atoms ? __uint_as_float(v0[j]) : 0.f);
+                    if (32 + j < n_mma) st_leader_f32(mine + (32 + j) * 32 + lane, num_atoms ? __uint_as_float(v1[j]) : 0.f);
+                }
             }
-            quad_sync();
+        }
+        if (cs > 1) {
+            cluster_arrive();
+            if (krank == 0) {
+                cluster_wait();                                      // all partial logits have landed here
+                const int tid2 = (int)threadIdx.x - 64;              // 0..127 over the four epilogue warps
+                for (int i = tid2; i < n_mma * 32; i += 128) {
+                    float acc = part_s[i];
+                    for (int r = 1; r < cs; ++r) acc += part_s[r * (n_mma * 32) + i];    // rank order: independent of timing
+                    lg_s[i] = acc;
+                }
+            }
+        }
+        quad_sync();
+        if (!*abort_flag && krank == 0) {
             float p[16];
             float mx = -INFINITY;
 #pragma unroll
@@ -401,10 +450,15 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
 
 // Launch geometry of the router kernel for a batch of B tokens: tokens per CTA, K-atoms per stage, ring depth.
 struct RouterGeometry {
-    int tok_tile, atoms, stages, pi_in_smem, tmem_cols, grid;
+    int tok_tile, atoms, stages, pi_in_smem, tmem_cols, grid, ksplit, part_off;
     bool reg;
     size_t smem;
 };
+
+static bool ksplit_enabled() {       // EW_DISABLE_KSPLIT=1: every CTA runs the whole K range (debugging and A/B runs)
+    static const bool on = [] { const char *e = getenv("EW_DISABLE_KSPLIT"); return !(e && e[0] == '1'); }();
+    return on;
+}
 
 static bool router_geometry(const ew_pool *p, int B, RouterGeometry *g) {
     const ew_config_t &c = p->cfg;
@@ -413,21 +467,35 @@ static bool router_geometry(const ew_pool *p, int B, RouterGeometry *g) {
     g->tok_tile = B <= 32 * p->sm_count ? 32 : B <= 64 * p->sm_count ? 64 : 128;
     const size_t pi_bytes = (size_t)c.max_adapters * M * 4;
     g->pi_in_smem = pi_bytes <= (size_t)kMaxPiSmem;
-    const size_t tail = 1024 /*alignment*/ + kTileRows * kBlockK * 2 + 8 * (2 * kMaxStages + 1) + 16 +
-                        (g->pi_in_smem ? pi_bytes : 0) + 64;
     g->reg = M <= 64;
+    const int tiles = (B + g->tok_tile - 1) / g->tok_tile, atoms_all = c.hidden / kBlockK;
+    // K split over a cluster where the tiles alone would leave most SMs idle
+    g->ksplit = 1;
+    if (g->reg && g->tok_tile == 32 && ksplit_enabled()) {
+        if (tiles * 8 <= p->sm_count && atoms_all >= 8) g->ksplit = 8;
+        else if (tiles * 4 <= p->sm_count && atoms_all >= 4) g->ksplit = 4;
+    }
+    const size_t part_bytes = g->ksplit > 1 ? (size_t)g->ksplit * n_mma * 32 * 4 : 0;
+    const size_t fixed = kTileRows * kBlockK * 2 + 8 * (2 * kMaxStages + 1) + 8 + (g->pi_in_smem ? pi_bytes : 0);   // slack, barriers, map
+    const size_t tail = 1024 /*alignment*/ + fixed + 16 + part_bytes + 64;
     const size_t pbuf_bytes = g->reg ? 0 : (size_t)M * kTileRows * 4;
     for (int atoms = kMaxAtoms; atoms >= 1; atoms >>= 1) {      // as many K-atoms per stage as leave a ring of >= 3 (else 2) stages
         const int stage_bytes = atoms * (g->tok_tile * kBlockK * 2 + ((n_mma * kBlockK * 2 + 1023) & ~1023));
         int stages = (int)((227 * 1024 - tail) / stage_bytes);
         if (stages > kMaxStages) stages = kMaxStages;
-        const bool fits = (size_t)stages * stage_bytes + kTileRows * kBlockK * 2 >= pbuf_bytes;
-        if ((stages >= 3 || (atoms == 1 && stages >= 2)) && fits) {
+        if (g->ksplit > 1) {                                        // a CTA only has atoms_all / ksplit atoms to load
+            const int need = ((atoms_all + g->ksplit - 1) / g->ksplit + atoms - 1) / atoms;
+            if (stages > (need < 2 ? 2 : need)) stages = need < 2 ? 2 : need;
+        }
+        const bool fits = (size_t)stages * stage_bytes + kTileRows * kBlockK * 2 >= pbuf_bytes &&
+                          (size_t)stages * stage_bytes >= (size_t)(64 * 32 + 3 * 2 * 4 * 32) * 4;   // the epilogue's scratch aliases the ring
+        if ((stages >= 3 || ((atoms == 1 || g->ksplit > 1) && stages >= 2)) && fits) {
             g->atoms = atoms;
             g->stages = stages;
+            g->part_off = (int)(((size_t)stages * stage_bytes + fixed + 15) & ~(size_t)15);
             g->smem = (size_t)stages * stage_bytes + tail;
             g->tmem_cols = n_mma <= 32 ? 32 : n_mma <= 64 ? 64 : n_mma <= 128 ? 128 : 256;
-            g->grid = (B + g->tok_tile - 1) / g->tok_tile;
+            g->grid = tiles * g->ksplit;
             return true;
         }
     }
@@ -444,13 +512,30 @@ static int router_launch(ew_pool *p, int layer, const void *x, const RouterGeome
     A.H = c.hidden; A.M = c.num_experts; A.k = c.top_k; A.N = c.max_adapters; A.renormalize = c.renormalize;
     A.scale = c.routed_scale;
     A.stages = g.stages; A.tmem_cols = g.tmem_cols; A.pi_in_smem = g.pi_in_smem; A.tok_tile = g.tok_tile; A.atoms = g.atoms;
-    if (pdl) {
-        if (g.reg) return launch_pdl(router_kernel<true>, dim3(g.grid), dim3(kThreads), g.smem, st, map_x, map_r, A);
-        return launch_pdl(router_kernel<false>, dim3(g.grid), dim3(kThreads), g.smem, st, map_x, map_r, A);
+    A.ksplit = g.ksplit; A.part_off = g.part_off;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(g.grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = g.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    if (g.ksplit > 1) {
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = g.ksplit;
+        attr[n_attr].val.clusterDim.y = 1;
+        attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
     }
-    if (g.reg) router_kernel<true><<<g.grid, kThreads, g.smem, st>>>(map_x, map_r, A);
-    else router_kernel<false><<<g.grid, kThreads, g.smem, st>>>(map_x, map_r, A);
-    return (int)cudaGetLastError();
+    if (pdl && pdl_enabled()) {
+        attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+        ++n_attr;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n_attr;
+    if (g.reg) return (int)cudaLaunchKernelEx(&cfg, router_kernel<true>, map_x, map_r, A);
+    return (int)cudaLaunchKernelEx(&cfg, router_kernel<false>, map_x, map_r, A);
 }
 
 }  // namespace

@@ -162,10 +162,10 @@ def test_slot_address_reads_back_the_loaded_weights():
     pool.destroy()
 
 
-@pytest.mark.parametrize("switch", ["EW_DISABLE_PDL", "EW_DISABLE_FAT"])
+@pytest.mark.parametrize("switch", ["EW_DISABLE_PDL", "EW_DISABLE_FAT", "EW_DISABLE_KSPLIT"])
 def test_debugging_switches_in_a_fresh_process(switch):
-    """The two environment switches of the library (plain stream order instead of overlapped launches; every block
-    on the weight-streaming kernel) are read once per process, so each is exercised in a process of its own: the
+    """The environment switches of the library (plain stream order instead of overlapped launches; every block on
+    the weight-streaming kernel; no K split in the router) are read once per process, so each is exercised in a process of its own: the
     tiny layer, the decode layer and a prefill-sized odd shape against the oracle."""
     import os
     import subprocess
@@ -173,7 +173,7 @@ def test_debugging_switches_in_a_fresh_process(switch):
     env = dict(os.environ, **{switch: "1"})
     here = os.path.dirname(os.path.abspath(__file__))
     r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-x", "-m", "gpu", os.path.join(here, "test_gpu_parity.py"), "-k",
-                        "test_c0_tiny_layer or test_c1_decode_layer or (test_odd_shapes and shape8)"],
+                        "test_c0_tiny_layer or test_c1_decode_layer or (test_odd_shapes and shape10)"],
                        env=env, capture_output=True, text=True, timeout=900)
     assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
     assert " passed" in r.stdout and "4 passed" in r.stdout, r.stdout[-500:]
@@ -609,6 +609,8 @@ def test_adapter_churn_under_load():
     dict(hidden=64, inter=64, num_experts=256, num_shared=0, top_k=2, max_adapters=20, e_max=1, n_tokens=70),  # expert map too large for shared memory
     dict(hidden=64, inter=64, num_experts=64, num_shared=1, top_k=32, max_adapters=2, e_max=4, n_tokens=50),    # the largest k
     dict(hidden=64, inter=64, num_experts=64, num_shared=1, top_k=32, max_adapters=2, e_max=4, n_tokens=600),   # and with prefill tiles
+    dict(hidden=320, inter=96, num_experts=12, num_shared=1, top_k=3, max_adapters=2, e_max=2, n_tokens=40),   # router K split over 4 CTAs, 5 K-atoms: one CTA has none
+    dict(hidden=576, inter=64, num_experts=24, num_shared=0, top_k=4, max_adapters=2, e_max=3, n_tokens=90),   # router K split over 8 CTAs, 9 K-atoms: ragged shares
     # prefill-sized batches (128-row gather tiles in GEMM-1, 256-row CTA-pair tiles in GEMM-2) on shapes off the tile sizes
     dict(hidden=128, inter=200, num_experts=8, num_shared=1, top_k=2, max_adapters=3, e_max=3, n_tokens=3001),  # H = one weight tile: half-empty tile pair
     dict(hidden=192, inter=72, num_experts=4, num_shared=0, top_k=4, max_adapters=2, e_max=4, n_tokens=1500),   # k = M, I < one tile

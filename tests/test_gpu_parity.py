@@ -615,6 +615,7 @@ def test_adapter_churn_under_load():
     dict(hidden=128, inter=200, num_experts=8, num_shared=1, top_k=2, max_adapters=3, e_max=3, n_tokens=3001),  # H = one weight tile: half-empty tile pair
     dict(hidden=192, inter=72, num_experts=4, num_shared=0, top_k=4, max_adapters=2, e_max=4, n_tokens=1500),   # k = M, I < one tile
     dict(hidden=320, inter=264, num_experts=80, num_shared=2, top_k=3, max_adapters=4, e_max=5, n_tokens=5000), # M > 64 with 64-token router tiles
+    dict(hidden=64, inter=64, num_experts=8, num_shared=1, top_k=2, max_adapters=2, e_max=2, n_tokens=12000),   # 128-token router tiles, 47 fat blocks per shared expert
 ])
 @pytest.mark.parametrize("renorm", [0, 1])
 def test_odd_shapes(shape, renorm):

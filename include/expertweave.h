@@ -85,6 +85,10 @@ typedef struct {
     uint64_t live_experts;        /* routed base + adapter experts currently loaded, over all layers */
     uint64_t adapters_loaded;
     uint64_t workspace_bytes;
+    uint64_t last_forward_kernels; /* kernels the most recent forward launched: 4 (decode-sized batch: router, GEMM-1,
+                                      GEMM-2, combine; the GEMM kernels derive their work items themselves), 5 (the
+                                      same with the planning kernel) or 7 (prefill-sized batch: planning kernel and
+                                      two kernels per GEMM); 0 before the first forward                        */
 } ew_stats_t;
 
 /* Create a pool: reserves, per layer and per stacked linear (gate|up fused as one tensor, down as
@@ -138,7 +142,7 @@ ew_status_t ew_pool_trim(ew_pool_t *pool);
 /* The adapter-aware MoE layer forward (Sections 2.1, 4.1, 4.3), asynchronous on `cuda_stream`:
  *   softmax router + top-k over the M base experts (ties to the lower index)
  *   -> batched rerouting  slot = adapter_ids[t] < 0 ? id : Pi[layer][adapter_ids[t]][id]
- *   -> per-slot token counts, permutation into slot-contiguous rows
+ *   -> per-slot token counts, permutation into slot-contiguous rows (as index tables: no copy of x is made)
  *   -> grouped SwiGLU FFN over the live slots and the shared experts (fp32 accumulation)
  *   -> out[t] = sum_j w[t,j] * FFN_slot(t,j)(x[t]) + sum_shared FFN(x[t]), rounded once to bf16.
  *   x            device bf16 [n_tokens, H], 16-byte aligned
@@ -183,10 +187,12 @@ ew_status_t ew_moe_forward_host(ew_pool_t *pool, int32_t layer, const void *x_ho
                                 const int32_t *adapter_ids_host, int32_t n_tokens, void *out_host,
                                 void *cuda_stream);
 
-/* Per-kernel timing.  While enabled, every forward records CUDA events on its stream around its five
+/* Per-kernel timing.  While enabled, every forward records CUDA events on its stream around its
  * kernels (no host synchronisation).  ew_profile_read waits for the recorded forwards, adds up the
  * elapsed milliseconds per kernel into ms[5] = {route (incl. zeroing the counts), permute+plan,
  * GEMM-1+SwiGLU, GEMM-2, combine}, writes how many forwards were measured, and clears the record.
+ * A decode-sized forward has no planning kernel (ew_stats_t.last_forward_kernels = 4): its ms[1] is the
+ * cost of the two event records alone, and the GEMM kernels' times include the derivation of their work items.
  * At most 4096 forwards are recorded between two reads. */
 ew_status_t ew_profile_enable(ew_pool_t *pool, int32_t on);
 ew_status_t ew_profile_read(ew_pool_t *pool, double *ms, int32_t *n_forwards);

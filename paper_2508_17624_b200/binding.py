@@ -39,7 +39,7 @@ class EwStats(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in
                 ("page_bytes", "va_reserved_bytes", "pages_mapped", "pages_free", "pages_created_total",
                  "physical_bytes", "live_expert_bytes", "padding_bytes", "live_experts", "adapters_loaded",
-                 "workspace_bytes")]
+                 "workspace_bytes", "last_forward_kernels")]
 
     def as_dict(self):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}

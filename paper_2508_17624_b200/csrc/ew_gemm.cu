@@ -34,6 +34,7 @@
 #include <cuda_bf16.h>
 
 #include "ew_internal.h"
+#include "ew_plan.cuh"
 #include "ew_tc.cuh"
 
 namespace ew {
@@ -56,7 +57,11 @@ struct Cfg {
     static constexpr int kTmemColsRaw = kAccCols * kAccStages;
     static constexpr int kTmemCols = kTmemColsRaw <= 32 ? 32 : kTmemColsRaw <= 64 ? 64 : kTmemColsRaw <= 128 ? 128
                                      : kTmemColsRaw <= 256 ? 256 : 512;
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int kRingBytes = kStages * kStageBytes;
+    // self-planned forwards: the CTA's own items, 16 bytes each, behind the barriers (as many as the CTA's shared memory leaves)
+    static constexpr int kSelfCapRaw = (227 * 1024 - kRingBytes - 1024 - 256) / 16;
+    static constexpr int kSelfCap = kSelfCapRaw > 256 ? 256 : kSelfCapRaw;
+    static constexpr int kSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kSelfCap * 16;
 };
 
 // ------------------------------------------------------------------------------------------- kernel
@@ -78,7 +83,7 @@ __global__ void __launch_bounds__(GLU ? kThreads + kGatherThreads : kThreads, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
                     const __grid_constant__ CUtensorMap map_a_big, const GemmItem *items,
                     const int32_t *n_items_ptr, int K, int out_rows_per_slot, void *out,
-                    int *err, const uint8_t *x_rows, const int32_t *src_tok, int n_x_rows) {
+                    int *err, const uint8_t *x_rows, const int32_t *src_tok, int n_x_rows, const plan::SelfPlan sp) {
     // GEMM-1 gathers its token rows from x (shared experts: TMA boxes of x through map_a / map_a_big);
     // GEMM-2 reads the activation rows GEMM-1 wrote through map_a / map_a_big
     constexpr bool GATHER = GLU;
@@ -93,6 +98,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
     const uint32_t bar_tfull = bar_empty + 8 * C::kStages, bar_tempty = bar_tfull + 16;
     uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(bars + 2 * C::kStages + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
+    int4 *self_items = reinterpret_cast<int4 *>(smem_al + C::kRingBytes + 256);     // [kSelfCap]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = (K + kBlockK - 1) / kBlockK;
@@ -117,7 +123,14 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    pdl_launch_dependents();
+    // Self-planned forwards (no planning kernel ran): this CTA's items are derived from the router's counts, with the
+    // ring - not yet in use - as scratch.  GEMM-1 does that after its wait for the router kernel (and rehearses it
+    // before, see derive_items) and only then releases GEMM-2; GEMM-2 therefore starts with the counts final and plans
+    // while it waits for GEMM-1's last CTAs.
+    const bool self = sp.counts != nullptr;
+    constexpr int kScanWarp = 2;
+    int n_mine = 0;
+    if (!self) pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -125,16 +138,40 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
     // The item list and the activations come from the previous kernels: nothing of them may be read before this
     // wait.  (The pointers are deliberately not __restrict__/const-qualified read-only data: the compiler may
     // hoist such loads above the wait.)
-    pdl_wait();
-    const int n_items = *reinterpret_cast<const volatile int32_t *>(n_items_ptr);
+    if (self) {
+        // one call site, executed twice by GEMM-1 (rehearsal before the wait, then for real) and once by GEMM-2
+        // (for real, before the wait)
+#pragma unroll 1
+        for (int rep = (GLU && sp.rehearse) ? 0 : 1; rep < 2; ++rep) {
+            if (GLU && rep == 1) {
+                pdl_wait();
+                pdl_launch_dependents();
+            }
+            n_mine = plan::derive_items(reinterpret_cast<int32_t *>(smem_al), sp, (int)blockDim.x, kScanWarp, self_items, C::kSelfCap,
+                                        GLU && rep == 0);
+        }
+        if (!GLU) {
+            pdl_wait();
+        }
+    } else {
+        // every gridDim.x-th item of the planning kernel's list
+        pdl_wait();
+        const int n_items = *reinterpret_cast<const volatile int32_t *>(n_items_ptr);
+        n_mine = n_items > (int)blockIdx.x ? (n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    }
+    // this CTA's j-th item
+    auto item_at = [&](int j) -> GemmItem {
+        if (self) return plan::unpack_item(self_items[j], sp.B);
+        return items[blockIdx.x + (size_t)j * gridDim.x];
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
-                const GemmItem it = items[w];
+            for (int w = 0; w < n_mine && ok; ++w) {
+                const GemmItem it = item_at(w);
                 const int nchunk = (it.rows + kChunkRows - 1) / kChunkRows;
                 // thin items fetch their rows in 32-row boxes; fat ones (prefill) with one NT-row box per stage
                 const bool big = NT >= 128 && it.rows > 2 * kChunkRows;
@@ -176,8 +213,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
         if (lane == 0) {
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
-            for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
-                const GemmItem it = items[w];
+            for (int w = 0; w < n_mine && ok; ++w) {
+                const GemmItem it = item_at(w);
                 const int n = ((it.rows + 15) >> 4) << 4;
                 const uint32_t idesc = instr_desc(n);
                 if (!(ok = mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1, abort_flag, err))) break;
@@ -225,8 +262,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
         }
         uint32_t stage = 0, phase = 0;
         bool ok = true;
-        for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
-            const GemmItem it = items[w];
+        for (int w = 0; w < n_mine && ok; ++w) {
+            const GemmItem it = item_at(w);
             const int n = ((it.rows + 15) >> 4) << 4;
             const uint8_t *src[kRowsPerThread];                  // rows beyond n are not read by the MMA: not fetched
 #pragma unroll
@@ -256,8 +293,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
         const int row = lg * 32 + lane;                 // row inside the 128-row weight tile
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
-        for (int w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
-            const GemmItem it = items[w];
+        for (int w = 0; w < n_mine && ok; ++w) {
+            const GemmItem it = item_at(w);
             if (!(ok = mbar_wait_warp(bar_tfull + 8 * acc, acc_phase, abort_flag, err))) break;
             tc_fence_after();
             const uint32_t t0 = tmem_base + ((uint32_t)(lg * 32) << 16) + acc * C::kAccCols;
@@ -636,11 +673,36 @@ int launch_fat(ew_pool *p, const CUtensorMap &mw, const CUtensorMap &ma, const G
 
 template <int NT, bool GLU>
 int launch_one(ew_pool *p, const CUtensorMap &mw, const CUtensorMap &ma, const CUtensorMap &mab, const GemmItem *items,
-               const int32_t *n_items, int K, int out_rows, void *out, cudaStream_t st, const void *x_rows, int n_x_rows) {
+               const int32_t *n_items, int K, int out_rows, void *out, cudaStream_t st, const void *x_rows, int n_x_rows,
+               const plan::SelfPlan &sp) {
     using C = Cfg<NT, GLU>;
+    // self-planned forwards read the router's slot-major token table instead of the planning kernel's row -> token table
+    const int32_t *tok_table = sp.counts ? p->ws.slot_tok : p->ws.src_tok;
     return launch_pdl(grouped_gemm_kernel<NT, GLU>, dim3(p->sm_count), dim3(GLU ? kThreads + kGatherThreads : kThreads),
                       C::kSmemBytes, st, mw, ma, mab, items, n_items, K, out_rows, out, p->ws.err, (const uint8_t *)x_rows,
-                      (const int32_t *)p->ws.src_tok, n_x_rows);
+                      tok_table, n_x_rows, sp);
+}
+
+template <int NT, bool GLU>
+void self_limits(int *cap, size_t *scratch_bytes) {
+    *cap = Cfg<NT, GLU>::kSelfCap;
+    *scratch_bytes = Cfg<NT, GLU>::kRingBytes;
+}
+
+plan::SelfPlan self_plan_args(const ew_pool *p, int B, int pass) {
+    plan::SelfPlan sp = {};
+    if (!p->self_plan) return sp;
+    const ew_config_t &c = p->cfg;
+    sp.counts = p->ws.counts;
+    sp.B = B; sp.k = c.top_k; sp.P = p->P; sp.S = c.num_shared;
+    sp.nt_shift = p->token_tile == 32 ? 5 : p->token_tile == 64 ? 6 : 7;
+    sp.R = ((pass ? c.hidden : c.inter) + 127) / 128;
+    sp.pass = pass;
+    // per-kernel profiling puts events between the kernels: nothing runs beside the router kernel then, and a
+    // rehearsal would only be added to GEMM-1's measured time
+    sp.rehearse = p->profiling_this_forward ? 0 : 1;
+    if (!pass) { sp.slot_ids = p->ws.slot_ids; sp.rank = p->ws.rank; sp.offsets = p->ws.offsets; sp.inv = p->ws.inv; }
+    return sp;
 }
 
 template <int NT, bool GLU>
@@ -650,6 +712,27 @@ int setup_one() {
 }
 
 }  // namespace
+
+// Whether a forward of B tokens with NT-row items can run without the planning kernel: every CTA of the GEMM kernels
+// must be able to hold its own items (whatever the routing turns out to be) and the planning scratch in shared memory.
+bool self_plan_fits(const ew_pool *p, int B, int NT) {
+    const ew_config_t &c = p->cfg;
+    int cap1, cap2;
+    size_t scr1, scr2;
+    switch (NT) {
+        case 32: self_limits<32, true>(&cap1, &scr1); self_limits<32, false>(&cap2, &scr2); break;
+        case 64: self_limits<64, true>(&cap1, &scr1); self_limits<64, false>(&cap2, &scr2); break;
+        default: self_limits<128, true>(&cap1, &scr1); self_limits<128, false>(&cap2, &scr2); break;
+    }
+    const size_t need = plan::self_plan_words(p->P, c.num_shared) * 4;
+    if (need > scr1 || need > scr2 || p->P + c.num_shared > plan::kSelfMaxGroups) return false;
+    // token blocks of any routing: at most floor(B k / NT) full ones plus one ragged block per live slot, plus the shared experts'
+    const long long pairs = (long long)B * c.top_k;
+    const long long blocks = pairs / NT + (pairs < p->P ? pairs : p->P) + (long long)c.num_shared * ((B + NT - 1) / NT);
+    const long long R1 = (c.inter + 127) / 128, R2 = (c.hidden + 127) / 128;
+    const long long per1 = (blocks * R1 + p->sm_count - 1) / p->sm_count, per2 = (blocks * R2 + p->sm_count - 1) / p->sm_count;
+    return per1 <= cap1 && per2 <= cap2 && R1 < 65536 && R2 < 65536;
+}
 
 int gemm_setup(ew_pool *) {
     int rc = 0;
@@ -668,26 +751,28 @@ int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, const CUtensor
     const LayerState &L = p->layers[layer];
     const int K = p->cfg.hidden, I = p->cfg.inter;
     const Workspace &w = p->ws;
+    const plan::SelfPlan sp = self_plan_args(p, B, 0);
     int rc;
     switch (p->token_tile) {
-        case 32: rc = launch_one<32, true>(p, L.map_w13, map_x, map_x, w.items1, w.n_items, K, I, w.act, st, x, B); break;
-        case 64: rc = launch_one<64, true>(p, L.map_w13, map_x, map_x, w.items1, w.n_items, K, I, w.act, st, x, B); break;
-        default: rc = launch_one<128, true>(p, L.map_w13, map_x, map_x_big, w.items1, w.n_items, K, I, w.act, st, x, B); break;
+        case 32: rc = launch_one<32, true>(p, L.map_w13, map_x, map_x, w.items1, w.n_items, K, I, w.act, st, x, B, sp); break;
+        case 64: rc = launch_one<64, true>(p, L.map_w13, map_x, map_x, w.items1, w.n_items, K, I, w.act, st, x, B, sp); break;
+        default: rc = launch_one<128, true>(p, L.map_w13, map_x, map_x_big, w.items1, w.n_items, K, I, w.act, st, x, B, sp); break;
     }
     if (rc || !p->fat) return rc;
     return launch_fat<true>(p, L.map_w13, map_x_big, w.fat1, w.n_items + 2, K, I, w.act, st, x, B);
 }
 
-int launch_gemm2(ew_pool *p, int layer, int, cudaStream_t st) {
+int launch_gemm2(ew_pool *p, int layer, int B, cudaStream_t st) {
     const LayerState &L = p->layers[layer];
     const int K = p->cfg.inter, H = p->cfg.hidden;
     const Workspace &w = p->ws;
     const CUtensorMap &a = p->map_act, &ab = p->map_act_big;
+    const plan::SelfPlan sp = self_plan_args(p, B, 1);
     int rc;
     switch (p->token_tile) {
-        case 32: rc = launch_one<32, false>(p, L.map_w2, a, a, w.items2, w.n_items + 1, K, H, w.y, st, nullptr, 0); break;
-        case 64: rc = launch_one<64, false>(p, L.map_w2, a, a, w.items2, w.n_items + 1, K, H, w.y, st, nullptr, 0); break;
-        default: rc = launch_one<128, false>(p, L.map_w2, a, ab, w.items2, w.n_items + 1, K, H, w.y, st, nullptr, 0); break;
+        case 32: rc = launch_one<32, false>(p, L.map_w2, a, a, w.items2, w.n_items + 1, K, H, w.y, st, nullptr, 0, sp); break;
+        case 64: rc = launch_one<64, false>(p, L.map_w2, a, a, w.items2, w.n_items + 1, K, H, w.y, st, nullptr, 0, sp); break;
+        default: rc = launch_one<128, false>(p, L.map_w2, a, ab, w.items2, w.n_items + 1, K, H, w.y, st, nullptr, 0, sp); break;
     }
     if (rc || !p->fat) return rc;
     return launch_fat<false>(p, L.map_w2, ab, w.fat2, w.n_items + 3, K, H, w.y, st, nullptr, 0);

@@ -39,6 +39,7 @@ struct Workspace {
     GemmItem *items1 = nullptr, *items2 = nullptr;   // thin items
     GemmItem *fat1 = nullptr, *fat2 = nullptr;       // fat items (prefill-sized batches)
     int32_t *src_tok = nullptr;    // [Bmax*k] token of each slot-contiguous row: GEMM-1 fetches those rows of x itself
+    int32_t *slot_tok = nullptr;   // [P, B] self-planned forwards: the tokens of each slot in rank order, written by the router kernel
     void *act = nullptr;           // [S*Bmax + Bmax*k, I] bf16 SwiGLU output
     float *y = nullptr;            // [S*Bmax + Bmax*k, H] fp32 expert outputs
     int32_t *err = nullptr;        // device error word
@@ -65,6 +66,8 @@ struct ew_pool {
     int P = 0;                      // M + N * E_max
     int token_tile = 32;            // NT: token rows per thin work item (32, 64 or 128)
     bool fat = false;               // prefill-sized batch: blocks of more than 128 rows run on the CTA-pair kernel
+    int last_forward_kernels = 0;   // kernels launched by the most recent forward (reported by ew_pool_stats)
+    bool self_plan = false;         // decode-sized batch: no planning kernel, the GEMM kernels derive their items from the counts
     ew::PageBackend *be = nullptr;
     ew::PagePool pages;
     std::vector<ew::LayerState> layers;
@@ -78,6 +81,7 @@ struct ew_pool {
     cudaEvent_t route_event = nullptr;   // last ew_route_noalloc call (created with the pool: that call creates nothing)
     bool route_event_used = false;
     bool profiling = false;
+    bool profiling_this_forward = false;    // the forward being launched records events between its kernels
     std::vector<cudaEvent_t> prof_events;   // 6 per recorded forward
     size_t prof_used = 0;                   // events in use
     // ew_moe_forward_host: double-buffered device staging and three internal streams, so that the upload of call
@@ -117,6 +121,8 @@ struct DeviceGuard {
 bool pdl_enabled();
 // EW_DISABLE_FAT=1 keeps every block of token rows on the weight-streaming kernel (128-row blocks at prefill).
 bool fat_enabled();
+// EW_DISABLE_SELFPLAN=1 runs the planning kernel for every batch size.
+bool self_plan_enabled();
 
 // Launch with programmatic stream serialization (the kernel calls pdl_wait() before it reads its
 // predecessor's output).
@@ -155,6 +161,7 @@ int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid
                    int32_t *counts, cudaStream_t st);
 int launch_route_logits(ew_pool *p, int layer, const float *logits, const int32_t *aid, int B, int32_t *topk_ids,
                         float *topk_w, int32_t *slot_ids, int32_t *counts, cudaStream_t st);
+bool self_plan_fits(const ew_pool *p, int B, int NT);   // a forward of B tokens with NT-row items can skip the planning kernel
 int gemm_setup(ew_pool *p);   // once per pool: opt in to the shared memory the GEMM kernels need
 int router_setup(ew_pool *p); // once per pool: the router kernels' attributes and the fixed scratch array's device address
 

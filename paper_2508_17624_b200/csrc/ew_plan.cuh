@@ -3,7 +3,11 @@
 // tables (inv: pair -> row, src_tok: row -> token), and the work-item lists of the grouped GEMM kernels.
 //
 // All functions are block-wide: every thread of the CTA calls them with the same arguments; `nthreads` =
-// blockDim.x must be a multiple of 32 and at most 256.
+// blockDim.x must be a multiple of 32 and at most 256 (derive_items: any multiple of 32).
+//
+// Decode-sized batches skip the planning kernel altogether ("self-planned" forwards): the router records each
+// slot's tokens in a slot-major table, and every CTA of the GEMM kernels repeats the scan of the counts and derives
+// its own items of the list that write_items would have written (derive_items).
 #pragma once
 #include "ew_internal.h"
 
@@ -144,6 +148,143 @@ __device__ inline void write_items(int32_t *sm, const int32_t *cnt_s, const Para
             }
         }
     }
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Self-planned forwards (decode-sized batches: thin items only).
+struct SelfPlan {
+    const int32_t *counts;       // [P] per-slot pair counts of the router kernel; null: walk the planner's item list
+    int B, k, P, S;
+    int nt_shift;                // token rows per item NT = 1 << nt_shift (32, 64 or 128)
+    int R;                       // weight tiles per group of this GEMM
+    int pass;                    // 0: GEMM-1 (+ SwiGLU), 1: GEMM-2
+    int rehearse;                // GEMM-1: run the planning code once before the wait for the router kernel (see derive_items)
+    // GEMM-1 only: its CTAs also publish what the combine step (and the debugging outputs) need
+    const int32_t *slot_ids, *rank;      // [B*k] from the router kernel
+    int32_t *offsets, *inv;              // out: [P + 1] exclusive scan of the counts, [B*k] pair -> slot-contiguous row
+};
+
+constexpr int kSelfMaxGroups = 1024;     // P + S of a self-planned forward: one warp scans them
+
+// One derived item, packed: x = slot | tile << 16, y = first input row, z = first output row,
+// w = rows | from_x << 8 | chain << 16.
+__device__ inline GemmItem unpack_item(const int4 v, int chain_rows) {
+    GemmItem it;
+    it.slot = v.x & 0xffff; it.tile = (int)((uint32_t)v.x >> 16);
+    it.in_row = v.y; it.out_row = v.z;
+    it.rows = v.w & 0xff; it.from_x = (v.w >> 8) & 1; it.chain = (int)((uint32_t)v.w >> 16);
+    it.chain_rows = chain_rows;
+    return it;
+}
+
+// Shared-memory words derive_items needs as scratch (may alias memory that is only used after the call):
+// offsets [P + 1], block scan [G + 1], clamped counts [P].
+__host__ __device__ constexpr size_t self_plan_words(int P, int S) { return (size_t)(P + 1) + (size_t)(P + S + 1) + (size_t)P; }
+
+// Items blockIdx.x, blockIdx.x + gridDim.x, ... of the thin list of pass A.pass, in list order, packed into
+// mine[0 .. n) (n is returned; the host has checked that n <= cap for every possible routing).  The list is the one
+// write_items builds with fat = 0: groups in order (shared experts, then slots), per group (weight tile, token block);
+// in GEMM-2 the shared experts form one group chained along K.  One difference: a routed GEMM-1 item's in_row indexes
+// the router's slot-major token table ([P][B]: slot * B + first row of the block) instead of the row -> token table of
+// the planning kernel.  With A.inv set (GEMM-1) the CTAs also write offsets and inv.
+//
+// The code runs once per CTA and launch, in GEMM-1 on the critical path between the router kernel's end and the first
+// weight load, so it is written for latency and kept small (its instructions are cold, see below): all threads stage
+// the counters in shared memory; warp `scan_warp` scans counts and token blocks with shuffles; then one thread per item
+// finds its group by binary search while the other threads write inv.  Three barriers in all.
+//
+// `dry`: a rehearsal that writes nothing to global memory and tolerates any values in the counters.  The instructions
+// are cold when a CTA gets here (every forward streams the live weights through L2 and evicts them; cold, an earlier
+// form of this function took 3.5 us in GEMM-1 and 6.8 us in GEMM-2 of the decode layer against ~1 us to read a
+// prepared list), so GEMM-1 rehearses it while it waits for the router kernel.
+// (The rehearsal and the real call must execute the same instructions: the caller makes both from one call site in a
+// loop that is not unrolled.  The function is inlined there so that the kernel's parameters stay in constant memory;
+// as a separate function it received them through the stack, which cost several dependent L2 round trips.)
+__device__ __forceinline__ int derive_items(int32_t *sm, const SelfPlan &A, int nthreads, int scan_warp, int4 *mine, int cap,
+                                                bool dry) {
+    const int P = A.P, S = A.S, B = A.B, G = P + S;
+    int32_t *off = sm;                       // [P + 1] exclusive scan of the counts
+    int32_t *eblk = sm + P + 1;              // [G + 1] exclusive scan of the groups' token blocks in this pass
+    int32_t *cnt_s = eblk + G + 1;           // [P] the counts (clamped to [0, B]: a rehearsal may see anything)
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long n_pairs = (long long)B * A.k;
+    // this thread's first pair (GEMM-1): the loads go out together with the loads of the counts
+    const long long q0 = (long long)blockIdx.x * nthreads + threadIdx.x;
+    int my_slot = 0, my_rank = 0;
+    if (A.inv && q0 < n_pairs) { my_slot = __ldcg(A.slot_ids + q0); my_rank = __ldcg(A.rank + q0); }
+    // all threads: the counts, clamped to [0, B] (a rehearsal may see anything), into shared memory
+    for (int i = threadIdx.x; i < P; i += nthreads) cnt_s[i] = min(max(__ldcg(A.counts + i), 0), B);
+    __syncthreads();
+    if (warp == scan_warp) {
+        const int per = (G + 31) >> 5, g0 = lane * per, g1 = min(g0 + per, G);       // lane owns groups [g0, g1)
+        const int round_up = (1 << A.nt_shift) - 1;
+        int csum = 0, bsum = 0;
+#pragma unroll 4
+        for (int g = g0; g < g1; ++g) {
+            const int rows = g < S ? B : cnt_s[g - S];
+            if (g >= S) csum += rows;
+            // GEMM-2: the shared experts 1 .. S-1 ride in group 0's items
+            if (!(A.pass && g > 0 && g < S)) bsum += (rows + round_up) >> A.nt_shift;
+        }
+        int cinc = csum, binc = bsum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int c = __shfl_up_sync(0xffffffffu, cinc, o), b = __shfl_up_sync(0xffffffffu, binc, o);
+            if (lane >= o) { cinc += c; binc += b; }
+        }
+        int crun = cinc - csum, brun = binc - bsum;
+#pragma unroll 4
+        for (int g = g0; g < g1; ++g) {
+            const int rows = g < S ? B : cnt_s[g - S];
+            eblk[g] = brun;
+            if (!(A.pass && g > 0 && g < S)) brun += (rows + round_up) >> A.nt_shift;
+            if (g >= S) { off[g - S] = crun; crun += rows; }
+        }
+        if (lane == 31) { off[P] = cinc; eblk[G] = binc; }
+    }
+    __syncthreads();
+    const int total = eblk[G] * A.R;
+    const int y_base = S > 0 ? B : 0;
+    int n_mine = total > (int)blockIdx.x ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    n_mine = min(n_mine, cap);
+    // one thread per item, taken from the top of the CTA so that they are not the threads that write inv first
+    const int j = nthreads - 1 - (int)threadIdx.x;
+    for (int jj = j; jj < n_mine; jj += nthreads) {
+        const int i = (int)blockIdx.x + jj * (int)gridDim.x;
+        const int b = i / A.R;                                   // block coordinate: eblk[g] <= b < eblk[g + 1]
+        int lo = 0, hi = G;                                      // invariant: eblk[lo] <= b < eblk[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (eblk[mid] <= b) lo = mid; else hi = mid;
+        }
+        const int g = lo;
+        const bool shared = g < S;
+        const int rows = shared ? B : cnt_s[g - S];
+        const int nt = max(eblk[g + 1] - eblk[g], 1);
+        const int local = i - eblk[g] * A.R;
+        int tile = local, c = 0;
+        if (nt > 1) { tile = local / nt; c = local - tile * nt; }
+        const int r0 = c << A.nt_shift;
+        const int slot = shared ? P + g : g - S;
+        const int act0 = shared ? g * B : S * B + off[shared ? 0 : g - S];
+        const int in0 = shared ? 0 : (g - S) * B;                // routed rows: index into the slot-major token table
+        const int y0 = shared ? 0 : y_base + off[shared ? 0 : g - S];
+        const int in_base = A.pass ? act0 : in0, out_base = A.pass ? y0 : act0;
+        const int from_x = (!A.pass && shared) ? 1 : 0, chain = (A.pass && shared) ? S : 1;
+        mine[jj] = make_int4(slot | (tile << 16), in_base + r0, out_base + r0,
+                             min(1 << A.nt_shift, rows - r0) | (from_x << 8) | (chain << 16));
+    }
+    if (A.inv) {
+        if (blockIdx.x == 0 && !dry)
+            for (int i = threadIdx.x; i <= P; i += nthreads) A.offsets[i] = off[i];
+        for (long long q = q0; q < n_pairs; q += (long long)gridDim.x * nthreads) {
+            if (q != q0) { my_slot = __ldcg(A.slot_ids + q); my_rank = __ldcg(A.rank + q); }
+            const int dest = off[min(max(my_slot, 0), P - 1)] + my_rank;
+            if (dest >= 0 && dest < n_pairs && !dry) A.inv[q] = dest;    // always, unless the routing kernel gave up midway
+        }
+    }
+    __syncthreads();
+    return n_mine;
 }
 
 }  // namespace plan

@@ -14,6 +14,10 @@ bool fat_enabled() {
     static const bool on = [] { const char *e = getenv("EW_DISABLE_FAT"); return !(e && e[0] == '1'); }();
     return on;
 }
+bool self_plan_enabled() {
+    static const bool on = [] { const char *e = getenv("EW_DISABLE_SELFPLAN"); return !(e && e[0] == '1'); }();
+    return on;
+}
 bool pdl_enabled() {
     static const bool on = [] { const char *e = getenv("EW_DISABLE_PDL"); return !(e && e[0] == '1'); }();
     return on;
@@ -102,6 +106,8 @@ static ew_status_t alloc_workspace(ew_pool *p) {
     size_t rbf = (P + S) + (S * Bm + Bm * k) / 128 + 1;
     size_t r1 = (I + 127) / 128, r2 = (H + 127) / 128, rf2 = (H + 255) / 256;
     size_t rows = S * Bm + Bm * k + 32;     // +32: a token tile may start at the last row
+    // self-planned forwards (batches below the prefill threshold of pick_token_tile): [P][B] tokens per slot
+    size_t Bs = std::min(Bm, (size_t)128 * c.num_experts / k + 1);
     struct Seg { void **ptr; size_t bytes; };
     Workspace &w = p->ws;
     Seg segs[] = {
@@ -110,6 +116,7 @@ static ew_status_t alloc_workspace(ew_pool *p) {
         {(void **)&w.offsets, (P + 1) * 4}, {(void **)&w.n_items, 16}, {(void **)&w.items1, rb * r1 * sizeof(GemmItem)},
         {(void **)&w.items2, rb * r2 * sizeof(GemmItem)}, {(void **)&w.fat1, rbf * r1 * sizeof(GemmItem)},
         {(void **)&w.fat2, rbf * rf2 * sizeof(GemmItem)}, {(void **)&w.src_tok, (Bm * k + 32) * 4},
+        {(void **)&w.slot_tok, (P * Bs + 32) * 4},
         {(void **)&w.act, rows * I * 2}, {(void **)&w.y, rows * H * 4}, {(void **)&w.err, 256},
         {(void **)&w.loaded, (size_t)c.max_adapters * 4 + 16},
         {&p->stage_x[0], Bm * H * 2}, {&p->stage_out[0], Bm * H * 2}, {(void **)&p->stage_aid[0], Bm * 4},
@@ -482,6 +489,7 @@ extern "C" ew_status_t ew_pool_stats(ew_pool_t *p, ew_stats_t *out) {
     out->live_experts = p->live_experts;
     for (auto &a : p->adapter_counts) out->adapters_loaded += !a.empty();
     out->workspace_bytes = p->ws.bytes;
+    out->last_forward_kernels = p->last_forward_kernels;
     return EW_OK;
 }
 
@@ -586,6 +594,8 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     const int tile = pick_token_tile(p, B);
     p->fat = tile == 256 && fat_enabled();
     p->token_tile = tile == 256 ? 128 : tile;
+    // decode-sized batches run without the planning kernel when every GEMM CTA can hold its own items
+    p->self_plan = !p->fat && tile != 256 && self_plan_enabled() && self_plan_fits(p, B, p->token_tile);
     if (p->token_tile >= 128) {
         uint32_t bbox[2] = {64, 128};
         if (make_tensor_map(p, &map_x_big, x, 2, dx, bbox)) return EW_ERR_CUDA;
@@ -601,6 +611,7 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
         pe = p->prof_events.data() + p->prof_used;
         p->prof_used += 6;
     }
+    p->profiling_this_forward = pe != nullptr;
 #define PROF_MARK(i) do { if (pe) CU_TRY(cudaEventRecord(pe[i], st)); } while (0)
     {
         ew_status_t ordered = order_after_other_streams(p, st);
@@ -611,20 +622,23 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     p->counts_clean = false;
     LAUNCH_TRY(launch_route(p, layer, x, aid, B, st));
     PROF_MARK(1);
-    LAUNCH_TRY(launch_permute(p, B, st));
+    if (!p->self_plan) LAUNCH_TRY(launch_permute(p, B, st));
     PROF_MARK(2);
     if (topk_ids) CU_TRY(cudaMemcpyAsync(topk_ids, p->ws.topk_ids, nk * 4, cudaMemcpyDeviceToDevice, st));
     if (topk_w) CU_TRY(cudaMemcpyAsync(topk_w, p->ws.topk_w, nk * 4, cudaMemcpyDeviceToDevice, st));
     if (slot_ids) CU_TRY(cudaMemcpyAsync(slot_ids, p->ws.slot_ids, nk * 4, cudaMemcpyDeviceToDevice, st));
     if (counts) CU_TRY(cudaMemcpyAsync(counts, p->ws.counts, (size_t)p->P * 4, cudaMemcpyDeviceToDevice, st));
+    // the pair -> row table and the offsets come from the planning kernel, or (self-planned forwards) from GEMM-1's CTAs
+    if (p->self_plan) LAUNCH_TRY(launch_gemm1(p, layer, map_x, map_x_big, x, B, st));
     if (inv) CU_TRY(cudaMemcpyAsync(inv, p->ws.inv, nk * 4, cudaMemcpyDeviceToDevice, st));
     if (offsets) CU_TRY(cudaMemcpyAsync(offsets, p->ws.offsets, ((size_t)p->P + 1) * 4, cudaMemcpyDeviceToDevice, st));
-    LAUNCH_TRY(launch_gemm1(p, layer, map_x, map_x_big, x, B, st));
+    if (!p->self_plan) LAUNCH_TRY(launch_gemm1(p, layer, map_x, map_x_big, x, B, st));
     PROF_MARK(3);
     LAUNCH_TRY(launch_gemm2(p, layer, B, st));
     PROF_MARK(4);
     LAUNCH_TRY(launch_combine(p, B, out, st));
     p->counts_clean = true;                             // the combine kernel zeroes the counters when it is done with them
+    p->last_forward_kernels = p->self_plan ? 4 : p->fat ? 7 : 5;
     PROF_MARK(5);
 #undef PROF_MARK
     return note_forward(p, st);

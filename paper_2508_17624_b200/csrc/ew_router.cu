@@ -65,6 +65,7 @@ struct RouterArgs {
     float *topk_w;
     int32_t *slot_ids, *rank, *counts;
     int *err;
+    int32_t *slot_tok = nullptr;   // [P][B] or null.  Forwards without a planning kernel: the token of the pair at position r of slot s
 };
 
 // write one selected pair: reroute through Pi, outputs (the histogram follows in emit_ranks)
@@ -90,7 +91,11 @@ __device__ __forceinline__ void emit_ranks(const RouterArgs &A, int t, const int
             if (r0 + u < A.k) got[u] = atomicAdd(A.counts + (r0 == 0 ? sl[u] : A.slot_ids[(size_t)t * A.k + r0 + u]), 1);
 #pragma unroll
         for (int u = 0; u < 8; ++u)
-            if (r0 + u < A.k) A.rank[(size_t)t * A.k + r0 + u] = got[u];
+            if (r0 + u < A.k) {
+                A.rank[(size_t)t * A.k + r0 + u] = got[u];
+                if (A.slot_tok && got[u] >= 0 && got[u] < A.B)
+                    A.slot_tok[(size_t)(r0 == 0 ? sl[u] : A.slot_ids[(size_t)t * A.k + r0 + u]) * A.B + got[u]] = t;
+            }
     }
 }
 
@@ -320,6 +325,7 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                         if (A.renormalize) w = w / wsum;
                         A.topk_w[o] = (A.renormalize || A.scale != 1.f) ? w * A.scale : w;
                         A.rank[o] = got[u];
+                        if (A.slot_tok && got[u] >= 0 && got[u] < A.B) A.slot_tok[(size_t)my_slot[u] * A.B + got[u]] = t;
                     }
             }
         }
@@ -547,6 +553,7 @@ int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B
     A.aid = aid; A.B = B;
     A.topk_ids = p->ws.topk_ids; A.topk_w = p->ws.topk_w; A.slot_ids = p->ws.slot_ids; A.rank = p->ws.rank;
     A.counts = p->ws.counts; A.err = p->ws.err;
+    A.slot_tok = p->self_plan ? p->ws.slot_tok : nullptr;
     return router_launch(p, layer, x, g, A, true, st);
 }
 

@@ -373,7 +373,7 @@ def run_extras(sampler, device):
     """The other parts of the metric, one record each, every one with the clocks sampled while it ran."""
     out = {}
     for name, fn in (("c2_prefill", extra_prefill), ("c3_stack_slice", extra_stack), ("c4_reroute", extra_reroute),
-                     ("padding_mode", extra_padding)):
+                     ("padding_mode", extra_padding), ("expert_parallel_emulated", extra_expert_parallel)):
         try:
             sampler.take()
             rec = fn(device, sampler)
@@ -585,6 +585,43 @@ def extra_padding(device, sampler, pairs=7):
             "latency_delta_max": float(np.max(delta)),
             "physical_bytes_on_demand": stats[0]["physical_bytes"], "physical_bytes_padding": stats[1]["physical_bytes"],
             "saved_frac": 1.0 - stats[0]["physical_bytes"] / stats[1]["physical_bytes"]}
+
+
+def extra_expert_parallel(device, sampler):
+    """Expert parallelism with the ranks emulated on this one GPU: each rank's pool holds its block of the experts
+    (ep_size = R), the ranks run one after the other, and each rank's partial forward is timed alone - the time one
+    GPU of an R-GPU deployment would spend per layer before the all-reduce, which is not measured here (one GPU)."""
+    import torch
+    from paper_2508_17624_b200 import binding, workloads as wl
+    cfg = wl.CONFIGS["c1"]
+    bank = wl.NoiseBank(cfg.seed)
+    tuned = wl.tuned_sets(cfg)
+    base = wl.gen_base_layer(cfg, 0, bank)
+    ads = [wl.gen_adapter_layer(cfg, i, 0, tuned[i][0], bank) for i in range(cfg.max_adapters)]
+    x = torch.from_numpy(wl.gen_tokens(cfg).view(np.int16)).cuda().view(torch.bfloat16)
+    aid = torch.from_numpy(wl.gen_adapter_ids(cfg)).cuda()
+    rec = {"workload": WORKLOADS["c1"], "all_reduce": "not measured (one GPU): fp32 [tokens, H] per layer = %d bytes" % (cfg.n_tokens * cfg.hidden * 4),
+           "ranks": {}}
+    for R, ranks in ((2, (0, 1)), (8, (0, 1, 7))):
+        per_rank = {}
+        for r in ranks:
+            pool = binding.Pool.from_config(cfg, device=device, ep_size=R, ep_rank=r)
+            pool.load_base(0, base.router_w, base.routed.w_gate, base.routed.w_up, base.routed.w_down, base.shared.w_gate,
+                           base.shared.w_up, base.shared.w_down)
+            for i, e in enumerate(ads):
+                pool.load_adapter(i, np.array([len(tuned[i][0])], np.int32), tuned[i][0].astype(np.int32), e.w_gate, e.w_up, e.w_down)
+            part = torch.empty((cfg.n_tokens, cfg.hidden), dtype=torch.float32, device="cuda")
+            for _ in range(20):
+                pool.moe_forward_partial(0, x, aid, part)
+            with sampler.window():
+                reg = timed_regions(lambda: pool.moe_forward_partial(0, x, aid, part), 300, _sync_barrier, min_total_s=0.2, max_regions=5)
+            st = pool.stats()
+            per_rank[str(r)] = {"ms_per_partial_forward": float(np.median(reg)) / 300, "live_experts": st["live_experts"],
+                                "physical_bytes": st["physical_bytes"], "kernels_per_forward": st["last_forward_kernels"]}
+            assert pool.last_device_error() == 0
+            pool.destroy()
+        rec["ranks"]["ep%d" % R] = per_rank
+    return rec
 
 
 def run_reroute(args):

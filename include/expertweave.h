@@ -65,11 +65,14 @@ typedef struct {
     float routed_scale;    /* multiplies the k combine weights (1.0 for the DeepSeek-V2-Lite shape) */
     int32_t pool_mode;     /* 0: pages mapped on demand under live experts (Section 4.2)
                               1: "padding" baseline of Section 3.1: the whole tensor is backed at creation */
-    int32_t reserved0;
+    int32_t ep_size;       /* expert parallelism (Section 5.1: "EP for MoE layers"): number of ranks the experts are
+                              partitioned over; 0 or 1 = none.  See ew_moe_forward_partial.                  */
     uint64_t page_bytes;   /* physical page size; 0 = the driver's minimum granularity (2 MiB on B200);
                               otherwise a multiple of it                                            */
     uint64_t prealloc_pages; /* pages created up front and kept in the pool's free list            */
     uint64_t max_pages;    /* 0 = unlimited; else creating more pages than this fails with EW_ERR_OOM */
+    int32_t ep_rank;       /* this pool's rank in [0, ep_size)                                              */
+    int32_t reserved0;
 } ew_config_t;
 
 /* Memory accounting (Section 4.2; Section 3.1's F_mem is padding_bytes / live_expert_bytes). */
@@ -174,6 +177,28 @@ ew_status_t ew_moe_forward_debug(ew_pool_t *pool, int32_t layer, const void *x, 
                                  int32_t n_tokens, void *out, void *cuda_stream, int32_t *topk_ids,
                                  float *topk_w, int32_t *slot_ids, int32_t *counts, int32_t *inv,
                                  int32_t *offsets);
+
+/* Expert parallelism (Section 5.1: tensor parallelism for self-attention, expert parallelism for the MoE layers;
+ * Section 5.2 runs TP = EP = 8 and 2).  The paper does not say how tokens reach experts on other devices; under tensor-
+ * parallel attention every rank holds the hidden states of all tokens, so this build needs no token exchange:
+ * a pool created with ep_size = R > 1 and ep_rank = r holds the base experts
+ *     [r * ceil(M/R), min(M, (r+1) * ceil(M/R)))
+ * with every adapter's re-tuned copies of them (a pair's device is decided by its base expert id alone, so a
+ * rerouted pair never leaves the rank of its base expert), and the shared experts [r * ceil(S/R), ...) likewise;
+ * ew_load_base / ew_load_adapter take the same full arguments on every rank and map and copy only that share, the
+ * other slots of the virtual tensors stay unbacked (Section 4.2's on-demand pages), and the expert map is the same
+ * on all ranks.  ew_moe_forward_partial runs the layer on ALL n_tokens tokens: the router (redundantly on every
+ * rank), then the grouped FFN over the pairs whose expert lives here, and writes the rank's partial sums
+ *     partial[t] = sum over local pairs j of w[t,j] * FFN_slot(t,j)(x[t]) + sum over local shared experts FFN(x[t])
+ * unrounded: DEVICE fp32 [n_tokens, H], 16-byte aligned.  The caller adds the R partials (an all-reduce; the Python
+ * package does it with torch.distributed) and calls ew_ep_finish on the sum for the layer's single rounding to bf16
+ * (summed: DEVICE fp32 [n_tokens, H]; out: DEVICE bf16 [n_tokens, H]; they may not overlap).
+ * On such a pool ew_moe_forward, ew_moe_forward_debug and ew_moe_forward_host fail with EW_ERR_INVALID_ARG.
+ * With ep_size <= 1 ew_moe_forward_partial is the whole layer, unrounded.  Other arguments, ordering and errors as
+ * for ew_moe_forward. */
+ew_status_t ew_moe_forward_partial(ew_pool_t *pool, int32_t layer, const void *x, const int32_t *adapter_ids,
+                                   int32_t n_tokens, float *partial, void *cuda_stream);
+ew_status_t ew_ep_finish(ew_pool_t *pool, const float *summed, int32_t n_tokens, void *out, void *cuda_stream);
 
 /* Same forward with HOST buffers, pipelined across calls: x and adapter_ids are uploaded to device staging
  * owned by the pool, the forward runs on them and the result is downloaded to out_host.  Upload, kernels and

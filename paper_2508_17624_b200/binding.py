@@ -23,7 +23,7 @@ STATUS_NAMES = ["EW_OK", "EW_ERR_INVALID_ARG", "EW_ERR_OOM", "EW_ERR_SLOT_IN_USE
 EXPORTS = ["ew_pool_create", "ew_pool_destroy", "ew_load_base", "ew_load_adapter", "ew_unload_adapter",
            "ew_pool_trim", "ew_moe_forward", "ew_moe_forward_debug", "ew_moe_forward_host", "ew_profile_enable",
            "ew_profile_read", "ew_reroute", "ew_reroute_unfused", "ew_route_logits", "ew_route_noalloc", "ew_selftest_bounded_wait", "ew_get_expert_map",
-           "ew_pool_stats", "ew_last_device_error", "ew_slot_address", "ew_status_str", "ew_last_error_string"]
+           "ew_moe_forward_partial", "ew_ep_finish", "ew_pool_stats", "ew_last_device_error", "ew_slot_address", "ew_status_str", "ew_last_error_string"]
 
 
 class EwConfig(C.Structure):
@@ -31,8 +31,8 @@ class EwConfig(C.Structure):
                 ("num_experts", C.c_int32), ("num_shared", C.c_int32), ("top_k", C.c_int32),
                 ("max_adapters", C.c_int32), ("e_max", C.c_int32), ("max_tokens", C.c_int32),
                 ("renormalize", C.c_int32), ("routed_scale", C.c_float), ("pool_mode", C.c_int32),
-                ("reserved0", C.c_int32), ("page_bytes", C.c_uint64), ("prealloc_pages", C.c_uint64),
-                ("max_pages", C.c_uint64)]
+                ("ep_size", C.c_int32), ("page_bytes", C.c_uint64), ("prealloc_pages", C.c_uint64),
+                ("max_pages", C.c_uint64), ("ep_rank", C.c_int32), ("reserved0", C.c_int32)]
 
 
 class EwStats(C.Structure):
@@ -101,10 +101,10 @@ class Pool:
     def __init__(self, *, device: int = 0, num_layers: int = 1, hidden: int, inter: int, num_experts: int,
                  num_shared: int, top_k: int, max_adapters: int, e_max: int, max_tokens: int,
                  renormalize: int = 0, routed_scale: float = 1.0, pool_mode: int = 0, page_bytes: int = 0,
-                 prealloc_pages: int = 0, max_pages: int = 0):
+                 prealloc_pages: int = 0, max_pages: int = 0, ep_size: int = 0, ep_rank: int = 0):
         self.cfg = EwConfig(device, num_layers, hidden, inter, num_experts, num_shared, top_k, max_adapters,
-                            e_max, max_tokens, renormalize, routed_scale, pool_mode, 0, page_bytes,
-                            prealloc_pages, max_pages)
+                            e_max, max_tokens, renormalize, routed_scale, pool_mode, ep_size, page_bytes,
+                            prealloc_pages, max_pages, ep_rank, 0)
         self._h = C.c_void_p()
         _check(lib().ew_pool_create(C.byref(self.cfg), C.byref(self._h)), "ew_pool_create")
 
@@ -154,6 +154,23 @@ class Pool:
             out = torch.empty_like(x)
         _check(lib().ew_moe_forward(self._h, layer, _dp(x), _dp(adapter_ids), x.shape[0], _dp(out), _stream()),
                "ew_moe_forward")
+        return out
+
+    def moe_forward_partial(self, layer, x, adapter_ids, partial=None):
+        """This rank's unrounded partial sums, fp32 [n_tokens, H] (expert parallelism; see the header)."""
+        import torch
+        if partial is None:
+            partial = torch.empty(x.shape, dtype=torch.float32, device=x.device)
+        _check(lib().ew_moe_forward_partial(self._h, layer, _dp(x), _dp(adapter_ids), x.shape[0], _dp(partial), _stream()),
+               "ew_moe_forward_partial")
+        return partial
+
+    def ep_finish(self, summed, out=None):
+        """bf16 result from the sum of all ranks' partials."""
+        import torch
+        if out is None:
+            out = torch.empty(summed.shape, dtype=torch.bfloat16, device=summed.device)
+        _check(lib().ew_ep_finish(self._h, _dp(summed), summed.shape[0], _dp(out), _stream()), "ew_ep_finish")
         return out
 
     def moe_forward_debug(self, layer, x, adapter_ids):

@@ -694,7 +694,7 @@ plan::SelfPlan self_plan_args(const ew_pool *p, int B, int pass) {
     if (!p->self_plan) return sp;
     const ew_config_t &c = p->cfg;
     sp.counts = p->ws.counts;
-    sp.B = B; sp.k = c.top_k; sp.P = p->P; sp.S = c.num_shared;
+    sp.B = B; sp.k = c.top_k; sp.P = p->P; sp.S = p->sh_hi - p->sh_lo; sp.sh0 = p->sh_lo;
     sp.nt_shift = p->token_tile == 32 ? 5 : p->token_tile == 64 ? 6 : 7;
     sp.R = ((pass ? c.hidden : c.inter) + 127) / 128;
     sp.pass = pass;
@@ -724,7 +724,7 @@ bool self_plan_fits(const ew_pool *p, int B, int NT) {
         case 64: self_limits<64, true>(&cap1, &scr1); self_limits<64, false>(&cap2, &scr2); break;
         default: self_limits<128, true>(&cap1, &scr1); self_limits<128, false>(&cap2, &scr2); break;
     }
-    const size_t need = plan::self_plan_words(p->P, c.num_shared) * 4;
+    const size_t need = plan::self_plan_words(p->P, c.num_shared) * 4;      // (fewer shared experts with expert parallelism)
     if (need > scr1 || need > scr2 || p->P + c.num_shared > plan::kSelfMaxGroups) return false;
     // token blocks of any routing: at most floor(B k / NT) full ones plus one ragged block per live slot, plus the shared experts'
     const long long pairs = (long long)B * c.top_k;

@@ -64,6 +64,10 @@ struct LayerState {
 struct ew_pool {
     ew_config_t cfg;
     int P = 0;                      // M + N * E_max
+    // expert parallelism: this rank holds the base experts [own_lo, own_hi) with every adapter's copies of them, and
+    // the shared experts [sh_lo, sh_hi); without it, all of them
+    int own_lo = 0, own_hi = 0, sh_lo = 0, sh_hi = 0;
+    std::vector<std::vector<std::pair<int32_t, int32_t>>> adapter_owned;   // [N][L] positions [first, last) of an adapter's tuned experts held here
     int token_tile = 32;            // NT: token rows per thin work item (32, 64 or 128)
     bool fat = false;               // prefill-sized batch: blocks of more than 128 rows run on the CTA-pair kernel
     int last_forward_kernels = 0;   // kernels launched by the most recent forward (reported by ew_pool_stats)
@@ -156,7 +160,8 @@ int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, const CUtensor
                  cudaStream_t st);
 int pick_token_tile(const ew_pool *p, int B);
 int launch_gemm2(ew_pool *p, int layer, int B, cudaStream_t st);
-int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st);
+int launch_combine(ew_pool *p, int B, void *out, bool f32_out, cudaStream_t st);   // f32_out: fp32 partial sums (expert parallelism)
+int launch_round_bf16(const float *in, void *out, size_t n, cudaStream_t st);
 int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid, int B, int32_t *slots,
                    int32_t *counts, cudaStream_t st);
 int launch_route_logits(ew_pool *p, int layer, const float *logits, const int32_t *aid, int B, int32_t *topk_ids,

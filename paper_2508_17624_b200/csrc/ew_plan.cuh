@@ -41,7 +41,8 @@ __device__ inline void block_exclusive_scan(const int32_t *in, int32_t *out, int
 }
 
 struct Params {
-    int B, k, P, S;
+    int B, k, P;
+    int S, sh0;          // shared experts computed here: slots P + sh0 .. P + sh0 + S - 1 (all of them without expert parallelism)
     int NT;              // token rows per "thin" work item (swap-AB kernel: weight tile x up to NT token rows)
     int fat;             // 1: blocks of more than kFatMin rows go to the CTA-pair kernel (256 token rows x 256 weight rows)
     int R1, R2;          // weight tiles per group of the thin GEMM-1 / GEMM-2 items (128 rows each)
@@ -115,7 +116,7 @@ __device__ inline void write_items(int32_t *sm, const int32_t *cnt_s, const Para
         const bool shared = g < S;
         const int rows = shared ? B : cnt_s[g - S];
         if (rows == 0) continue;
-        const int slot = shared ? P + g : g - S;
+        const int slot = shared ? P + A.sh0 + g : g - S;
         const int in0 = shared ? 0 : off[g - S];                  // GEMM-1 reads x rows (shared) or slot-contiguous rows
         const int act0 = shared ? g * B : S * B + off[g - S];     // rows of act: GEMM-1 writes them, GEMM-2 reads them
         const int y0 = shared ? 0 : y_base + off[g - S];          // rows of Y
@@ -154,7 +155,8 @@ __device__ inline void write_items(int32_t *sm, const int32_t *cnt_s, const Para
 // Self-planned forwards (decode-sized batches: thin items only).
 struct SelfPlan {
     const int32_t *counts;       // [P] per-slot pair counts of the router kernel; null: walk the planner's item list
-    int B, k, P, S;
+    int B, k, P;
+    int S, sh0;                  // shared experts computed here: slots P + sh0 .. P + sh0 + S - 1
     int nt_shift;                // token rows per item NT = 1 << nt_shift (32, 64 or 128)
     int R;                       // weight tiles per group of this GEMM
     int pass;                    // 0: GEMM-1 (+ SwiGLU), 1: GEMM-2
@@ -265,7 +267,7 @@ __device__ __forceinline__ int derive_items(int32_t *sm, const SelfPlan &A, int 
         int tile = local, c = 0;
         if (nt > 1) { tile = local / nt; c = local - tile * nt; }
         const int r0 = c << A.nt_shift;
-        const int slot = shared ? P + g : g - S;
+        const int slot = shared ? P + A.sh0 + g : g - S;
         const int act0 = shared ? g * B : S * B + off[shared ? 0 : g - S];
         const int in0 = shared ? 0 : (g - S) * B;                // routed rows: index into the slot-major token table
         const int y0 = shared ? 0 : y_base + off[shared ? 0 : g - S];
@@ -279,8 +281,9 @@ __device__ __forceinline__ int derive_items(int32_t *sm, const SelfPlan &A, int 
             for (int i = threadIdx.x; i <= P; i += nthreads) A.offsets[i] = off[i];
         for (long long q = q0; q < n_pairs; q += (long long)gridDim.x * nthreads) {
             if (q != q0) { my_slot = __ldcg(A.slot_ids + q); my_rank = __ldcg(A.rank + q); }
-            const int dest = off[min(max(my_slot, 0), P - 1)] + my_rank;
-            if (dest >= 0 && dest < n_pairs && !dry) A.inv[q] = dest;    // always, unless the routing kernel gave up midway
+            // position -1: the pair belongs to another rank (expert parallelism)
+            const int dest = my_rank < 0 ? -1 : off[min(max(my_slot, 0), P - 1)] + my_rank;
+            if (dest < n_pairs && !dry) A.inv[q] = dest;         // always, unless the routing kernel gave up midway
         }
     }
     __syncthreads();

@@ -181,7 +181,8 @@ extern "C" ew_status_t ew_pool_create(const ew_config_t *cfg, ew_pool_t **out) {
     if (c.num_layers < 1 || c.hidden < 64 || c.inter < 8 || c.hidden % 64 || c.inter % 8 || c.num_experts < 1 ||
         c.num_experts > 256 || c.num_shared < 0 || c.top_k < 1 || c.top_k > 32 || c.top_k > c.num_experts ||
         c.max_adapters < 0 || c.e_max < 0 || c.max_tokens < 1 || (c.pool_mode != 0 && c.pool_mode != 1) ||
-        (c.max_adapters > 0 && c.e_max < 1)) {
+        (c.max_adapters > 0 && c.e_max < 1) || c.ep_size < 0 || c.ep_size > c.num_experts ||
+        (c.ep_size > 1 ? (c.ep_rank < 0 || c.ep_rank >= c.ep_size) : c.ep_rank != 0)) {
         set_last_error("ew_pool_create: configuration out of range");
         return EW_ERR_INVALID_ARG;
     }
@@ -189,6 +190,14 @@ extern "C" ew_status_t ew_pool_create(const ew_config_t *cfg, ew_pool_t **out) {
     if (!p) return EW_ERR_OOM;
     p->cfg = c;
     p->P = c.num_experts + c.max_adapters * c.e_max;
+    {   // expert parallelism: contiguous blocks of base experts (and of shared experts) per rank
+        const int R = c.ep_size > 1 ? c.ep_size : 1, r = c.ep_rank;
+        const int per = (c.num_experts + R - 1) / R, per_s = (c.num_shared + R - 1) / R;
+        p->own_lo = std::min(c.num_experts, r * per);
+        p->own_hi = std::min(c.num_experts, p->own_lo + per);
+        p->sh_lo = std::min(c.num_shared, r * per_s);
+        p->sh_hi = std::min(c.num_shared, p->sh_lo + per_s);
+    }
     bool gpu = c.device >= 0;
     ew_status_t st = EW_OK;
     std::string err;
@@ -228,6 +237,7 @@ extern "C" ew_status_t ew_pool_create(const ew_config_t *cfg, ew_pool_t **out) {
     p->pages.page_bytes = page;
     p->pages.max_pages = c.max_pages;
     p->adapter_counts.assign(c.max_adapters, {});
+    p->adapter_owned.assign(c.max_adapters, {});
     size_t H = c.hidden, I = c.inter, slots = (size_t)p->P + c.num_shared;
     p->layers.resize(c.num_layers);
     for (auto &L : p->layers) {
@@ -325,14 +335,16 @@ extern "C" ew_status_t ew_load_base(ew_pool_t *p, int32_t layer, const void *rou
     DeviceGuard guard;
     if (gpu) CU_TRY(guard.enter(c.device));
     LayerState &L = p->layers[layer];
-    size_t M = c.num_experts, S = c.num_shared, P = p->P;
+    size_t M = c.num_experts, P = p->P;
+    // the experts this rank holds (all of them without expert parallelism): base [m0, m0 + Mo), shared [s0, s0 + So)
+    const size_t m0 = p->own_lo, Mo = p->own_hi - p->own_lo, s0 = p->sh_lo, So = p->sh_hi - p->sh_lo;
     if (!L.base_mapped && c.pool_mode == 0) {
         ew_status_t st;
-        if ((st = be_status(p, L.w13.map_slots(0, M))) != EW_OK) return st;
-        if ((st = be_status(p, L.w2.map_slots(0, M))) != EW_OK) { L.w13.unmap_slots(0, M); return st; }
-        if ((st = be_status(p, L.w13.map_slots(P, S))) != EW_OK) { L.w13.unmap_slots(0, M); L.w2.unmap_slots(0, M); return st; }
-        if ((st = be_status(p, L.w2.map_slots(P, S))) != EW_OK) {
-            L.w13.unmap_slots(0, M); L.w2.unmap_slots(0, M); L.w13.unmap_slots(P, S);
+        if ((st = be_status(p, L.w13.map_slots(m0, Mo))) != EW_OK) return st;
+        if ((st = be_status(p, L.w2.map_slots(m0, Mo))) != EW_OK) { L.w13.unmap_slots(m0, Mo); return st; }
+        if ((st = be_status(p, L.w13.map_slots(P + s0, So))) != EW_OK) { L.w13.unmap_slots(m0, Mo); L.w2.unmap_slots(m0, Mo); return st; }
+        if ((st = be_status(p, L.w2.map_slots(P + s0, So))) != EW_OK) {
+            L.w13.unmap_slots(m0, Mo); L.w2.unmap_slots(m0, Mo); L.w13.unmap_slots(P + s0, So);
             return st;
         }
     }
@@ -341,15 +353,17 @@ extern "C" ew_status_t ew_load_base(ew_pool_t *p, int32_t layer, const void *rou
         // forwards in flight may still read the old weights of this layer
         for (auto &e : p->fwd_events) CU_TRY(cudaEventSynchronize(e.second));
         if (p->route_event_used) CU_TRY(cudaEventSynchronize(p->route_event));
+        const size_t blk = (size_t)c.inter * c.hidden * 2;
+        auto at = [blk](const void *base, size_t i) { return (const void *)((const char *)base + i * blk); };
         CU_TRY(cudaMemcpyAsync(L.router_w, router_w, M * c.hidden * 2, cudaMemcpyDefault, p->copy_stream));
-        ew_status_t st = copy_experts(p, L, 0, M, w_gate, w_up, w_down);
-        if (st == EW_OK && S) st = copy_experts(p, L, P, S, sh_gate, sh_up, sh_down);
+        ew_status_t st = copy_experts(p, L, m0, Mo, at(w_gate, m0), at(w_up, m0), at(w_down, m0));
+        if (st == EW_OK && So) st = copy_experts(p, L, P + s0, So, at(sh_gate, s0), at(sh_up, s0), at(sh_down, s0));
         if (st != EW_OK) return st;
         CU_TRY(cudaStreamSynchronize(p->copy_stream));
     }
     if (!L.base_loaded) {                               // counted once, when the first load of the layer has succeeded
-        p->live_experts += M;
-        p->live_expert_bytes += (M + S) * 3 * (size_t)c.inter * c.hidden * 2;
+        p->live_experts += Mo;
+        p->live_expert_bytes += (Mo + So) * 3 * (size_t)c.inter * c.hidden * 2;
     }
     L.base_loaded = true;
     return EW_OK;
@@ -380,6 +394,19 @@ extern "C" ew_status_t ew_load_adapter(ew_pool_t *p, int32_t a, const int32_t *c
     DeviceGuard guard;
     if (gpu) CU_TRY(guard.enter(c.device));
     size_t delta = (size_t)M + (size_t)a * c.e_max;     // Delta_i = M + i * E_max
+    // Expert parallelism: of each layer's tuned experts (ascending base ids) this rank holds those whose base expert
+    // it holds, a contiguous run [first, last) of positions; the others' slots stay unmapped here.
+    std::vector<std::pair<int32_t, int32_t>> own(L);
+    size_t owned_total = 0;
+    for (size_t l = 0, q0 = 0; l < (size_t)L; q0 += counts[l], ++l) {
+        int lo = 0, hi = 0;
+        for (int r = 0; r < counts[l]; ++r) {
+            if (expert_ids[q0 + r] < p->own_lo) ++lo;
+            if (expert_ids[q0 + r] < p->own_hi) ++hi;
+        }
+        own[l] = {lo, hi};
+        owned_total += hi - lo;
+    }
     ew_status_t st = EW_OK;
     // Layer by layer, tensor by tensor: map the slots' pages (driver calls on this thread, ~0.1 ms per page), then
     // queue the copy into them, so that the copies run while the next pages are being mapped.
@@ -389,11 +416,12 @@ extern "C" ew_status_t ew_load_adapter(ew_pool_t *p, int32_t a, const int32_t *c
     size_t q = 0;
     for (int l = 0; l < L && st == EW_OK; ++l) {
         LayerState &Ls = p->layers[l];
-        if (vmm && (st = be_status(p, Ls.w13.map_slots(delta, counts[l]))) == EW_OK) ++done13;
+        const size_t first = delta + own[l].first, n = own[l].second - own[l].first, src = q + own[l].first;
+        if (vmm && (st = be_status(p, Ls.w13.map_slots(first, n))) == EW_OK) ++done13;
         if (st == EW_OK && gpu)
-            st = copy_gate_up(p, Ls, delta, counts[l], (const char *)w_gate + q * blk, (const char *)w_up + q * blk);
-        if (st == EW_OK && vmm && (st = be_status(p, Ls.w2.map_slots(delta, counts[l]))) == EW_OK) ++done2;
-        if (st == EW_OK && gpu) st = copy_down(p, Ls, delta, counts[l], (const char *)w_down + q * blk);
+            st = copy_gate_up(p, Ls, first, n, (const char *)w_gate + src * blk, (const char *)w_up + src * blk);
+        if (st == EW_OK && vmm && (st = be_status(p, Ls.w2.map_slots(first, n))) == EW_OK) ++done2;
+        if (st == EW_OK && gpu) st = copy_down(p, Ls, first, n, (const char *)w_down + src * blk);
         q += counts[l];
     }
     if (gpu && cudaStreamSynchronize(p->copy_stream) != cudaSuccess && st == EW_OK) {   // also before any rollback
@@ -401,8 +429,8 @@ extern "C" ew_status_t ew_load_adapter(ew_pool_t *p, int32_t a, const int32_t *c
         st = EW_ERR_CUDA;
     }
     if (st != EW_OK) {
-        for (int l = 0; l < done13; ++l) p->layers[l].w13.unmap_slots(delta, counts[l]);
-        for (int l = 0; l < done2; ++l) p->layers[l].w2.unmap_slots(delta, counts[l]);
+        for (int l = 0; l < done13; ++l) p->layers[l].w13.unmap_slots(delta + own[l].first, own[l].second - own[l].first);
+        for (int l = 0; l < done2; ++l) p->layers[l].w2.unmap_slots(delta + own[l].first, own[l].second - own[l].first);
         return st;
     }
     // publish: Pi[l][a][j] = Delta + rank of j, only after the weights are in place
@@ -418,8 +446,9 @@ extern "C" ew_status_t ew_load_adapter(ew_pool_t *p, int32_t a, const int32_t *c
         CU_TRY(cudaStreamSynchronize(p->copy_stream));
     }
     p->adapter_counts[a].assign(counts, counts + L);
-    p->live_experts += total;
-    p->live_expert_bytes += total * 3 * blk;
+    p->adapter_owned[a] = own;
+    p->live_experts += owned_total;
+    p->live_expert_bytes += owned_total * 3 * blk;
     return EW_OK;
 }
 
@@ -452,14 +481,16 @@ extern "C" ew_status_t ew_unload_adapter(ew_pool_t *p, int32_t a) {
     // 3. drop the reference counts; pages reaching zero go back to the pool
     size_t delta = (size_t)M + (size_t)a * c.e_max, total = 0;
     for (int l = 0; l < L; ++l) {
-        int e = p->adapter_counts[a][l];
+        const auto &o = p->adapter_owned[a][l];
+        const int e = o.second - o.first;
         total += e;
         if (c.pool_mode == 0) {
-            p->layers[l].w13.unmap_slots(delta, e);
-            p->layers[l].w2.unmap_slots(delta, e);
+            p->layers[l].w13.unmap_slots(delta + o.first, e);
+            p->layers[l].w2.unmap_slots(delta + o.first, e);
         }
     }
     p->adapter_counts[a].clear();
+    p->adapter_owned[a].clear();
     p->live_experts -= total;
     p->live_expert_bytes -= total * 3 * (size_t)c.inter * c.hidden * 2;
     return EW_OK;
@@ -569,12 +600,16 @@ static ew_status_t note_forward(ew_pool *p, cudaStream_t st) {
         }                                                                                      \
     } while (0)
 
-extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const void *x, const int32_t *aid,
-                                            int32_t B, void *out, void *cuda_stream, int32_t *topk_ids,
-                                            float *topk_w, int32_t *slot_ids, int32_t *counts, int32_t *inv,
-                                            int32_t *offsets) {
+// The forward.  f32_out: `out` receives this rank's fp32 partial sums instead of the rounded bf16 result.
+static ew_status_t forward_impl(ew_pool_t *p, int32_t layer, const void *x, const int32_t *aid, int32_t B, void *out,
+                                bool f32_out, void *cuda_stream, int32_t *topk_ids, float *topk_w, int32_t *slot_ids,
+                                int32_t *counts, int32_t *inv, int32_t *offsets) {
     if (!p || layer < 0 || layer >= p->cfg.num_layers || B < 0 || B > p->cfg.max_tokens) return EW_ERR_INVALID_ARG;
     if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
+    if (!f32_out && p->cfg.ep_size > 1) {
+        set_last_error("this pool holds one rank's share of the experts: call ew_moe_forward_partial, add the ranks' partial sums, then ew_ep_finish");
+        return EW_ERR_INVALID_ARG;
+    }
     if (B == 0) return EW_OK;
     if (!x || !aid || !out || ((uintptr_t)x & 15) || ((uintptr_t)out & 15)) return EW_ERR_INVALID_ARG;
     if (!p->layers[layer].base_loaded) return EW_ERR_NOT_LOADED;
@@ -636,7 +671,7 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     PROF_MARK(3);
     LAUNCH_TRY(launch_gemm2(p, layer, B, st));
     PROF_MARK(4);
-    LAUNCH_TRY(launch_combine(p, B, out, st));
+    LAUNCH_TRY(launch_combine(p, B, out, f32_out, st));
     p->counts_clean = true;                             // the combine kernel zeroes the counters when it is done with them
     p->last_forward_kernels = p->self_plan ? 4 : p->fat ? 7 : 5;
     PROF_MARK(5);
@@ -644,10 +679,32 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
     return note_forward(p, st);
 }
 
+extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const void *x, const int32_t *aid,
+                                            int32_t B, void *out, void *cuda_stream, int32_t *topk_ids,
+                                            float *topk_w, int32_t *slot_ids, int32_t *counts, int32_t *inv,
+                                            int32_t *offsets) {
+    return forward_impl(p, layer, x, aid, B, out, false, cuda_stream, topk_ids, topk_w, slot_ids, counts, inv, offsets);
+}
+
 extern "C" ew_status_t ew_moe_forward(ew_pool_t *p, int32_t layer, const void *x, const int32_t *aid, int32_t B,
                                       void *out, void *cuda_stream) {
-    return ew_moe_forward_debug(p, layer, x, aid, B, out, cuda_stream, nullptr, nullptr, nullptr, nullptr, nullptr,
-                                nullptr);
+    return forward_impl(p, layer, x, aid, B, out, false, cuda_stream, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr);
+}
+
+extern "C" ew_status_t ew_moe_forward_partial(ew_pool_t *p, int32_t layer, const void *x, const int32_t *aid, int32_t B,
+                                              float *partial, void *cuda_stream) {
+    return forward_impl(p, layer, x, aid, B, partial, true, cuda_stream, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr);
+}
+
+extern "C" ew_status_t ew_ep_finish(ew_pool_t *p, const float *summed, int32_t B, void *out, void *cuda_stream) {
+    if (!p || B < 0) return EW_ERR_INVALID_ARG;
+    if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
+    if (B == 0) return EW_OK;
+    if (!summed || !out || ((uintptr_t)summed & 15) || ((uintptr_t)out & 7)) return EW_ERR_INVALID_ARG;
+    DeviceGuard guard;
+    CU_TRY(guard.enter(p->cfg.device));
+    LAUNCH_TRY(launch_round_bf16(summed, out, (size_t)B * p->cfg.hidden, (cudaStream_t)cuda_stream));
+    return EW_OK;
 }
 
 extern "C" ew_status_t ew_reroute(ew_pool_t *p, int32_t layer, const int32_t *topk_ids, const int32_t *aid,

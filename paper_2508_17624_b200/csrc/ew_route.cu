@@ -500,8 +500,11 @@ __global__ void __launch_bounds__(256) permute_kernel(const int32_t *slot_ids, c
         // one thread per (token, j) pair records the pair's row and the row's token
         const long long q = (long long)(blockIdx.x - kPlanners) * 256 + threadIdx.x;
         if (q < n_pairs) {
-            const int dest = off[slot_ids[q]] + rank[q];
-            if (dest < n_pairs) {            // always, unless the routing kernel gave up midway (error word set)
+            const int rk = rank[q];
+            const int dest = rk < 0 ? -1 : off[slot_ids[q]] + rk;    // position -1: the pair belongs to another rank (expert parallelism)
+            if (dest < 0) {
+                inv[q] = -1;
+            } else if (dest < n_pairs) {     // always, unless the routing kernel gave up midway (error word set)
                 inv[q] = dest;
                 src_tok[dest] = (int32_t)(q / A.k);
             }
@@ -517,9 +520,10 @@ __global__ void __launch_bounds__(256) permute_kernel(const int32_t *slot_ids, c
 // sum of the shared experts' outputs (GEMM-2 chains them along K); the routed rows start at Yb = B (0 without shared
 // experts).
 // ------------------------------------------------------------------------------------------------
+template <bool F32OUT>
 __global__ void __launch_bounds__(256) combine_kernel(const float4 *y, const int32_t *inv,
                                                       const float *w, int B, int k, int H, int S,
-                                                      uint2 *out, int32_t *counts, int P) {
+                                                      void *out, int32_t *counts, int P) {
     __shared__ int32_t rows[32];
     __shared__ float wts[32];
     const int t = blockIdx.x;
@@ -529,7 +533,8 @@ __global__ void __launch_bounds__(256) combine_kernel(const float4 *y, const int
         for (int i = threadIdx.x; i < P; i += blockDim.x) counts[i] = 0;
     const int y_base = S > 0 ? B : 0;
     if (threadIdx.x < k) {
-        rows[threadIdx.x] = y_base + inv[(size_t)t * k + threadIdx.x];
+        const int r = inv[(size_t)t * k + threadIdx.x];
+        rows[threadIdx.x] = r < 0 ? -1 : y_base + r;    // -1: the pair's expert lives on another rank (expert parallelism)
         wts[threadIdx.x] = w[(size_t)t * k + threadIdx.x];
     }
     __syncthreads();
@@ -537,6 +542,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const float4 *y, const int
     for (int v = threadIdx.x; v < hv; v += blockDim.x) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int j = 0; j < k; ++j) {
+            if (rows[j] < 0) continue;
             const float4 a = y[(size_t)rows[j] * hv + v];
             const float wj = wts[j];
             acc.x = fmaf(wj, a.x, acc.x); acc.y = fmaf(wj, a.y, acc.y);
@@ -546,11 +552,28 @@ __global__ void __launch_bounds__(256) combine_kernel(const float4 *y, const int
             const float4 a = y[(size_t)t * hv + v];
             acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
         }
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+        if (F32OUT) {                                   // this rank's partial sum, rounded after the sum over ranks
+            reinterpret_cast<float4 *>(out)[(size_t)t * hv + v] = acc;
+        } else {
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+            uint2 o;
+            o.x = *reinterpret_cast<const uint32_t *>(&lo);
+            o.y = *reinterpret_cast<const uint32_t *>(&hi);
+            reinterpret_cast<uint2 *>(out)[(size_t)t * hv + v] = o;
+        }
+    }
+}
+
+// out[i] = bf16(partial[i]): the single rounding of the layer's output, after the partial sums of all ranks have been
+// added (expert parallelism)
+__global__ void __launch_bounds__(256) round_bf16_kernel(const float4 *in, uint2 *out, size_t n4) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        const float4 a = in[i];
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
         uint2 o;
         o.x = *reinterpret_cast<const uint32_t *>(&lo);
         o.y = *reinterpret_cast<const uint32_t *>(&hi);
-        out[(size_t)t * hv + v] = o;
+        out[i] = o;
     }
 }
 
@@ -567,7 +590,7 @@ int pick_token_tile(const ew_pool *p, int B) {
 int launch_permute(ew_pool *p, int B, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
     plan::Params A;
-    A.B = B; A.k = c.top_k; A.P = p->P; A.S = c.num_shared;
+    A.B = B; A.k = c.top_k; A.P = p->P; A.S = p->sh_hi - p->sh_lo; A.sh0 = p->sh_lo;
     A.NT = p->token_tile; A.fat = p->fat ? 1 : 0;
     A.R1 = (c.inter + 127) / 128; A.R2 = (c.hidden + 127) / 128;
     A.RF1 = (c.inter + 127) / 128; A.RF2 = (c.hidden + 255) / 256;
@@ -575,15 +598,26 @@ int launch_permute(ew_pool *p, int B, cudaStream_t st) {
     A.n_items = p->ws.n_items;
     const long long pairs = (long long)B * c.top_k;
     const int grid = (int)((pairs + 255) / 256) + kPlanners;
-    const size_t smem = plan::smem_words(p->P, c.num_shared) * 4;
+    const size_t smem = plan::smem_words(p->P, A.S) * 4;
     return launch_pdl(permute_kernel, dim3(grid), dim3(256), smem, st, (const int32_t *)p->ws.slot_ids, (const int32_t *)p->ws.rank,
                       (const int32_t *)p->ws.counts, A, p->ws.inv, p->ws.src_tok);
 }
 
-int launch_combine(ew_pool *p, int B, void *out, cudaStream_t st) {
+int launch_combine(ew_pool *p, int B, void *out, bool f32_out, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
-    return launch_pdl(combine_kernel, dim3(B), dim3(256), 0, st, (const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B, c.top_k,
-                      c.hidden, c.num_shared, (uint2 *)out, p->ws.counts, p->P);
+    const int S = p->sh_hi - p->sh_lo;                  // the shared experts this rank computes
+    if (f32_out)
+        return launch_pdl(combine_kernel<true>, dim3(B), dim3(256), 0, st, (const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B,
+                          c.top_k, c.hidden, S, out, p->ws.counts, p->P);
+    return launch_pdl(combine_kernel<false>, dim3(B), dim3(256), 0, st, (const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B,
+                      c.top_k, c.hidden, S, out, p->ws.counts, p->P);
+}
+
+int launch_round_bf16(const float *in, void *out, size_t n, cudaStream_t st) {
+    const size_t n4 = n / 4;
+    const int grid = (int)std::min<size_t>((n4 + 255) / 256, 148 * 8);
+    round_bf16_kernel<<<grid, 256, 0, st>>>((const float4 *)in, (uint2 *)out, n4);
+    return (int)cudaGetLastError();
 }
 
 int launch_route_logits(ew_pool *p, int layer, const float *logits, const int32_t *aid, int B, int32_t *topk_ids,

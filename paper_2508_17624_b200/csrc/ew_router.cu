@@ -65,12 +65,15 @@ struct RouterArgs {
     float *topk_w;
     int32_t *slot_ids, *rank, *counts;
     int *err;
+    int own_lo = 0, own_hi = 1 << 30;   // expert parallelism: pairs whose base expert lies outside [own_lo, own_hi) belong to another rank:
+                                        // ids, weights and slot ids are written as usual, but they are not counted and get position -1
     int32_t *slot_tok = nullptr;   // [P][B] or null.  Forwards without a planning kernel: the token of the pair at position r of slot s
 };
 
 // write one selected pair: reroute through Pi, outputs (the histogram follows in emit_ranks)
 __device__ __forceinline__ void emit_pair(const RouterArgs &A, const int32_t *pi_s, int t, int r, int a, int id, float w,
-                                          int (&sl)[8]) {
+                                          int (&sl)[8], uint32_t &local_mask) {
+    if (id >= A.own_lo && id < A.own_hi) local_mask |= 1u << r;
     const int slot = a < 0 ? id : (A.pi_in_smem ? pi_s[a * A.M + id] : __ldg(A.pi + a * A.M + id));
     const size_t o = (size_t)t * A.k + r;
     A.topk_ids[o] = id;
@@ -83,12 +86,13 @@ __device__ __forceinline__ void emit_pair(const RouterArgs &A, const int32_t *pi
 
 // per-slot histogram: one atomic per pair, eight in flight per thread; the value returned is the
 // pair's position inside its slot's chunk
-__device__ __forceinline__ void emit_ranks(const RouterArgs &A, int t, const int (&sl)[8]) {
+__device__ __forceinline__ void emit_ranks(const RouterArgs &A, int t, const int (&sl)[8], uint32_t local_mask) {
     for (int r0 = 0; r0 < A.k; r0 += 8) {
         int got[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u)
-            if (r0 + u < A.k) got[u] = atomicAdd(A.counts + (r0 == 0 ? sl[u] : A.slot_ids[(size_t)t * A.k + r0 + u]), 1);
+            if (r0 + u < A.k)
+                got[u] = ((local_mask >> (r0 + u)) & 1u) ? atomicAdd(A.counts + (r0 == 0 ? sl[u] : A.slot_ids[(size_t)t * A.k + r0 + u]), 1) : -1;
 #pragma unroll
         for (int u = 0; u < 8; ++u)
             if (r0 + u < A.k) {
@@ -272,6 +276,7 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
             float wsum = 0.f;
             float my_w[8];                                           // weights and slots of the pairs this thread writes (r = g, g+4, ...)
             int my_slot[8];
+            uint32_t my_local = 0;                                   // bit u: pair g + 4u belongs to this rank (expert parallelism)
             for (int r = 0; r < k; ++r) {
                 float bv = -1.f;
                 int bi = 0;
@@ -308,6 +313,7 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
 #pragma unroll
                     for (int u = 0; u < 8; ++u)
                         if (u == (r >> 2)) { my_w[u] = wv; my_slot[u] = slot; }
+                    if (wi >= A.own_lo && wi < A.own_hi) my_local |= 1u << (r >> 2);
                 }
             }
             if (t < A.B) {
@@ -316,7 +322,7 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                 int got[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u)
-                    if (g + 4 * u < k) got[u] = atomicAdd(A.counts + my_slot[u], 1);
+                    if (g + 4 * u < k) got[u] = ((my_local >> u) & 1u) ? atomicAdd(A.counts + my_slot[u], 1) : -1;
 #pragma unroll
                 for (int u = 0; u < 8; ++u)
                     if (g + 4 * u < k) {
@@ -365,6 +371,7 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                     const int a = checked_aid(A.aid[t], A.N, A.loaded, A.err);
                     float wsum = 0.f;
                     int sl[8];
+                    uint32_t local_mask = 0;
                     for (int r = 0; r < k; ++r) {
                         float bv = -1.f;
                         int bi = 0;
@@ -377,9 +384,9 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
 #pragma unroll
                         for (int j = 0; j < 64; ++j) p[j] = (j == bi) ? -1.f : p[j];   // taken (probabilities are >= 0)
                         wsum += bv;
-                        emit_pair(A, pi_s, t, r, a, bi, bv, sl);
+                        emit_pair(A, pi_s, t, r, a, bi, bv, sl, local_mask);
                     }
-                    emit_ranks(A, t, sl);
+                    emit_ranks(A, t, sl, local_mask);
                     if (A.renormalize || A.scale != 1.f)
                         for (int r = 0; r < k; ++r) {
                             const size_t o = (size_t)t * k + r;
@@ -415,6 +422,7 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                     const int a = checked_aid(A.aid[t], A.N, A.loaded, A.err);
                     float wsum = 0.f;
                     int sl[8];
+                    uint32_t local_mask = 0;
                     for (int r = 0; r < k; ++r) {
                         float bv = -1.f;
                         int bi = 0;
@@ -426,9 +434,9 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                         }
                         pbuf[bi * kTileRows + tl] = -1.f;
                         wsum += bv;
-                        emit_pair(A, pi_s, t, r, a, bi, bv, sl);
+                        emit_pair(A, pi_s, t, r, a, bi, bv, sl, local_mask);
                     }
-                    emit_ranks(A, t, sl);
+                    emit_ranks(A, t, sl, local_mask);
                     if (A.renormalize || A.scale != 1.f)
                         for (int r = 0; r < k; ++r) {
                             const size_t o = (size_t)t * k + r;
@@ -554,6 +562,7 @@ int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B
     A.topk_ids = p->ws.topk_ids; A.topk_w = p->ws.topk_w; A.slot_ids = p->ws.slot_ids; A.rank = p->ws.rank;
     A.counts = p->ws.counts; A.err = p->ws.err;
     A.slot_tok = p->self_plan ? p->ws.slot_tok : nullptr;
+    A.own_lo = p->own_lo; A.own_hi = p->own_hi;
     return router_launch(p, layer, x, g, A, true, st);
 }
 

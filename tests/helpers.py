@@ -39,6 +39,28 @@ def oracle_layer(cfg, layer, bank, tuned, base=None, adapters=None) -> oracle.Or
                               base.routed.w_down, base.shared.w_gate, base.shared.w_up, base.shared.w_down, ads)
 
 
+def oracle_partial(cfg, layer, bank, tuned, x_bits, ids, slots, w, ep_size, ep_rank, base=None, adapters=None):
+    """What rank `ep_rank` of `ep_size` contributes to the layer output under expert parallelism, from the oracle:
+    the pairs whose base expert id lies in the rank's block keep their weight, all others get weight 0, and only
+    the rank's shared experts are present.  fp32 [B, H]; the sum over ranks is the oracle's layer output up to the
+    order of the fp32 additions."""
+    from paper_2508_17624_b200 import ep
+    base = base or wl.gen_base_layer(cfg, layer, bank)
+    s_lo, s_hi = ep.owned_range(cfg.num_shared, ep_size, ep_rank)
+    ocfg = oracle.OracleConfig(cfg.hidden, cfg.inter, cfg.num_experts, s_hi - s_lo, cfg.top_k, cfg.max_adapters, cfg.e_max)
+    ads = []
+    for i in range(cfg.max_adapters):
+        if adapters is not None and i not in adapters:
+            ads.append(None)
+            continue
+        ew = wl.gen_adapter_layer(cfg, i, layer, tuned[i][layer], bank)
+        ads.append((tuned[i][layer], ew.w_gate, ew.w_up, ew.w_down))
+    ol = oracle.OracleLayer(ocfg, base.router_w, base.routed.w_gate, base.routed.w_up, base.routed.w_down,
+                            base.shared.w_gate[s_lo:s_hi], base.shared.w_up[s_lo:s_hi], base.shared.w_down[s_lo:s_hi], ads)
+    mask = ep.local_pair_mask(ids, cfg.num_experts, ep_size, ep_rank)
+    return oracle.ffn_given_slots(ol, x_bits, slots, np.where(mask, w, np.float32(0)).astype(np.float32))
+
+
 def to_dev(bits_or_ids, dtype=None):
     import torch
     a = np.ascontiguousarray(bits_or_ids)

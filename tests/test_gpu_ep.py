@@ -1,0 +1,90 @@
+"""Expert parallelism on one GPU: the R ranks are R pools on the same device, run one after the other, and their partial
+sums are added with a plain tensor addition in the place of the all-reduce.  (Kernels of different ranks never wait on
+one another, so this is the multi-rank data path exactly, minus the link.)  Every rank's partial sum and the finished
+layer output are compared with the oracle."""
+import numpy as np
+import pytest
+
+import oracle
+from helpers import (MAX_ABS_TOL, REL_L2_TOL, bf16_to_f32, check_output, check_routing, oracle_layer, oracle_partial, to_dev)
+from paper_2508_17624_b200 import binding, ep, workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,R,n_tokens", [("c0", 2, None), ("c0", 4, 33), ("c0", 16, 100), ("c1", 2, None), ("c1", 8, None),
+                                             ("c1", 2, 3000)])
+def test_emulated_ranks_against_the_oracle(name, R, n_tokens):
+    import torch
+    cfg = wl.CONFIGS[name]
+    n = n_tokens or cfg.n_tokens
+    bank = wl.NoiseBank(cfg.seed)
+    x, aid = wl.gen_tokens(cfg, 0, n), wl.gen_adapter_ids(cfg, n)
+    xd, ad = to_dev(x), to_dev(aid)
+    # the routing of the batch, from a pool without expert parallelism, checked against the oracle
+    single = binding.Pool.from_config(cfg, max_tokens=n)
+    tuned, bases = binding.load_model(single, cfg, bank)
+    olayer = oracle_layer(cfg, 0, bank, tuned, base=bases[0])
+    r1 = single.moe_forward_debug(0, xd, ad)
+    torch.cuda.synchronize()
+    ids, w, slots, _ = check_routing(cfg, olayer, x, aid, r1)
+    whole = single.moe_forward_partial(0, xd, ad)       # without expert parallelism: the whole layer, unrounded
+    torch.cuda.synchronize()
+    assert torch.equal(single.ep_finish(whole), r1["out"])
+    s1 = single.stats()
+    single.destroy()
+
+    pools, partials, pages, kernels = [], [], 0, set()
+    for r in range(R):
+        pool = binding.Pool.from_config(cfg, max_tokens=n, ep_size=R, ep_rank=r)
+        binding.load_model(pool, cfg, bank)
+        with pytest.raises(binding.EwError):
+            pool.moe_forward(0, xd, ad)                 # a rank alone has no layer output
+        part = pool.moe_forward_partial(0, xd, ad)
+        torch.cuda.synchronize()
+        assert pool.last_device_error() == 0
+        want = oracle_partial(cfg, 0, bank, tuned, x, ids, slots, w, R, r, base=bases[0])
+        got = part.cpu().numpy()
+        scale = max(float(np.linalg.norm(want)), 1e-30)
+        assert float(np.linalg.norm(got - want)) / scale <= REL_L2_TOL, f"rank {r}"
+        assert float(np.abs(got - want).max()) <= MAX_ABS_TOL, f"rank {r}"
+        again = pool.moe_forward_partial(0, xd, ad)     # back to back: same bits
+        torch.cuda.synchronize()
+        assert torch.equal(again, part)
+        st = pool.stats()
+        pages += st["pages_mapped"]
+        kernels.add(st["last_forward_kernels"])
+        pools.append(pool)
+        partials.append(part)
+    # what the all-reduce does: the fp32 sum over ranks, then the layer's single rounding
+    summed = partials[0].clone()
+    for part in partials[1:]:
+        summed += part
+    out = pools[0].ep_finish(summed)
+    torch.cuda.synchronize()
+    check_output(olayer, x, slots, w, bf16_to_f32(out))
+    # against the unsharded forward only the order of the fp32 additions differs
+    a, b = bf16_to_f32(out), bf16_to_f32(r1["out"])
+    assert np.abs(a - b).max() <= 2.0 ** -7 * max(np.abs(b).max(), 1e-30)
+    assert (a != b).mean() < 0.05
+    # memory: the ranks together back what the single pool backs (page rounding at the blocks' edges aside)
+    assert s1["pages_mapped"] <= pages <= s1["pages_mapped"] + 4 * R * (cfg.max_adapters + 2)
+    assert kernels <= {4, 5, 7}
+    if n >= 3000:
+        assert kernels == {7}                           # prefill-sized: planning kernel and both GEMM kernels per GEMM
+    for pool in pools:
+        pool.destroy()
+
+
+def test_expert_parallel_layer_single_rank_on_gpu():
+    """ExpertParallelLayer without a process group is the plain forward."""
+    import torch
+    cfg = wl.CONFIGS["c0"]
+    bank = wl.NoiseBank(cfg.seed)
+    pool = binding.Pool.from_config(cfg)
+    binding.load_model(pool, cfg, bank)
+    x, aid = to_dev(wl.gen_tokens(cfg)), to_dev(wl.gen_adapter_ids(cfg))
+    out = ep.ExpertParallelLayer(pool).forward(0, x, aid)
+    torch.cuda.synchronize()
+    assert torch.equal(out, pool.moe_forward(0, x, aid))
+    pool.destroy()

@@ -7,8 +7,8 @@
 // (3-D descriptors ordered element, row, atom: shared memory receives one swizzled tile per atom).  Only the first
 // `tok_tile` rows of the 128-row MMA tile are loaded; the other rows hold whatever shared memory held
 // and feed accumulator lanes nobody reads.  TMEM lane i belongs to token i.  With 32-token tiles (small
-// batches) one warp spills the logits to shared memory and four threads share each token's softmax and
-// top-k (see the epilogue); with larger tiles every epilogue
+// batches) one warp spills the logits to shared memory and four adjacent lanes share each token's softmax and
+// top-k (quad_epilogue); with larger tiles every epilogue
 // thread owns one token: it reads its M logits from TMEM, forms the softmax probabilities in fp32, takes
 // k arg-max rounds (probability descending, lower index on ties), looks each chosen expert up in the
 // layer's expert map Pi (staged in shared memory) under the token's adapter id, and bumps the slot's
@@ -101,6 +101,114 @@ __device__ __forceinline__ void emit_ranks(const RouterArgs &A, int t, const int
                     A.slot_tok[(size_t)(r0 == 0 ? sl[u] : A.slot_ids[(size_t)t * A.k + r0 + u]) * A.B + got[u]] = t;
             }
     }
+}
+
+// Softmax, top-k, rerouting and histogram of one 32-token tile whose logits lie in shared memory (expert-major,
+// lg_s[j * 32 + token]), by the four epilogue warps: four adjacent lanes share a token, lane q of them owning the
+// experts [q E, q E + E).  Each lane sorts its probabilities once (a 63-comparator network of max/min pairs, values
+// only); the k rounds then look at the four lanes' heads alone - two shuffles for the maximum, a ballot for the
+// lowest lane that holds it (lower expert index on ties), a pop; the expert index of a value is looked up afterwards,
+// only for the values the lane contributed (lowest index with that value not taken yet, so ties inside a lane also go
+// to the lower index).  No shared-memory exchange and no barrier between the rounds.  KD: how many of a lane's sorted
+// values can be popped (8 for k <= 8, else 16).
+template <int KD>
+__device__ __forceinline__ void quad_epilogue(const RouterArgs &A, const float *lg_s, const int32_t *pi_s, int tok0, int E, int a) {
+    constexpr unsigned kFull = 0xffffffffu;
+    const int tid2 = (int)threadIdx.x - 64;                          // 0..127 over the four epilogue warps
+    const int tl = tid2 >> 2, q = tid2 & 3;                          // token inside the tile, quarter of the experts
+    const int t = tok0 + tl, M = A.M, k = A.k;
+    const unsigned group_shift = threadIdx.x & 28;                   // first lane of this token's four within the warp
+    const bool live = t < A.B;
+    float e[16];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const int j = q * E + i;
+        e[i] = (i < E && j < M) ? lg_s[j * 32 + tl] : -INFINITY;
+        mx = fmaxf(mx, e[i]);
+    }
+    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 2));
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {                                   // exp(-inf) = 0 for the absent experts
+        e[i] = expf(e[i] - mx);
+        sum += e[i];
+    }
+    sum += __shfl_xor_sync(kFull, sum, 1);
+    sum += __shfl_xor_sync(kFull, sum, 2);
+    const float inv_sum = 1.f / sum;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) e[i] = (i < E && q * E + i < M) ? e[i] * inv_sum : -1.f;   // absent experts below every real one
+
+    float s0[16];                                                    // the lane's probabilities sorted descending
+#pragma unroll
+    for (int i = 0; i < 16; ++i) s0[i] = e[i];
+#define EW_CE(x, y) { const float hi_ = fmaxf(s0[x], s0[y]), lo_ = fminf(s0[x], s0[y]); s0[x] = hi_; s0[y] = lo_; }
+    EW_CE(0, 1) EW_CE(2, 3) EW_CE(0, 2) EW_CE(1, 3) EW_CE(1, 2) EW_CE(4, 5) EW_CE(6, 7) EW_CE(4, 6) EW_CE(5, 7)
+    EW_CE(5, 6) EW_CE(0, 4) EW_CE(2, 6) EW_CE(2, 4) EW_CE(1, 5) EW_CE(3, 7) EW_CE(3, 5) EW_CE(1, 2) EW_CE(3, 4)
+    EW_CE(5, 6) EW_CE(8, 9) EW_CE(10, 11) EW_CE(8, 10) EW_CE(9, 11) EW_CE(9, 10) EW_CE(12, 13) EW_CE(14, 15)
+    EW_CE(12, 14) EW_CE(13, 15) EW_CE(13, 14) EW_CE(8, 12) EW_CE(10, 14) EW_CE(10, 12) EW_CE(9, 13) EW_CE(11, 15)
+    EW_CE(11, 13) EW_CE(9, 10) EW_CE(11, 12) EW_CE(13, 14) EW_CE(0, 8) EW_CE(4, 12) EW_CE(4, 8) EW_CE(2, 10)
+    EW_CE(6, 14) EW_CE(6, 10) EW_CE(2, 4) EW_CE(6, 8) EW_CE(10, 12) EW_CE(1, 9) EW_CE(5, 13) EW_CE(5, 9)
+    EW_CE(3, 11) EW_CE(7, 15) EW_CE(7, 11) EW_CE(3, 5) EW_CE(7, 9) EW_CE(11, 13) EW_CE(1, 2) EW_CE(3, 4)
+    EW_CE(5, 6) EW_CE(7, 8) EW_CE(9, 10) EW_CE(11, 12) EW_CE(13, 14)
+#undef EW_CE
+    float s[KD];                                                     // the part of it that is popped during the rounds
+#pragma unroll
+    for (int i = 0; i < KD; ++i) s[i] = s0[i];
+    unsigned won = 0;                                                // bit r: this lane's head won round r
+    float wsum = 0.f;
+    for (int r = 0; r < k; ++r) {
+        float wv = s[0];
+        wv = fmaxf(wv, __shfl_xor_sync(kFull, wv, 1));
+        wv = fmaxf(wv, __shfl_xor_sync(kFull, wv, 2));
+        const unsigned holders = (__ballot_sync(kFull, s[0] == wv) >> group_shift) & 0xfu;
+        wsum += wv;
+        if (q == __ffs(holders) - 1) {                               // the lowest lane that holds it pops its head
+            won |= 1u << r;
+#pragma unroll
+            for (int i = 0; i < KD - 1; ++i) s[i] = s[i + 1];
+            s[KD - 1] = -2.f;
+        }
+    }
+    // this lane's wins, in round order, are s0[0], s0[1], ...: outputs first, all histogram atomics in flight together
+    // (the value returned is the pair's position inside its slot's chunk), then the positions
+    unsigned taken = 0;
+    int p_slot[KD], p_r[KD], got[KD];                                // pending pairs: slot (-1: another rank's, -2: none), round
+#pragma unroll
+    for (int j = 0; j < KD; ++j) {
+        p_slot[j] = -2;
+        p_r[j] = 0;
+        if (won && live) {
+            const int r = __ffs(won) - 1;
+            won &= won - 1;
+            const float wv = s0[j];
+            unsigned eq = 0;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) eq |= (e[i] == wv) ? (1u << i) : 0u;
+            const int idx = __ffs(eq & ~taken) - 1;                  // lowest index with that value not taken yet
+            taken |= 1u << idx;
+            const int id = q * E + idx;
+            const int slot = a < 0 ? id : (A.pi_in_smem ? pi_s[a * M + id] : __ldg(A.pi + a * M + id));
+            const size_t o = (size_t)t * k + r;
+            float w = wv;
+            if (A.renormalize) w = w / wsum;
+            A.topk_ids[o] = id;
+            A.slot_ids[o] = slot;
+            A.topk_w[o] = (A.renormalize || A.scale != 1.f) ? w * A.scale : w;
+            p_slot[j] = (id >= A.own_lo && id < A.own_hi) ? slot : -1;      // expert parallelism: another rank's pair is not counted
+            p_r[j] = r;
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < KD; ++j) got[j] = p_slot[j] >= 0 ? atomicAdd(A.counts + p_slot[j], 1) : -1;
+#pragma unroll
+    for (int j = 0; j < KD; ++j)
+        if (p_slot[j] >= -1) {
+            A.rank[(size_t)t * k + p_r[j]] = got[j];
+            if (A.slot_tok && got[j] >= 0 && got[j] < A.B) A.slot_tok[(size_t)p_slot[j] * A.B + got[j]] = t;
+        }
 }
 
 // REG = true: M <= 64, the token's probabilities stay in registers
@@ -199,20 +307,17 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
     } else if (REG && tok_tile == 32) {
         // epilogue for 32-token tiles (small batches, where this kernel's latency is exposed): the logits sit in
         // TMEM lanes 0..31 only, which one warp can read; that warp spills them to shared memory and then all four
-        // epilogue warps work on them, four threads per token, each owning a quarter of the experts: partial max
-        // and partial sum for the softmax, then k rounds of "publish my best remaining candidate, everybody picks
-        // the best of the token's four" (value descending, lower expert index on ties).
-        const int g = warp & 3;                                      // expert group of this thread
-        const int E = n_mma >> 2;                                    // experts per group (4, 8, 12 or 16)
-        const int t = tok0 + lane;
+        // epilogue warps work on them, four threads per token, each owning a quarter of the experts (quad_epilogue).
+        const int g = warp & 3;                                      // g == 0: the warp that reads TMEM
+        const int E = n_mma >> 2;                                    // experts per quarter (4, 8, 12 or 16)
         const int k = A.k;
         auto quad_sync = [] { asm volatile("bar.sync 1, 128;" ::: "memory"); };   // the four epilogue warps
+        // the adapter id of this thread's token (quad_epilogue's mapping), fetched while the logits are still being computed
+        const int t_mine = tok0 + (((int)threadIdx.x - 64) >> 2);
+        const int a_mine = (krank == 0 && t_mine < A.B) ? checked_aid(A.aid[t_mine], A.N, A.loaded, A.err) : -1;
         mbar_wait(bar_done, 0, abort_flag, A.err);
         quad_sync();                                                 // every epilogue thread is past its (bounded) wait
         float *lg_s = reinterpret_cast<float *>(smem_al);            // [n_mma][32] logits, expert-major (the ring has drained)
-        float *red_s = lg_s + 64 * 32;                               // [2][4][32] partial max, partial sum
-        float *cv_s = red_s + 2 * 4 * 32;                            // [2][4][32] candidate values, double-buffered by round
-        int *ci_s = reinterpret_cast<int *>(cv_s + 2 * 4 * 32);      // [2][4][32] candidate expert ids
         float *part_s = reinterpret_cast<float *>(smem_al + A.part_off);   // K split: [cs][n_mma][32] partial logits (CTA 0's is used)
         if (!*abort_flag && g == 0) {
             tc_fence_after();
@@ -249,91 +354,8 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
         }
         quad_sync();
         if (!*abort_flag && krank == 0) {
-            float p[16];
-            float mx = -INFINITY;
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int j = g * E + i;
-                p[i] = (i < E && j < M) ? lg_s[j * 32 + lane] : -INFINITY;
-                mx = fmaxf(mx, p[i]);
-            }
-            red_s[g * 32 + lane] = mx;
-            quad_sync();
-            mx = fmaxf(fmaxf(red_s[lane], red_s[32 + lane]), fmaxf(red_s[64 + lane], red_s[96 + lane]));
-            float sum = 0.f;
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {                           // exp(-inf) = 0 for the absent experts
-                p[i] = expf(p[i] - mx);
-                sum += p[i];
-            }
-            red_s[128 + g * 32 + lane] = sum;
-            quad_sync();
-            sum = ((red_s[128 + lane] + red_s[160 + lane]) + red_s[192 + lane]) + red_s[224 + lane];
-            const float inv_sum = 1.f / sum;
-#pragma unroll
-            for (int i = 0; i < 16; ++i) p[i] = (i < E && g * E + i < M) ? p[i] * inv_sum : -1.f;
-            const int a = t < A.B ? checked_aid(A.aid[t], A.N, A.loaded, A.err) : -1;
-            float wsum = 0.f;
-            float my_w[8];                                           // weights and slots of the pairs this thread writes (r = g, g+4, ...)
-            int my_slot[8];
-            uint32_t my_local = 0;                                   // bit u: pair g + 4u belongs to this rank (expert parallelism)
-            for (int r = 0; r < k; ++r) {
-                float bv = -1.f;
-                int bi = 0;
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {                       // branch-free selects; strict >: the lower index keeps a tie
-                    const bool gt = p[i] > bv;
-                    bv = gt ? p[i] : bv;
-                    bi = gt ? i : bi;
-                }
-                const int buf = (r & 1) * 128;
-                cv_s[buf + g * 32 + lane] = bv;
-                ci_s[buf + g * 32 + lane] = g * E + bi;
-                quad_sync();
-                float wv = cv_s[buf + lane];
-                int wg = 0;
-#pragma unroll
-                for (int q = 1; q < 4; ++q) {                        // groups in ascending expert order: strict > keeps the lower index
-                    const float c = cv_s[buf + q * 32 + lane];
-                    const bool gt = c > wv;
-                    wv = gt ? c : wv;
-                    wg = gt ? q : wg;
-                }
-                const int wi = ci_s[buf + wg * 32 + lane];
-                if (wg == g) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) p[i] = (i == bi) ? -1.f : p[i];   // taken (probabilities are >= 0)
-                }
-                wsum += wv;
-                if ((r & 3) == g && t < A.B) {                       // the token's four threads share the output work
-                    const int slot = a < 0 ? wi : (A.pi_in_smem ? pi_s[a * M + wi] : __ldg(A.pi + a * M + wi));
-                    const size_t o = (size_t)t * k + r;
-                    A.topk_ids[o] = wi;
-                    A.slot_ids[o] = slot;
-#pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        if (u == (r >> 2)) { my_w[u] = wv; my_slot[u] = slot; }
-                    if (wi >= A.own_lo && wi < A.own_hi) my_local |= 1u << (r >> 2);
-                }
-            }
-            if (t < A.B) {
-                // per-slot histogram: one atomic per pair, all of this thread's in flight together; the value
-                // returned is the pair's position inside its slot's chunk
-                int got[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u)
-                    if (g + 4 * u < k) got[u] = ((my_local >> u) & 1u) ? atomicAdd(A.counts + my_slot[u], 1) : -1;
-#pragma unroll
-                for (int u = 0; u < 8; ++u)
-                    if (g + 4 * u < k) {
-                        const size_t o = (size_t)t * k + g + 4 * u;
-                        float w = my_w[u];
-                        if (A.renormalize) w = w / wsum;
-                        A.topk_w[o] = (A.renormalize || A.scale != 1.f) ? w * A.scale : w;
-                        A.rank[o] = got[u];
-                        if (A.slot_tok && got[u] >= 0 && got[u] < A.B) A.slot_tok[(size_t)my_slot[u] * A.B + got[u]] = t;
-                    }
-            }
+            if (k <= 8) quad_epilogue<8>(A, lg_s, pi_s, tok0, E, a_mine);
+            else quad_epilogue<16>(A, lg_s, pi_s, tok0, E, a_mine);
         }
     } else {
         // epilogue: thread <-> token

@@ -675,7 +675,19 @@ def check_shape(shape, renorm, seed):
     ids, w, slots, flips = check_routing(cfg, olayer, x, aid, r, weight_rtol=WEIGHT_RTOL * max(1.0, x_scale))
     assert flips <= max(2, cfg.n_tokens // 20)
     check_output(olayer, x, slots, w, bf16_to_f32(r["out"]))
+    kernels = pool.stats()["last_forward_kernels"]
     pool.destroy()
+    return kernels
+
+
+def test_kernels_per_forward_and_the_planning_fallback():
+    """Which form of the forward ran is reported by the pool: four kernels for a decode-sized batch (the GEMM kernels
+    derive their own work items), seven for a prefill-sized one (planning kernel, two kernels per GEMM), and five - the
+    planning kernel kept - for a decode-sized batch whose items a GEMM CTA could not hold in its shared memory: here
+    704 slots x 32 weight tiles of GEMM-2 are up to 170 items per CTA.  Each against the oracle."""
+    assert check_shape(dict(hidden=128, inter=200, num_experts=40, num_shared=1, top_k=5, max_adapters=3, e_max=4, n_tokens=77), 0, 5) == 4
+    assert check_shape(dict(hidden=192, inter=72, num_experts=4, num_shared=0, top_k=4, max_adapters=2, e_max=4, n_tokens=1500), 0, 5) == 7
+    assert check_shape(dict(hidden=4096, inter=64, num_experts=64, num_shared=2, top_k=8, max_adapters=20, e_max=32, n_tokens=1024), 0, 5) == 5
 
 
 def test_c3_stack_throughput_report():

@@ -30,6 +30,7 @@ namespace {
 using namespace tc;
 
 constexpr int kThreads = 192;
+constexpr int kThreadsBig = 320;     // large tiles: eight epilogue warps, so that 64 tokens are selected in one pass
 constexpr int kTileRows = 128;
 constexpr int kMaxStages = 16;
 constexpr int kMaxAtoms = 4;         // 64-element K-atoms per TMA box and pipeline stage: 4, 2 or 1
@@ -59,6 +60,8 @@ struct RouterArgs {
     int B, H, M, k, N, renormalize;
     float scale;
     int stages, tmem_cols, pi_in_smem, tok_tile, atoms;
+    int big_quad;          // 64- and 128-token tiles: four lanes per token and a histogram per CTA (needs room in the drained ring)
+    int P;                 // slots of the pool (size of the counters)
     int ksplit;            // CTAs per cluster that share one token tile, each with 1/ksplit of K (1: no cluster)
     int part_off;          // byte offset of the partial-logit buffer [ksplit][n_mma][32] floats in shared memory
     int32_t *topk_ids;
@@ -111,11 +114,17 @@ __device__ __forceinline__ void emit_ranks(const RouterArgs &A, int t, const int
 // only for the values the lane contributed (lowest index with that value not taken yet, so ties inside a lane also go
 // to the lower index).  No shared-memory exchange and no barrier between the rounds.  KD: how many of a lane's sorted
 // values can be popped (8 for k <= 8, else 16).
+//
+// lg_s[j * stride + token]; this call handles the tile's tokens tl_base .. tl_base + 31.  hist_s null: the pairs are
+// counted in the global counters right away (the value returned is the pair's position in its slot).  Otherwise (large
+// batches, where thousands of pairs per slot would queue up at one counter) they are counted in the CTA's own
+// histogram, the position inside the CTA is stored, and the caller adds the CTA's base per slot afterwards.
 template <int KD>
-__device__ __forceinline__ void quad_epilogue(const RouterArgs &A, const float *lg_s, const int32_t *pi_s, int tok0, int E, int a) {
+__device__ __forceinline__ void quad_epilogue(const RouterArgs &A, const float *lg_s, int stride, int tl_base, const int32_t *pi_s,
+                                              int tok0, int E, int a, int32_t *hist_s) {
     constexpr unsigned kFull = 0xffffffffu;
     const int tid2 = (int)threadIdx.x - 64;                          // 0..127 over the four epilogue warps
-    const int tl = tid2 >> 2, q = tid2 & 3;                          // token inside the tile, quarter of the experts
+    const int tl = tl_base + (tid2 >> 2), q = tid2 & 3;              // token inside the tile, quarter of the experts
     const int t = tok0 + tl, M = A.M, k = A.k;
     const unsigned group_shift = threadIdx.x & 28;                   // first lane of this token's four within the warp
     const bool live = t < A.B;
@@ -124,7 +133,7 @@ __device__ __forceinline__ void quad_epilogue(const RouterArgs &A, const float *
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
         const int j = q * E + i;
-        e[i] = (i < E && j < M) ? lg_s[j * 32 + tl] : -INFINITY;
+        e[i] = (i < E && j < M) ? lg_s[j * stride + tl] : -INFINITY;
         mx = fmaxf(mx, e[i]);
     }
     mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 1));
@@ -202,18 +211,18 @@ __device__ __forceinline__ void quad_epilogue(const RouterArgs &A, const float *
         }
     }
 #pragma unroll
-    for (int j = 0; j < KD; ++j) got[j] = p_slot[j] >= 0 ? atomicAdd(A.counts + p_slot[j], 1) : -1;
+    for (int j = 0; j < KD; ++j) got[j] = p_slot[j] >= 0 ? atomicAdd((hist_s ? hist_s : A.counts) + p_slot[j], 1) : -1;
 #pragma unroll
     for (int j = 0; j < KD; ++j)
         if (p_slot[j] >= -1) {
             A.rank[(size_t)t * k + p_r[j]] = got[j];
-            if (A.slot_tok && got[j] >= 0 && got[j] < A.B) A.slot_tok[(size_t)p_slot[j] * A.B + got[j]] = t;
+            if (!hist_s && A.slot_tok && got[j] >= 0 && got[j] < A.B) A.slot_tok[(size_t)p_slot[j] * A.B + got[j]] = t;
         }
 }
 
 // REG = true: M <= 64, the token's probabilities stay in registers
 template <bool REG>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsBig, 1)
 router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_r, const RouterArgs A) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -261,7 +270,7 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (A.pi_in_smem)
-        for (int i = threadIdx.x; i < A.N * M; i += kThreads) pi_s[i] = A.pi[i];
+        for (int i = threadIdx.x; i < A.N * M; i += blockDim.x) pi_s[i] = A.pi[i];
     pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
@@ -354,8 +363,79 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
         }
         quad_sync();
         if (!*abort_flag && krank == 0) {
-            if (k <= 8) quad_epilogue<8>(A, lg_s, pi_s, tok0, E, a_mine);
-            else quad_epilogue<16>(A, lg_s, pi_s, tok0, E, a_mine);
+            if (k <= 8) quad_epilogue<8>(A, lg_s, 32, 0, pi_s, tok0, E, a_mine, nullptr);
+            else quad_epilogue<16>(A, lg_s, 32, 0, pi_s, tok0, E, a_mine, nullptr);
+        }
+    } else if (REG && A.big_quad) {
+        // epilogue for 64- and 128-token tiles (large batches): the warps that own TMEM lanes with tokens spill the
+        // logits to shared memory (the ring has drained), then eight warps go through the tile 64 tokens at a time
+        // with four lanes per token (quad_epilogue; one warp works through its eight tokens' selection in ~9 us of
+        // dependent instructions, so the passes are spread over warps rather than run one after the other).  The pairs are counted in a histogram of the CTA; afterwards one
+        // atomic per live slot fetches the CTA's base in the global counter, and a sweep over the tile's pairs turns the
+        // positions inside the CTA into positions inside the slot.  (Counting every pair in the global counters
+        // directly took 10-17 us of an 8192-token batch: some 700 returning atomics queue up per base expert.)
+        const int lgp = warp & 3;
+        const int E = n_mma >> 2;
+        const int k = A.k;
+        const int tid2 = (int)threadIdx.x - 64;
+        auto quad_sync = [] { asm volatile("bar.sync 1, 256;" ::: "memory"); };   // the eight epilogue warps (320 threads per CTA in this mode)
+        constexpr int kEpi = kThreadsBig - 64;
+        float *lg_s = reinterpret_cast<float *>(smem_al);            // [n_mma][tok_tile] logits, expert-major
+        int32_t *hist_s = reinterpret_cast<int32_t *>(lg_s + 64 * tok_tile);      // [P] pairs of this CTA per slot, then the CTA's base
+        int32_t *aid_s = hist_s + A.P;                               // [tok_tile] checked adapter ids
+        const int P = A.P;
+        // adapter ids of the tile's tokens, fetched while the logits are still being computed (kept in registers until
+        // the ring has drained)
+        const int a_reg = (tid2 < tok_tile && tok0 + tid2 < A.B) ? checked_aid(A.aid[tok0 + tid2], A.N, A.loaded, A.err) : -1;
+        mbar_wait(bar_done, 0, abort_flag, A.err);
+        quad_sync();                                                 // every epilogue thread is past its (bounded) wait
+        const bool go = !*abort_flag;
+        if (go) {
+            for (int i = tid2; i < P; i += kEpi) hist_s[i] = 0;
+            if (tid2 < tok_tile) aid_s[tid2] = a_reg;
+            if (warp < 6 && lgp * 32 < tok_tile) {                  // warps 2..5 own the four TMEM lane groups
+                tc_fence_after();
+                const uint32_t t0 = tmem_base + ((uint32_t)(lgp * 32) << 16);
+                uint32_t v0[32], v1[32];
+                if (n_mma >= 32) tc_ld32(t0, v0); else tc_ld16(t0, v0);
+                if (n_mma > 32) { if (n_mma - 32 >= 32) tc_ld32(t0 + 32, v1); else tc_ld16(t0 + 32, v1); }
+                tc_wait_ld();
+                float *col = lg_s + lgp * 32 + lane;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    if (j < n_mma) col[j * tok_tile] = __uint_as_float(v0[j]);
+                    if (32 + j < n_mma) col[(32 + j) * tok_tile] = __uint_as_float(v1[j]);
+                }
+            }
+        }
+        quad_sync();
+        if (go) {
+#pragma unroll 1
+            for (int tb = 0; tb < tok_tile; tb += 64) {           // 256 threads: 64 tokens per pass
+                const int a = aid_s[tb + (tid2 >> 2)];
+                if (k <= 8) quad_epilogue<8>(A, lg_s, tok_tile, tb, pi_s, tok0, E, a, hist_s);
+                else quad_epilogue<16>(A, lg_s, tok_tile, tb, pi_s, tok0, E, a, hist_s);
+            }
+        }
+        quad_sync();
+        if (go)
+            for (int i = tid2; i < P; i += kEpi) {
+                const int c = hist_s[i];
+                if (c) hist_s[i] = atomicAdd(A.counts + i, c);        // the CTA's first position in slot i
+            }
+        quad_sync();
+        if (go) {
+            const int n_q = min(tok_tile, A.B - tok0) * k;
+            for (int qq = tid2; qq < n_q; qq += kEpi) {
+                const size_t o = (size_t)tok0 * k + qq;
+                int r = *reinterpret_cast<volatile int32_t *>(A.rank + o);
+                if (r >= 0) {                                         // (-1: another rank's pair, expert parallelism)
+                    const int slot = *reinterpret_cast<volatile int32_t *>(A.slot_ids + o);
+                    r += hist_s[slot];
+                    A.rank[o] = r;
+                    if (A.slot_tok && r < A.B) A.slot_tok[(size_t)slot * A.B + r] = tok0 + qq / k;
+                }
+            }
         }
     } else {
         // epilogue: thread <-> token
@@ -486,7 +566,7 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
 
 // Launch geometry of the router kernel for a batch of B tokens: tokens per CTA, K-atoms per stage, ring depth.
 struct RouterGeometry {
-    int tok_tile, atoms, stages, pi_in_smem, tmem_cols, grid, ksplit, part_off;
+    int tok_tile, atoms, stages, pi_in_smem, tmem_cols, grid, ksplit, part_off, big_quad;
     bool reg;
     size_t smem;
 };
@@ -529,6 +609,9 @@ static bool router_geometry(const ew_pool *p, int B, RouterGeometry *g) {
             g->atoms = atoms;
             g->stages = stages;
             g->part_off = (int)(((size_t)stages * stage_bytes + fixed + 15) & ~(size_t)15);
+            // the large-tile epilogue keeps logits, a histogram over the slots and the tile's adapter ids in the drained ring
+            g->big_quad = g->reg && g->tok_tile >= 64 &&
+                          (size_t)stages * stage_bytes >= ((size_t)64 * g->tok_tile + p->P + g->tok_tile) * 4;
             g->smem = (size_t)stages * stage_bytes + tail;
             g->tmem_cols = n_mma <= 32 ? 32 : n_mma <= 64 ? 64 : n_mma <= 128 ? 128 : 256;
             g->grid = tiles * g->ksplit;
@@ -548,10 +631,10 @@ static int router_launch(ew_pool *p, int layer, const void *x, const RouterGeome
     A.H = c.hidden; A.M = c.num_experts; A.k = c.top_k; A.N = c.max_adapters; A.renormalize = c.renormalize;
     A.scale = c.routed_scale;
     A.stages = g.stages; A.tmem_cols = g.tmem_cols; A.pi_in_smem = g.pi_in_smem; A.tok_tile = g.tok_tile; A.atoms = g.atoms;
-    A.ksplit = g.ksplit; A.part_off = g.part_off;
+    A.ksplit = g.ksplit; A.part_off = g.part_off; A.big_quad = g.big_quad; A.P = p->P;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(g.grid);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(g.big_quad ? kThreadsBig : kThreads);
     cfg.dynamicSmemBytes = g.smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];

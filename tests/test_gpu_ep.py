@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("name,R,n_tokens", [("c0", 2, None), ("c0", 4, 33), ("c0", 16, 100), ("c1", 2, None), ("c1", 8, None),
-                                             ("c1", 2, 3000)])
+                                             ("c1", 2, 3000), ("c0", 2, 6000), ("c0", 4, 12000)])
 def test_emulated_ranks_against_the_oracle(name, R, n_tokens):
     import torch
     cfg = wl.CONFIGS[name]

@@ -68,6 +68,26 @@ def test_route_noalloc_matches_forward_twice_in_a_row(name):
     pool.destroy()
 
 
+@pytest.mark.parametrize("n", [6000, 10000])
+def test_route_noalloc_large_batches(n):
+    """Batches beyond 4736 tokens take the router's large-tile form (64- and 128-token tiles, a histogram per CTA whose
+    bases come from the caller's counters): ids, weights, slot ids and counts against the oracle."""
+    import torch
+    cfg = wl.CONFIGS["c0"]
+    assert n * cfg.top_k <= 65536
+    bank = wl.NoiseBank(cfg.seed)
+    pool = binding.Pool.from_config(cfg)
+    tuned, bases = binding.load_model(pool, cfg, bank)
+    olayer = oracle_layer(cfg, 0, bank, tuned, base=bases[0])
+    x_bits, aid_np = wl.gen_tokens(cfg, 0, n), wl.gen_adapter_ids(cfg, n)
+    ids, w, slots, counts, status = _route(pool, cfg, to_dev(x_bits), to_dev(aid_np), n)
+    assert status == 0
+    _, _, _, flips = check_routing(cfg, olayer, x_bits, aid_np, dict(topk_ids=ids, topk_w=w, slot_ids=slots, counts=counts))
+    assert flips <= max(4, n // 500)
+    assert counts.sum() == n * cfg.top_k
+    pool.destroy()
+
+
 def test_route_noalloc_rejects_sizes_beyond_the_array():
     import torch
     cfg = wl.CONFIGS["c0"]

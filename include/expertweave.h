@@ -200,6 +200,20 @@ ew_status_t ew_moe_forward_partial(ew_pool_t *pool, int32_t layer, const void *x
                                    int32_t n_tokens, float *partial, void *cuda_stream);
 ew_status_t ew_ep_finish(ew_pool_t *pool, const float *summed, int32_t n_tokens, void *out, void *cuda_stream);
 
+/* The same exchange done by the kernel that produces the data (Section 5.1's deployment; the fused form of the step
+ * above).  ew_moe_forward_scatter runs the partial forward and its last kernel stores the rank's partial sums straight
+ * into every rank's gather buffer: gather_bufs is a DEVICE array of ep_size pointers, gather_bufs[r'] = rank r''s
+ * buffer, fp32 [ep_size, n_tokens, H], 16-byte aligned, of which this call fills block ep_rank.  The buffers of the
+ * other ranks must be device memory this GPU can store to (peer access, an imported allocation, symmetric memory);
+ * plain stores only, nothing is loaded from a peer.  When the scatter calls of ALL ranks for this step have completed
+ * (a barrier between the ranks that the caller provides, ordered on the stream), ew_ep_finish_gathered adds the
+ * ep_size blocks of this rank's own buffer in rank order and rounds once: the same bits on every rank and in every
+ * run, whatever the interconnect did.  It serves an all-gather of the ew_moe_forward_partial results just as well.
+ * gathered: DEVICE fp32 [ep_size, n_tokens, H]; out: DEVICE bf16 [n_tokens, H].  Errors as for ew_moe_forward. */
+ew_status_t ew_moe_forward_scatter(ew_pool_t *pool, int32_t layer, const void *x, const int32_t *adapter_ids,
+                                   int32_t n_tokens, float *const *gather_bufs, void *cuda_stream);
+ew_status_t ew_ep_finish_gathered(ew_pool_t *pool, const float *gathered, int32_t n_tokens, void *out, void *cuda_stream);
+
 /* Same forward with HOST buffers, pipelined across calls: x and adapter_ids are uploaded to device staging
  * owned by the pool, the forward runs on them and the result is downloaded to out_host.  Upload, kernels and
  * download run on three streams of the pool with double-buffered staging, so that, with page-locked host

@@ -23,7 +23,7 @@ STATUS_NAMES = ["EW_OK", "EW_ERR_INVALID_ARG", "EW_ERR_OOM", "EW_ERR_SLOT_IN_USE
 EXPORTS = ["ew_pool_create", "ew_pool_destroy", "ew_load_base", "ew_load_adapter", "ew_unload_adapter",
            "ew_pool_trim", "ew_moe_forward", "ew_moe_forward_debug", "ew_moe_forward_host", "ew_profile_enable",
            "ew_profile_read", "ew_reroute", "ew_reroute_unfused", "ew_route_logits", "ew_route_noalloc", "ew_selftest_bounded_wait", "ew_get_expert_map",
-           "ew_moe_forward_partial", "ew_ep_finish", "ew_pool_stats", "ew_last_device_error", "ew_slot_address", "ew_status_str", "ew_last_error_string"]
+           "ew_moe_forward_partial", "ew_ep_finish", "ew_moe_forward_scatter", "ew_ep_finish_gathered", "ew_pool_stats", "ew_last_device_error", "ew_slot_address", "ew_status_str", "ew_last_error_string"]
 
 
 class EwConfig(C.Structure):
@@ -171,6 +171,20 @@ class Pool:
         if out is None:
             out = torch.empty(summed.shape, dtype=torch.bfloat16, device=summed.device)
         _check(lib().ew_ep_finish(self._h, _dp(summed), summed.shape[0], _dp(out), _stream()), "ew_ep_finish")
+        return out
+
+    def moe_forward_scatter(self, layer, x, adapter_ids, gather_ptrs):
+        """Partial forward whose last kernel stores the partial sums into every rank's gather buffer; `gather_ptrs`:
+        device int64 tensor with the ep_size buffer addresses (see the header)."""
+        _check(lib().ew_moe_forward_scatter(self._h, layer, _dp(x), _dp(adapter_ids), x.shape[0], _dp(gather_ptrs), _stream()),
+               "ew_moe_forward_scatter")
+
+    def ep_finish_gathered(self, gathered, out=None):
+        """bf16 result from this rank's gather buffer [ep_size, n_tokens, H] (blocks added in rank order)."""
+        import torch
+        if out is None:
+            out = torch.empty(gathered.shape[1:], dtype=torch.bfloat16, device=gathered.device)
+        _check(lib().ew_ep_finish_gathered(self._h, _dp(gathered), gathered.shape[1], _dp(out), _stream()), "ew_ep_finish_gathered")
         return out
 
     def moe_forward_debug(self, layer, x, adapter_ids):

@@ -160,8 +160,10 @@ int launch_gemm1(ew_pool *p, int layer, const CUtensorMap &map_x, const CUtensor
                  cudaStream_t st);
 int pick_token_tile(const ew_pool *p, int B);
 int launch_gemm2(ew_pool *p, int layer, int B, cudaStream_t st);
-int launch_combine(ew_pool *p, int B, void *out, bool f32_out, cudaStream_t st);   // f32_out: fp32 partial sums (expert parallelism)
-int launch_round_bf16(const float *in, void *out, size_t n, cudaStream_t st);
+// out_mode 0: bf16 result; 1: fp32 partial sums (expert parallelism); 2: fp32 partial sums stored into every rank's
+// gather buffer (`out` = device array of ep_size pointers)
+int launch_combine(ew_pool *p, int B, void *out, int out_mode, cudaStream_t st);
+int launch_round_bf16(const float *in, int n_parts, void *out, size_t n, cudaStream_t st);   // out = bf16(in[0] + ... + in[n_parts - 1])
 int launch_reroute(ew_pool *p, int layer, const int32_t *ids, const int32_t *aid, int B, int32_t *slots,
                    int32_t *counts, cudaStream_t st);
 int launch_route_logits(ew_pool *p, int layer, const float *logits, const int32_t *aid, int B, int32_t *topk_ids,

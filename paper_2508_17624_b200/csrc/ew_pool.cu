@@ -600,13 +600,14 @@ static ew_status_t note_forward(ew_pool *p, cudaStream_t st) {
         }                                                                                      \
     } while (0)
 
-// The forward.  f32_out: `out` receives this rank's fp32 partial sums instead of the rounded bf16 result.
+// The forward.  out_mode 0: `out` receives the rounded bf16 result; 1: this rank's fp32 partial sums; 2: `out` is a device
+// array of ep_size gather buffers, each of which receives the partial sums in block ep_rank.
 static ew_status_t forward_impl(ew_pool_t *p, int32_t layer, const void *x, const int32_t *aid, int32_t B, void *out,
-                                bool f32_out, void *cuda_stream, int32_t *topk_ids, float *topk_w, int32_t *slot_ids,
+                                int out_mode, void *cuda_stream, int32_t *topk_ids, float *topk_w, int32_t *slot_ids,
                                 int32_t *counts, int32_t *inv, int32_t *offsets) {
     if (!p || layer < 0 || layer >= p->cfg.num_layers || B < 0 || B > p->cfg.max_tokens) return EW_ERR_INVALID_ARG;
     if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
-    if (!f32_out && p->cfg.ep_size > 1) {
+    if (out_mode == 0 && p->cfg.ep_size > 1) {
         set_last_error("this pool holds one rank's share of the experts: call ew_moe_forward_partial, add the ranks' partial sums, then ew_ep_finish");
         return EW_ERR_INVALID_ARG;
     }
@@ -671,7 +672,7 @@ static ew_status_t forward_impl(ew_pool_t *p, int32_t layer, const void *x, cons
     PROF_MARK(3);
     LAUNCH_TRY(launch_gemm2(p, layer, B, st));
     PROF_MARK(4);
-    LAUNCH_TRY(launch_combine(p, B, out, f32_out, st));
+    LAUNCH_TRY(launch_combine(p, B, out, out_mode, st));
     p->counts_clean = true;                             // the combine kernel zeroes the counters when it is done with them
     p->last_forward_kernels = p->self_plan ? 4 : p->fat ? 7 : 5;
     PROF_MARK(5);
@@ -683,17 +684,35 @@ extern "C" ew_status_t ew_moe_forward_debug(ew_pool_t *p, int32_t layer, const v
                                             int32_t B, void *out, void *cuda_stream, int32_t *topk_ids,
                                             float *topk_w, int32_t *slot_ids, int32_t *counts, int32_t *inv,
                                             int32_t *offsets) {
-    return forward_impl(p, layer, x, aid, B, out, false, cuda_stream, topk_ids, topk_w, slot_ids, counts, inv, offsets);
+    return forward_impl(p, layer, x, aid, B, out, 0, cuda_stream, topk_ids, topk_w, slot_ids, counts, inv, offsets);
 }
 
 extern "C" ew_status_t ew_moe_forward(ew_pool_t *p, int32_t layer, const void *x, const int32_t *aid, int32_t B,
                                       void *out, void *cuda_stream) {
-    return forward_impl(p, layer, x, aid, B, out, false, cuda_stream, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr);
+    return forward_impl(p, layer, x, aid, B, out, 0, cuda_stream, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr);
 }
 
 extern "C" ew_status_t ew_moe_forward_partial(ew_pool_t *p, int32_t layer, const void *x, const int32_t *aid, int32_t B,
                                               float *partial, void *cuda_stream) {
-    return forward_impl(p, layer, x, aid, B, partial, true, cuda_stream, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr);
+    return forward_impl(p, layer, x, aid, B, partial, 1, cuda_stream, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr);
+}
+
+extern "C" ew_status_t ew_moe_forward_scatter(ew_pool_t *p, int32_t layer, const void *x, const int32_t *aid, int32_t B,
+                                              float *const *gather_bufs, void *cuda_stream) {
+    return forward_impl(p, layer, x, aid, B, (void *)gather_bufs, 2, cuda_stream, nullptr, nullptr, nullptr, nullptr, nullptr,
+                        nullptr);
+}
+
+extern "C" ew_status_t ew_ep_finish_gathered(ew_pool_t *p, const float *gathered, int32_t B, void *out, void *cuda_stream) {
+    if (!p || B < 0) return EW_ERR_INVALID_ARG;
+    if (p->cfg.device < 0) return EW_ERR_NO_DEVICE;
+    if (B == 0) return EW_OK;
+    if (!gathered || !out || ((uintptr_t)gathered & 15) || ((uintptr_t)out & 7)) return EW_ERR_INVALID_ARG;
+    DeviceGuard guard;
+    CU_TRY(guard.enter(p->cfg.device));
+    LAUNCH_TRY(launch_round_bf16(gathered, p->cfg.ep_size > 1 ? p->cfg.ep_size : 1, out, (size_t)B * p->cfg.hidden,
+                                 (cudaStream_t)cuda_stream));
+    return EW_OK;
 }
 
 extern "C" ew_status_t ew_ep_finish(ew_pool_t *p, const float *summed, int32_t B, void *out, void *cuda_stream) {
@@ -703,7 +722,7 @@ extern "C" ew_status_t ew_ep_finish(ew_pool_t *p, const float *summed, int32_t B
     if (!summed || !out || ((uintptr_t)summed & 15) || ((uintptr_t)out & 7)) return EW_ERR_INVALID_ARG;
     DeviceGuard guard;
     CU_TRY(guard.enter(p->cfg.device));
-    LAUNCH_TRY(launch_round_bf16(summed, out, (size_t)B * p->cfg.hidden, (cudaStream_t)cuda_stream));
+    LAUNCH_TRY(launch_round_bf16(summed, 1, out, (size_t)B * p->cfg.hidden, (cudaStream_t)cuda_stream));
     return EW_OK;
 }
 

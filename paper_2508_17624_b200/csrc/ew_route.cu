@@ -520,10 +520,14 @@ __global__ void __launch_bounds__(256) permute_kernel(const int32_t *slot_ids, c
 // sum of the shared experts' outputs (GEMM-2 chains them along K); the routed rows start at Yb = B (0 without shared
 // experts).
 // ------------------------------------------------------------------------------------------------
-template <bool F32OUT>
+// OUT = 0: rounded bf16 result.  1: this rank's fp32 partial sums (expert parallelism, added by an all-reduce).
+// 2: the same partial sums stored straight into every rank's gather buffer - `out` is a device array of ep_size
+// pointers, buffer r' = rank r''s [ep_size][B][H] fp32 area, of which this rank fills block ep_rank: the exchange step
+// of the layer done by the kernel that produces the data, with plain (peer) stores.
+template <int OUT>
 __global__ void __launch_bounds__(256) combine_kernel(const float4 *y, const int32_t *inv,
                                                       const float *w, int B, int k, int H, int S,
-                                                      void *out, int32_t *counts, int P) {
+                                                      void *out, int32_t *counts, int P, int ep_size, int ep_rank) {
     __shared__ int32_t rows[32];
     __shared__ float wts[32];
     const int t = blockIdx.x;
@@ -552,7 +556,11 @@ __global__ void __launch_bounds__(256) combine_kernel(const float4 *y, const int
             const float4 a = y[(size_t)t * hv + v];
             acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
         }
-        if (F32OUT) {                                   // this rank's partial sum, rounded after the sum over ranks
+        if (OUT == 2) {
+            float4 *const *dst = reinterpret_cast<float4 *const *>(out);
+            const size_t o = ((size_t)ep_rank * B + t) * hv + v;
+            for (int r = 0; r < ep_size; ++r) dst[r][o] = acc;
+        } else if (OUT == 1) {                          // this rank's partial sum, rounded after the sum over ranks
             reinterpret_cast<float4 *>(out)[(size_t)t * hv + v] = acc;
         } else {
             const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
@@ -564,11 +572,16 @@ __global__ void __launch_bounds__(256) combine_kernel(const float4 *y, const int
     }
 }
 
-// out[i] = bf16(partial[i]): the single rounding of the layer's output, after the partial sums of all ranks have been
-// added (expert parallelism)
-__global__ void __launch_bounds__(256) round_bf16_kernel(const float4 *in, uint2 *out, size_t n4) {
+// out[i] = bf16(in[0][i] + in[1][i] + ... + in[R-1][i]), added in that order (R = 1: the single rounding of a sum
+// that an all-reduce has already formed; R > 1: the gathered partial sums of all ranks, the same bits on every rank
+// and in every run)
+__global__ void __launch_bounds__(256) round_bf16_kernel(const float4 *in, uint2 *out, size_t n4, int R) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
-        const float4 a = in[i];
+        float4 a = in[i];
+        for (int r = 1; r < R; ++r) {
+            const float4 b = in[(size_t)r * n4 + i];
+            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        }
         const __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
         uint2 o;
         o.x = *reinterpret_cast<const uint32_t *>(&lo);
@@ -603,20 +616,21 @@ int launch_permute(ew_pool *p, int B, cudaStream_t st) {
                       (const int32_t *)p->ws.counts, A, p->ws.inv, p->ws.src_tok);
 }
 
-int launch_combine(ew_pool *p, int B, void *out, bool f32_out, cudaStream_t st) {
+int launch_combine(ew_pool *p, int B, void *out, int out_mode, cudaStream_t st) {
     const ew_config_t &c = p->cfg;
     const int S = p->sh_hi - p->sh_lo;                  // the shared experts this rank computes
-    if (f32_out)
-        return launch_pdl(combine_kernel<true>, dim3(B), dim3(256), 0, st, (const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B,
-                          c.top_k, c.hidden, S, out, p->ws.counts, p->P);
-    return launch_pdl(combine_kernel<false>, dim3(B), dim3(256), 0, st, (const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B,
-                      c.top_k, c.hidden, S, out, p->ws.counts, p->P);
+    const int R = c.ep_size > 1 ? c.ep_size : 1;
+    auto go = [&](auto kernel) {
+        return launch_pdl(kernel, dim3(B), dim3(256), 0, st, (const float4 *)p->ws.y, p->ws.inv, p->ws.topk_w, B, c.top_k,
+                          c.hidden, S, out, p->ws.counts, p->P, R, c.ep_rank);
+    };
+    return out_mode == 2 ? go(combine_kernel<2>) : out_mode == 1 ? go(combine_kernel<1>) : go(combine_kernel<0>);
 }
 
-int launch_round_bf16(const float *in, void *out, size_t n, cudaStream_t st) {
+int launch_round_bf16(const float *in, int n_parts, void *out, size_t n, cudaStream_t st) {
     const size_t n4 = n / 4;
     const int grid = (int)std::min<size_t>((n4 + 255) / 256, 148 * 8);
-    round_bf16_kernel<<<grid, 256, 0, st>>>((const float4 *)in, (uint2 *)out, n4);
+    round_bf16_kernel<<<grid, 256, 0, st>>>((const float4 *)in, (uint2 *)out, n4, n_parts);
     return (int)cudaGetLastError();
 }
 

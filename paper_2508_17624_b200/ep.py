@@ -10,8 +10,15 @@ slots a rank owns are backed by physical pages there.
 Exchange.  The paper does not describe one.  Under tensor-parallel attention every rank already holds the hidden
 states of all tokens, so no token travels: every rank routes all tokens (the router is replicated), computes the
 pairs whose expert it holds, and the ranks' fp32 partial sums are added by one all-reduce per layer; the sum is
-rounded to bf16 once.  All arithmetic of a rank runs in the library (`ew_moe_forward_partial`, `ew_ep_finish`);
-this module only places the all-reduce (torch.distributed: NCCL on GPUs) between the two calls.
+rounded to bf16 once.  All arithmetic of a rank runs in the library; this module only places the exchange between the
+library's calls.  Three forms of it:
+
+  forward           ew_moe_forward_partial -> all-reduce (torch.distributed; NCCL on GPUs) -> ew_ep_finish
+  forward_gathered  ew_moe_forward_partial -> all-gather -> ew_ep_finish_gathered: the partial sums are added in rank
+                    order on every rank, so the result has the same bits everywhere and in every run
+  forward_scatter   ew_moe_forward_scatter -> barrier -> ew_ep_finish_gathered: the combine kernel itself stores the
+                    partial sums into every rank's gather buffer over peer memory (no collective call on the data path);
+                    the caller supplies the peer-visible buffers and the barrier (e.g. from symmetric memory)
 """
 from typing import Optional, Tuple
 
@@ -66,3 +73,31 @@ class ExpertParallelLayer:
         if out is None:
             return self.pool.ep_finish(partial)
         return self.pool.ep_finish(partial, out)
+
+    def forward_gathered(self, layer: int, x, adapter_ids, out: Optional[object] = None):
+        """Same result up to the order of the fp32 additions, but deterministic: every rank adds the R partial sums in
+        rank order."""
+        import torch
+        partial = self.pool.moe_forward_partial(layer, x, adapter_ids)
+        world = self.world()
+        gathered = torch.empty((world,) + tuple(partial.shape), dtype=partial.dtype, device=partial.device)
+        if world > 1:
+            import torch.distributed as dist
+            dist.all_gather(list(gathered.unbind(0)), partial, group=self.group)     # block r = rank r's partial sums
+        else:
+            gathered[0].copy_(partial)
+        if out is None:
+            return self.pool.ep_finish_gathered(gathered)
+        return self.pool.ep_finish_gathered(gathered, out)
+
+    def forward_scatter(self, layer: int, x, adapter_ids, gather_ptrs, my_gather_buf, barrier, out: Optional[object] = None):
+        """The exchange inside the combine kernel.  `gather_ptrs`: device int64 tensor with the addresses of all ranks'
+        gather buffers (fp32 [R, B, H] each, peer-visible), `my_gather_buf`: this rank's own buffer as a tensor,
+        `barrier`: a callable that returns once every rank's scatter for this step has completed, ordered on the current
+        stream (with torch's symmetric memory: the handle's barrier).  Not exercised on more than one GPU in this
+        repository's tests; on one GPU the ranks are pools on the same device and the barrier is stream order."""
+        self.pool.moe_forward_scatter(layer, x, adapter_ids, gather_ptrs)
+        barrier()
+        if out is None:
+            return self.pool.ep_finish_gathered(my_gather_buf)
+        return self.pool.ep_finish_gathered(my_gather_buf, out)

@@ -117,6 +117,12 @@ class _OraclePool:
     def ep_finish(self, summed, out=None):
         return summed.to(torch.bfloat16)
 
+    def ep_finish_gathered(self, gathered, out=None):
+        acc = gathered[0].clone()
+        for r in range(1, gathered.shape[0]):          # rank order
+            acc += gathered[r]
+        return acc.to(torch.bfloat16)
+
 
 def _ep_worker(rank, world, port, out_dir):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
@@ -129,6 +135,8 @@ def _ep_worker(rank, world, port, out_dir):
     assert layer.world() == world
     out = layer.forward(0, x, aid)
     np.save(os.path.join(out_dir, f"out{rank}.npy"), out.view(torch.int16).numpy())
+    out_g = layer.forward_gathered(0, x, aid)
+    np.save(os.path.join(out_dir, f"gathered{rank}.npy"), out_g.view(torch.int16).numpy())
     dist.barrier()
     dist.destroy_process_group()
 
@@ -149,6 +157,12 @@ def test_two_gloo_ranks_add_up_to_the_oracle_layer(tmp_path):
     # bits, so a few results fall on the other side of a bf16 rounding boundary
     assert np.abs(got - want).max() <= 2.0 ** -7 * np.abs(want).max()
     assert (got != want).mean() < 0.02
+    # the all-gather form adds the partial sums in rank order on every rank: identical bits on both ranks, and the same
+    # closeness to the oracle
+    gath = [np.load(tmp_path / f"gathered{r}.npy") for r in range(world)]
+    assert np.array_equal(gath[0], gath[1])
+    got_g = torch.from_numpy(gath[0]).view(torch.bfloat16).float().numpy()
+    assert np.abs(got_g - want).max() <= 2.0 ** -7 * np.abs(want).max()
     # and no rank alone gives the answer: both hold experts the batch uses
     mask0 = ep.local_pair_mask(ids, cfg.num_experts, world, 0)
     assert mask0.any() and (~mask0).any()

@@ -130,7 +130,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
     const bool self = sp.counts != nullptr;
     constexpr int kScanWarp = 2;
     int n_mine = 0;
-    if (!self) pdl_launch_dependents();
+    // GEMM-1 of a self-planned forward releases GEMM-2 after its own wait (below).  GEMM-2 of such a forward does not
+    // release the combine kernel early at all (it is launched when GEMM-2 has finished): with the combine kernel's
+    // CTAs resident beside GEMM-2's, the decode layer measured 0.2876 instead of 0.2815 ms.
+    if (!self && !sp.hold_dependents) pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -447,7 +450,7 @@ fat_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
                      "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
-    pdl_launch_dependents();
+    if (GLU) pdl_launch_dependents();                 // (variant: GEMM-2's pair kernel does not release the combine kernel early)
     tc_fence_before();
     __syncthreads();
     cluster_sync_all();                               // the peer's barriers and TMEM are ready too
@@ -691,6 +694,7 @@ void self_limits(int *cap, size_t *scratch_bytes) {
 
 plan::SelfPlan self_plan_args(const ew_pool *p, int B, int pass) {
     plan::SelfPlan sp = {};
+    sp.hold_dependents = (pass == 1 && !p->fat) ? 1 : 0;      // GEMM-2's weight-streaming kernel followed by the combine kernel
     if (!p->self_plan) return sp;
     const ew_config_t &c = p->cfg;
     sp.counts = p->ws.counts;

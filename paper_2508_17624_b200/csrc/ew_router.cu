@@ -60,6 +60,7 @@ struct RouterArgs {
     int B, H, M, k, N, renormalize;
     float scale;
     int stages, tmem_cols, pi_in_smem, tok_tile, atoms;
+    int hold_dependents = 0;   // do not release the next kernel in the stream before this one has finished
     int big_quad;          // 64- and 128-token tiles: four lanes per token and a histogram per CTA (needs room in the drained ring)
     int P;                 // slots of the pool (size of the counters)
     int ksplit;            // CTAs per cluster that share one token tile, each with 1/ksplit of K (1: no cluster)
@@ -271,7 +272,7 @@ router_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
     }
     if (A.pi_in_smem)
         for (int i = threadIdx.x; i < A.N * M; i += blockDim.x) pi_s[i] = A.pi[i];
-    pdl_launch_dependents();
+    if (!A.hold_dependents) pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -668,6 +669,10 @@ int launch_route(ew_pool *p, int layer, const void *x, const int32_t *aid, int B
     A.counts = p->ws.counts; A.err = p->ws.err;
     A.slot_tok = p->self_plan ? p->ws.slot_tok : nullptr;
     A.own_lo = p->own_lo; A.own_hi = p->own_hi;
+    // followed by the planning kernel: not released early (its CTAs, resident beside this kernel's and waiting, cost the
+    // decode layer 3 us and the prefill layer 4 us); followed by GEMM-1 (self-planned forwards): released at once,
+    // GEMM-1 sets itself up and rehearses its item derivation meanwhile on the SMs this kernel leaves free
+    A.hold_dependents = p->self_plan ? 0 : 1;
     return router_launch(p, layer, x, g, A, true, st);
 }
 

@@ -33,6 +33,8 @@
 // issuing work, lets its copies in flight land, frees its TMEM and returns.
 #include <cuda_bf16.h>
 
+#include <cstdlib>
+
 #include "ew_internal.h"
 #include "ew_plan.cuh"
 #include "ew_tc.cuh"
@@ -133,7 +135,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
     // GEMM-1 of a self-planned forward releases GEMM-2 after its own wait (below).  GEMM-2 of such a forward does not
     // release the combine kernel early at all (it is launched when GEMM-2 has finished): with the combine kernel's
     // CTAs resident beside GEMM-2's, the decode layer measured 0.2876 instead of 0.2815 ms.
-    if (!self && !sp.hold_dependents) pdl_launch_dependents();
+    if (!self && !sp.hold_dependents && !sp.release_after_wait) pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -159,6 +161,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
     } else {
         // every gridDim.x-th item of the planning kernel's list
         pdl_wait();
+        if (sp.release_after_wait) pdl_launch_dependents();     // the CTA-pair kernel of this GEMM may start without a wait of its own
         const int n_items = *reinterpret_cast<const volatile int32_t *>(n_items_ptr);
         n_mine = n_items > (int)blockIdx.x ? (n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
     }
@@ -411,7 +414,7 @@ template <bool GLU>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GLU ? kFatThreadsGlu : kThreads, 1)
 fat_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
                 const GemmItem *items, const int32_t *n_items_ptr, int K, int out_cols, void *out, int *err,
-                const uint8_t *x_rows, const int32_t *src_tok, int n_x_rows) {
+                const uint8_t *x_rows, const int32_t *src_tok, int n_x_rows, int early_start) {
     using C = FatCfg;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -456,7 +459,11 @@ fat_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
     cluster_sync_all();                               // the peer's barriers and TMEM are ready too
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
-    pdl_wait();                                       // the item list and the token rows come from earlier kernels
+    // The item list and the activations come from earlier kernels.  early_start: the weight-streaming kernel of the same
+    // GEMM, this kernel's predecessor, released it only after its own wait (so everything before THAT kernel is
+    // complete, which is all this kernel reads) and still works on its last items: this kernel starts on the SMs it has
+    // left instead of idling through its tail, and waits for it at the end, so that whoever comes next can rely on both.
+    if (!early_start) pdl_wait();
     const int n_items = *reinterpret_cast<const volatile int32_t *>(n_items_ptr);
 
     if (warp == 0) {
@@ -645,12 +652,19 @@ fat_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
         long long t0 = clock64();
         while (clock64() - t0 < 2000000ll) {}
     }
+    if (early_start) pdl_wait();                      // this grid is complete only when its predecessor is
     tc_fence_before();
     __syncthreads();
     cluster_sync_all();                               // neither CTA leaves while the other may still touch it
     tc_fence_after();
     if (warp == 1)
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+}
+
+// EW_DISABLE_TAIL_OVERLAP=1: the CTA-pair kernel waits for the weight-streaming kernel of its GEMM before it starts.
+bool tail_overlap_enabled() {
+    static const bool on = [] { const char *e = getenv("EW_DISABLE_TAIL_OVERLAP"); return !(e && e[0] == '1'); }();
+    return on;
 }
 
 template <bool GLU>
@@ -670,8 +684,9 @@ int launch_fat(ew_pool *p, const CUtensorMap &mw, const CUtensorMap &ma, const G
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl_enabled() ? 2 : 1;
+    // (with the launch overlap switched off the kernels run one after the other anyway)
     return (int)cudaLaunchKernelEx(&cfg, fat_gemm_kernel<GLU>, mw, ma, items, n_items, K, out_cols, out, p->ws.err,
-                                   (const uint8_t *)x_rows, (const int32_t *)p->ws.src_tok, n_x_rows);
+                                   (const uint8_t *)x_rows, (const int32_t *)p->ws.src_tok, n_x_rows, tail_overlap_enabled() ? 1 : 0);
 }
 
 template <int NT, bool GLU>
@@ -695,6 +710,7 @@ void self_limits(int *cap, size_t *scratch_bytes) {
 plan::SelfPlan self_plan_args(const ew_pool *p, int B, int pass) {
     plan::SelfPlan sp = {};
     sp.hold_dependents = (pass == 1 && !p->fat) ? 1 : 0;      // GEMM-2's weight-streaming kernel followed by the combine kernel
+    sp.release_after_wait = (p->fat && tail_overlap_enabled()) ? 1 : 0;   // followed by the CTA-pair kernel of the same GEMM
     if (!p->self_plan) return sp;
     const ew_config_t &c = p->cfg;
     sp.counts = p->ws.counts;

@@ -162,6 +162,7 @@ struct SelfPlan {
     int pass;                    // 0: GEMM-1 (+ SwiGLU), 1: GEMM-2
     int rehearse;                // GEMM-1: run the planning code once before the wait for the router kernel (see derive_items)
     int hold_dependents;         // the kernel does not release its dependent kernel early (set when that is the combine kernel)
+    int release_after_wait;      // the kernel releases its dependent only after its own wait (set when that is the CTA-pair kernel of the same GEMM)
     // GEMM-1 only: its CTAs also publish what the combine step (and the debugging outputs) need
     const int32_t *slot_ids, *rank;      // [B*k] from the router kernel
     int32_t *offsets, *inv;              // out: [P + 1] exclusive scan of the counts, [B*k] pair -> slot-contiguous row

@@ -162,10 +162,12 @@ def test_slot_address_reads_back_the_loaded_weights():
     pool.destroy()
 
 
-@pytest.mark.parametrize("switch", ["EW_DISABLE_PDL", "EW_DISABLE_FAT", "EW_DISABLE_KSPLIT", "EW_DISABLE_SELFPLAN"])
+@pytest.mark.parametrize("switch", ["EW_DISABLE_PDL", "EW_DISABLE_FAT", "EW_DISABLE_KSPLIT", "EW_DISABLE_SELFPLAN",
+                                    "EW_DISABLE_TAIL_OVERLAP"])
 def test_debugging_switches_in_a_fresh_process(switch):
     """The environment switches of the library (plain stream order instead of overlapped launches; every block on
-    the weight-streaming kernel; no K split in the router; the planning kernel at every batch size) are read once per process, so each is exercised in a process of its own: the
+    the weight-streaming kernel; no K split in the router; the planning kernel at every batch size; the CTA-pair kernel
+    waiting for the weight-streaming kernel of its GEMM) are read once per process, so each is exercised in a process of its own: the
     tiny layer, the decode layer and a prefill-sized odd shape against the oracle."""
     import os
     import subprocess

@@ -122,6 +122,63 @@ def test_partial_sums_stored_into_every_ranks_gather_buffer(name, R, n_tokens):
         pool.destroy()
 
 
+def test_adapter_eviction_and_reload_on_rank_pools():
+    """Section 4.2's load / unload on pools that hold one rank's share: after an adapter is evicted on every rank its
+    tokens are served by the base experts (and flagged), pages return to each rank's free list, and a reload - into
+    reused pages - restores the adapter's output.  Outputs against the oracle with the matching adapter set."""
+    import torch
+    cfg = wl.CONFIGS["c0"]
+    R, n = 2, cfg.n_tokens
+    bank = wl.NoiseBank(cfg.seed)
+    x, aid = wl.gen_tokens(cfg), wl.gen_adapter_ids(cfg)
+    assert (aid == 1).any() and (aid == 0).any()
+    xd, ad = to_dev(x), to_dev(aid)
+    pools = []
+    tuned = None
+    for r in range(R):
+        pool = binding.Pool.from_config(cfg, ep_size=R, ep_rank=r)
+        tuned, bases = binding.load_model(pool, cfg, bank)
+        pools.append(pool)
+
+    def layer_output():
+        parts = [p.moe_forward_partial(0, xd, ad) for p in pools]
+        summed = parts[0].clone()
+        for part in parts[1:]:
+            summed += part
+        out = pools[0].ep_finish(summed)
+        torch.cuda.synchronize()
+        return bf16_to_f32(out)
+
+    def against_oracle(got, adapters):
+        olayer = oracle_layer(cfg, 0, bank, tuned, adapters=adapters)
+        ref, *_ = oracle.layer_forward(olayer, x, aid)
+        assert float(np.linalg.norm(got - ref) / np.linalg.norm(ref)) <= REL_L2_TOL
+        assert float(np.abs(got - ref).max()) <= MAX_ABS_TOL
+
+    full = layer_output()
+    against_oracle(full, None)
+    created = [p.stats()["pages_created_total"] for p in pools]
+    mapped = [p.stats()["pages_mapped"] for p in pools]
+    for p in pools:
+        p.unload_adapter(1)
+    without = layer_output()
+    for p in pools:
+        assert p.last_device_error() == 8           # EW_ERR_BAD_ADAPTER_ID_IN_BATCH: the evicted adapter's tokens were served as base tokens
+    against_oracle(without, [0])
+    assert np.abs(without - full).max() > 1e-3          # the adapter did matter
+    for p, m in zip(pools, mapped):
+        assert p.stats()["pages_mapped"] <= m
+    ew = wl.gen_adapter_layer(cfg, 1, 0, tuned[1][0], bank)
+    for p in pools:
+        p.load_adapter(1, np.array([len(tuned[1][0])], np.int32), tuned[1][0].astype(np.int32), ew.w_gate, ew.w_up, ew.w_down)
+    again = layer_output()
+    assert np.array_equal(again, full)
+    for p, c in zip(pools, created):
+        assert p.stats()["pages_created_total"] == c     # the reload reused the pages the eviction freed
+        assert p.last_device_error() == 0
+        p.destroy()
+
+
 def test_expert_parallel_layer_single_rank_on_gpu():
     """ExpertParallelLayer without a process group is the plain forward."""
     import torch

@@ -373,11 +373,15 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
 constexpr int kFatHalf = 128;
 constexpr int kFatN = 256;          // accumulator columns per set
 
+// GEMM-1 (GLU) stages its bf16 output rows through shared memory (see the epilogue); GEMM-2 writes its fp32 rows
+// straight from registers with 32-byte stores and spends that shared memory on a seventh stage instead (its time fell
+// with every stage added: 511 / 491 / 476 us at 4 / 5 / 6 stages of the prefill layer, while GEMM-1 did not react).
+template <bool GLU>
 struct FatCfg {
     static constexpr int kStageBytes = 2 * kATileBytes;                         // 16 KiB of token rows + 16 KiB of weight rows
     static constexpr int kOutRowBytes = 128 + 16;                               // epilogue staging: 128 bytes of a row, padded against bank conflicts
-    static constexpr int kOutBytes = 4 * 32 * kOutRowBytes;                     // 32 rows per epilogue warp
-    static constexpr int kStages = (kSmemBudget - kOutBytes) / kStageBytes > 8 ? 8 : (kSmemBudget - kOutBytes) / kStageBytes;   // 6
+    static constexpr int kOutBytes = GLU ? 4 * 32 * kOutRowBytes : 0;           // 32 rows per epilogue warp
+    static constexpr int kStages = (kSmemBudget - kOutBytes) / kStageBytes > 8 ? 8 : (kSmemBudget - kOutBytes) / kStageBytes;   // 6 / 7
     static constexpr int kSmemBytes = kStages * kStageBytes + kOutBytes + 1024 + 512;
 };
 constexpr int kFatThreadsGlu = kThreads + kGatherThreads + 32;                  // GEMM-1: gather warps and a relay warp
@@ -415,7 +419,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GLU ? kFatThreadsGlu
 fat_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
                 const GemmItem *items, const int32_t *n_items_ptr, int K, int out_cols, void *out, int *err,
                 const uint8_t *x_rows, const int32_t *src_tok, int n_x_rows, int early_start) {
-    using C = FatCfg;
+    using C = FatCfg<GLU>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -578,7 +582,7 @@ fat_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
         // per store instruction, so each warp passes 128 bytes of its 32 rows through shared memory and stores them
         // with eight lanes per row (four whole 128-byte pieces per instruction).
         const int lg = warp & 3;
-        uint8_t *stg = out_stage + lg * 32 * C::kOutRowBytes;
+        uint8_t *stg = out_stage + lg * 32 * C::kOutRowBytes;                // (GEMM-1 only; GEMM-2 has no staging area)
         uint8_t *stg_w = stg + lane * C::kOutRowBytes;                       // this thread's row of the staging tile
         const uint8_t *stg_r = stg + (lane >> 3) * C::kOutRowBytes + (lane & 7) * 16;   // row lane/8 (+4 per step), 16-byte piece lane%8
         constexpr int kElem = GLU ? 2 : 4;                                   // bytes per output element
@@ -620,12 +624,21 @@ fat_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant
                                 *reinterpret_cast<uint4 *>(stg_w + 64 * h + 16 * q) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
                         }
                     } else {
+                        // GEMM-2: the thread's 32 fp32 columns (128 bytes of its row) go out as four 32-byte stores, whole
+                        // sectors each; no staging
                         uint32_t v[32];
                         tc_ld32(t0 + e0, v);
                         tc_wait_ld();
+                        if (lane < rows_here) {
+                            uint8_t *gp = gbase + (size_t)lane * row_bytes + (size_t)e0 * kElem;
 #pragma unroll
-                        for (int q = 0; q < 8; ++q)
-                            *reinterpret_cast<uint4 *>(stg_w + 16 * q) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                            for (int q = 0; q < 4; ++q)
+                                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(gp + 32 * q), "r"(v[8 * q]),
+                                             "r"(v[8 * q + 1]), "r"(v[8 * q + 2]), "r"(v[8 * q + 3]), "r"(v[8 * q + 4]), "r"(v[8 * q + 5]),
+                                             "r"(v[8 * q + 6]), "r"(v[8 * q + 7])
+                                             : "memory");
+                        }
+                        continue;
                     }
                     __syncwarp();
                     // eight lanes per row: lane l writes bytes [16 (l%8), +16) of row l/8 + 4 i
@@ -673,7 +686,7 @@ int launch_fat(ew_pool *p, const CUtensorMap &mw, const CUtensorMap &ma, const G
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p->sm_count & ~1);
     cfg.blockDim = dim3(GLU ? kFatThreadsGlu : kThreads);
-    cfg.dynamicSmemBytes = FatCfg::kSmemBytes;
+    cfg.dynamicSmemBytes = FatCfg<GLU>::kSmemBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -758,8 +771,8 @@ int gemm_setup(ew_pool *) {
     int rc = 0;
     rc |= setup_one<32, true>() | setup_one<64, true>() | setup_one<128, true>();
     rc |= setup_one<32, false>() | setup_one<64, false>() | setup_one<128, false>();
-    rc |= (int)cudaFuncSetAttribute(fat_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FatCfg::kSmemBytes);
-    rc |= (int)cudaFuncSetAttribute(fat_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FatCfg::kSmemBytes);
+    rc |= (int)cudaFuncSetAttribute(fat_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FatCfg<true>::kSmemBytes);
+    rc |= (int)cudaFuncSetAttribute(fat_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FatCfg<false>::kSmemBytes);
     if (rc) set_last_error("cudaFuncSetAttribute(max dynamic shared memory) failed for a grouped GEMM kernel");
     return rc;
 }

@@ -838,6 +838,46 @@ def test_back_to_back_forwards_with_changing_inputs(name):
     pool.destroy()
 
 
+def test_back_to_back_forwards_of_every_form_on_one_pool():
+    """One pool, batches of very different sizes queued back to back without host synchronisation: each call picks its
+    own form of the forward (four kernels for the decode-sized ones, seven for the prefill-sized ones) and leaves
+    tables of the other forms behind in the shared workspace.  Every output against the oracle, and against the same
+    call made alone."""
+    import torch
+    cfg = wl.CONFIGS["c0"]
+    sizes = [7, 3000, 64, 1500, 256, 2999, 1, 640]
+    bank = wl.NoiseBank(cfg.seed)
+    pool = binding.Pool.from_config(cfg, max_tokens=max(sizes))
+    tuned, bases = binding.load_model(pool, cfg, bank)
+    olayer = oracle_layer(cfg, 0, bank, tuned, base=bases[0])
+    rng = np.random.default_rng(11)
+    batches, alone, forms = [], [], []
+    for n in sizes:
+        x = wl.f32_to_bf16_bits(rng.standard_normal((n, cfg.hidden)).astype(np.float32))
+        aid = rng.integers(-1, cfg.max_adapters, size=n).astype(np.int32)
+        r = pool.moe_forward_debug(0, to_dev(x), to_dev(aid))
+        torch.cuda.synchronize()
+        forms.append(pool.stats()["last_forward_kernels"])
+        ids, w, slots, _ = check_routing(cfg, olayer, x, aid, r)
+        check_output(olayer, x, slots, w, bf16_to_f32(r["out"]))
+        batches.append((to_dev(x), to_dev(aid)))
+        alone.append(r["out"].clone())
+    assert 4 in forms and 7 in forms
+    outs = [torch.empty_like(b[0]) for b in batches]
+    busy = torch.empty(1 << 28, dtype=torch.uint8, device="cuda")
+    for rep in range(4):
+        busy.zero_()
+        order = rng.permutation(len(batches))
+        for i in order:
+            pool.moe_forward(0, batches[i][0], batches[i][1], outs[i])
+        torch.cuda.synchronize()
+        for i in range(len(batches)):
+            assert torch.equal(outs[i], alone[i]), (rep, i, sizes[i])
+            outs[i].zero_()
+    assert pool.last_device_error() == 0
+    pool.destroy()
+
+
 def test_forwards_on_two_streams_share_the_workspace_in_order():
     """One pool, two streams, no host synchronisation between the calls: the pool makes a forward wait for the one
     issued before it on the other stream, so the single workspace is never used by two forwards at once."""
